@@ -1,0 +1,230 @@
+"""Pins for the CPU oracle: every check compares it with something that is not the
+oracle (brute-force dense algebra, closed forms, a literal sort, invariants)."""
+import numpy as np
+import pytest
+
+from oracle import ref
+from tests.helpers import DenseSim, mag_key, topk_by_sort
+
+
+def rel(a, b):
+    return np.linalg.norm(np.asarray(a, np.float64) - b) / max(np.linalg.norm(b), 1e-300)
+
+
+# ----------------------------------------------------------------- Top-k (Section 3.1)
+def _check_topk(a, k):
+    a = np.asarray(a, np.float32)
+    want_i, want_v = topk_by_sort(a, k)
+    for full in (False, True):
+        got_i, got_v = ref.topk(a, k, fullsort=full)
+        assert np.array_equal(got_i, want_i)
+        assert np.array_equal(got_v.view(np.uint32), want_v.view(np.uint32))
+
+
+def test_topk_random():
+    rng = np.random.default_rng(1)
+    for d, k in ((1, 1), (7, 3), (1000, 10), (4097, 4097), (50_000, 500)):
+        _check_topk(rng.standard_normal(d), k)
+
+
+def test_topk_ties_go_to_lower_index():
+    a = np.full(100, 2.5, np.float32)
+    idx, _ = ref.topk(a, 7)
+    assert idx.tolist() == list(range(7))
+    # +v and -v have the same magnitude: order decided by index alone
+    a = np.array([1.0, -3.0, 3.0, -3.0, 0.5, 3.0], np.float32)
+    idx, val = ref.topk(a, 2)
+    assert idx.tolist() == [1, 2] and val.tolist() == [-3.0, 3.0]
+    idx, _ = ref.topk(a, 3)
+    assert idx.tolist() == [1, 2, 3]
+    rng = np.random.default_rng(2)
+    _check_topk(rng.integers(-3, 4, 5000).astype(np.float32), 1234)
+
+
+def test_topk_zero_denormal_inf_nan_order():
+    tiny = np.float32(1e-45)  # smallest denormal
+    a = np.array([0.0, -0.0, tiny, -tiny, 1.0, np.inf, -np.inf, np.nan], np.float32)
+    # magnitude order by bit pattern: nan > inf > 1 > denormal > zero
+    assert ref.topk(a, 1)[0].tolist() == [7]
+    assert ref.topk(a, 3)[0].tolist() == [5, 6, 7]
+    assert ref.topk(a, 4)[0].tolist() == [4, 5, 6, 7]
+    assert ref.topk(a, 6)[0].tolist() == [2, 3, 4, 5, 6, 7]
+    assert ref.topk(a, 7)[0].tolist() == [0, 2, 3, 4, 5, 6, 7]  # +0 and -0 tie: lower index
+    _check_topk(a, 5)
+
+
+def test_topk_rejects_bad_arguments():
+    a = np.zeros(4, np.float32)
+    with pytest.raises(ValueError):
+        ref.topk(a, 5)
+    with pytest.raises(ValueError):
+        ref.topk(a, 0)
+
+
+# ------------------------------------------- error feedback (Algorithm 1, lines 5-7)
+def test_error_feedback_invariant_bitwise():
+    rng = np.random.default_rng(3)
+    d, m, k = 3001, 4, 37
+    o = ref.RefEFCP(d, m, k, 1e-3)
+    e_prev = np.zeros(d, np.float32)
+    for t in range(9):
+        g = (rng.standard_normal(d) * np.exp(rng.standard_normal(d))).astype(np.float32)
+        o.step(g)
+        a = (e_prev + g).astype(np.float32)  # independent fp32 add
+        assert np.array_equal(o.accumulator().view(np.uint32), a.view(np.uint32))
+        idx, val = o.row(t % m)
+        want_i, want_v = topk_by_sort(a, k)
+        assert np.array_equal(idx, want_i) and np.array_equal(val.view(np.uint32), want_v.view(np.uint32))
+        e = o.error()
+        assert np.all(e[idx].view(np.uint32) == 0)  # literally +0.0f at kept coordinates
+        dens = np.zeros(d, np.float32)
+        dens[idx] = val
+        assert np.array_equal((e + dens).view(np.uint32) & 0x7FFFFFFF, mag_key(a))
+        mask = np.ones(d, bool)
+        mask[idx] = False
+        assert np.array_equal(e[mask].view(np.uint32), a[mask].view(np.uint32))
+        e_prev = e
+    assert o.step_count == 9
+
+
+def test_k_equals_d_is_dense_mfac():
+    rng = np.random.default_rng(4)
+    d, m = 24, 5
+    o = ref.RefEFCP(d, m, d, 0.05)
+    G = np.zeros((m, d))
+    for t in range(8):
+        g = rng.standard_normal(d).astype(np.float32)
+        u = o.step(g)
+        assert not o.error().any()
+        G[t % m] = g
+        F = np.float32(0.05).astype(np.float64) * np.eye(d) + G.T @ G / m
+        assert rel(u, np.linalg.solve(F, g.astype(np.float64))) < 1e-6
+
+
+# --------------------------- inverse-Fisher-vector product (Section 2.1, Eq. 2) by brute force
+@pytest.mark.parametrize("acc_mode", [False, True])
+@pytest.mark.parametrize("d,m,k,steps,lam", [
+    (64, 1, 9, 3, 1e-2), (96, 2, 17, 5, 1e-3), (128, 4, 13, 11, 1e-4),
+    (256, 8, 40, 6, 1e-3),  # fewer steps than rows: unwritten rows are zero gradients
+    (200, 8, 21, 20, 1e-2),  # wraps twice
+])
+def test_update_matches_dense_solve(d, m, k, steps, lam, acc_mode):
+    rng = np.random.default_rng(d + m)
+    flags = ref.RHS_ACCUMULATOR if acc_mode else ref.RHS_COMPRESSED
+    o = ref.RefEFCP(d, m, k, lam, flags)
+    sim = DenseSim(d, m, k, lam, rhs_accumulator=acc_mode)
+    scale = np.exp(rng.standard_normal(d))
+    for t in range(steps):
+        g = (scale * rng.standard_normal(d)).astype(np.float32)
+        u = o.step(g)
+        want = sim.step(g)
+        assert np.array_equal(o.error().view(np.uint32), sim.e.view(np.uint32))
+        assert rel(u, want) < 2e-6, (t, rel(u, want))
+        # residual of the defining linear system, in dense fp64
+        # (u is rounded to fp32, so the bound is the rounding of u pushed through F)
+        F, x = sim.last["F"], sim.last["x"]
+        r = F @ u.astype(np.float64) - x
+        bound = 2.0 ** -23 * np.linalg.norm(np.abs(F) @ np.abs(u.astype(np.float64)))
+        assert np.linalg.norm(r) <= bound + 1e-6 * np.linalg.norm(x)
+        if not acc_mode:
+            assert rel(o.update_rowform(), want) < 2e-6
+    assert np.allclose(o.gram(), o.gram_full(), rtol=1e-13, atol=0)
+    assert np.allclose(o.gram(), sim.G @ sim.G.T, rtol=1e-12, atol=1e-12)
+
+
+def test_m1_closed_form():
+    # m = 1: F^-1 x = x/lam - g (g.x) / (lam (m lam + g.g))
+    rng = np.random.default_rng(5)
+    d, k, lam = 50, 6, np.float32(0.3)
+    g = rng.standard_normal(d).astype(np.float32)
+    o = ref.RefEFCP(d, 1, k, lam)
+    u = o.step(g)
+    idx, val = topk_by_sort(g, k)
+    c = np.zeros(d)
+    c[idx] = val
+    L = float(lam)
+    want = c / L - c * (c @ c) / (L * (L + c @ c))
+    assert rel(u, want) < 1e-6
+
+
+def test_disjoint_supports_closed_form():
+    # rows with disjoint supports: S diagonal, coef_j = p_j / (lam (m lam + |g_j|^2))
+    m, lam = 6, 1e-2
+    n2 = np.array([3.0, 0.5, 7.0, 0.0, 2.0, 11.0])
+    p = np.array([1.0, -2.0, 0.3, 0.0, 5.0, -1.0])
+    want = p / (lam * (m * lam + n2))
+    assert np.allclose(ref.woodbury_coef(np.diag(n2), p, lam), want, rtol=1e-13)
+    assert np.allclose(ref.wsm_coef(np.diag(n2), p, lam), want, rtol=1e-12)
+
+
+def test_large_lambda_limit_is_scaled_identity():
+    rng = np.random.default_rng(6)
+    d, m, k, lam = 300, 4, 30, np.float32(1e8)
+    o = ref.RefEFCP(d, m, k, lam)
+    for _ in range(6):
+        g = rng.standard_normal(d).astype(np.float32)
+        u = o.step(g)
+    idx, val = o.row(5 % m)
+    x = np.zeros(d)
+    x[idx] = val
+    assert rel(u, x / float(lam)) < 1e-6
+
+
+def test_wsm_recursion_equals_woodbury_and_dense_recursion():
+    rng = np.random.default_rng(7)
+    for m, d, lam in ((1, 5, 0.1), (3, 10, 1e-2), (16, 40, 1e-3), (48, 64, 1e-4)):
+        G = rng.standard_normal((m, d))
+        x = rng.standard_normal(d)
+        S, p = G @ G.T, G @ x
+        c1 = ref.woodbury_coef(S, p, lam)
+        c2 = ref.wsm_coef(S, p, lam)
+        assert rel(c2, c1) < 1e-8
+        # literal dense rank-one recursion, F_0 = lam I, F_j = F_{j-1} + g_j g_j^T / m
+        Finv = np.eye(d) / lam
+        for j in range(m):
+            v = Finv @ G[j]
+            Finv = Finv - np.outer(v, v) / (m + G[j] @ v)
+        want = Finv @ x
+        for c in (c1, c2):
+            assert rel(x / lam - G.T @ c, want) < 1e-7
+
+
+def test_planted_mistakes_are_caught():
+    # dropping the 1/m factor, or using lam instead of m*lam on the diagonal, must
+    # disagree with the dense definition by far more than the pin tolerance.
+    rng = np.random.default_rng(8)
+    m, d, lam = 4, 20, 1e-2
+    G = rng.standard_normal((m, d))
+    x = rng.standard_normal(d)
+    S, p = G @ G.T, G @ x
+    want = np.linalg.solve(lam * np.eye(d) + G.T @ G / m, x)
+    good = x / lam - G.T @ ref.woodbury_coef(S, p, lam)
+    assert rel(good, want) < 1e-9
+    bad1 = x / lam - G.T @ (np.linalg.solve(lam * np.eye(m) + S, p) / lam)
+    assert rel(bad1, want) > 1e-3
+
+
+def test_oracle_rejects_bad_arguments():
+    for args in ((0, 1, 1, 1e-3), (4, 0, 1, 1e-3), (4, 1, 0, 1e-3), (4, 1, 5, 1e-3),
+                 (4, 1, 1, 0.0), (4, 1, 1, float("nan")), (2**31, 1, 1, 1e-3)):
+        with pytest.raises(ValueError):
+            ref.RefEFCP(*args)
+
+
+def test_thread_count_does_not_change_results():
+    import os
+    import subprocess
+    import sys
+    code = (
+        "import numpy as np, sys; sys.path.insert(0, %r)\n"
+        "from oracle import ref\n"
+        "rng=np.random.default_rng(0); o=ref.RefEFCP(5000,64,50,1e-4)\n"
+        "for t in range(70): u=o.step(rng.standard_normal(5000).astype(np.float32))\n"
+        "import hashlib; print(hashlib.sha1(u.tobytes()+o.gram().tobytes()).hexdigest())\n"
+    ) % os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    outs = set()
+    for n in ("1", "3"):
+        env = dict(os.environ, OMP_NUM_THREADS=n)
+        outs.add(subprocess.run([sys.executable, "-c", code], env=env, check=True,
+                                capture_output=True, text=True).stdout.strip())
+    assert len(outs) == 1
