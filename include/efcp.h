@@ -1,0 +1,132 @@
+/*
+ * efcp.h - C ABI of the B200 (sm_100a) EFCP / Sparse M-FAC step library.
+ *
+ * One handle owns the whole optimizer state of one parameter vector of
+ * dimension d on one GPU: the error-feedback buffer xi (Algorithm 1, line 2),
+ * the sparse ring buffer G = (I, V) of the last m compressed accumulators
+ * (Section 3.1, "Sparsity format for G"), the m x m scalar-product matrix
+ * S = G G^T (Section 2.1, "Scalar Products (SP)") and the inverse of
+ * m*lambda*I + S from which the coefficients of Eq. (2) are read.
+ *
+ * Conventions for every call
+ *   - returns EFCP_OK (0) or a negative EFCP_E* code; never throws, never aborts;
+ *   - "device" pointers are CUDA device pointers valid on the handle's device,
+ *     "host" pointers are ordinary host memory; nothing is retained after return
+ *     except by the asynchronous work that efcp_step enqueues on the stream;
+ *   - the caller owns grad, update and the stream; the handle owns all state and
+ *     scratch, allocated once in efcp_create* on the device current at that time.
+ *   - a handle is not thread-safe; steps on one handle are ordered by the stream.
+ */
+#ifndef EFCP_H_
+#define EFCP_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct efcp_ctx efcp_ctx;
+
+#define EFCP_OK        0
+#define EFCP_EINVAL   -1  /* bad argument (null pointer, size out of range, bad lambda)   */
+#define EFCP_ENOMEM   -2  /* device or host allocation failed                              */
+#define EFCP_ECUDA    -3  /* a CUDA runtime call or launch failed (efcp_last_cuda_error)  */
+#define EFCP_ENUMERIC -4  /* non-finite gradient entry, or a non-positive pivot in the
+                             m x m update (window numerically singular for this lambda)  */
+#define EFCP_ETIMEOUT -5  /* a bounded device-side wait gave up                            */
+#define EFCP_EINTERNAL -6 /* an internal consistency check failed (selection count != k)  */
+
+/* flags for efcp_create_ex */
+#define EFCP_RHS_COMPRESSED  0u /* u_t = A(c_t): precondition the compressed accumulator
+                                   (Algorithm 1, line 8) - the default                    */
+#define EFCP_RHS_ACCUMULATOR 1u /* precondition the full accumulator a_t = xi_t + c_t     */
+
+/*
+ * efcp_create / efcp_create_ex - Algorithm 1 lines 1-2: set up an empty window and
+ * xi_0 = 0 for dimension d, window length m, k kept entries per step (Top-k of
+ * Section 3.1, k given as a count) and damping lambda (F_0 = lambda I, Section 2.1).
+ * Requires 1 <= k <= d < 2^31, 1 <= m <= 4096, lambda finite and > 0.
+ * Rows not written yet count as zero gradients; the 1/m of the empirical Fisher
+ * always uses the capacity m.  *out receives the handle (NULL on failure).
+ */
+int efcp_create(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float lambda);
+int efcp_create_ex(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float lambda,
+                   uint32_t flags);
+
+/*
+ * efcp_step - Algorithm 1 lines 5-8 for one gradient:
+ *     a = xi + g                      (fp32, one rounding per coordinate)
+ *     c = TopK_k(a)                   (global over d, exact, ties to the lower index)
+ *     xi = a - c                      (kept coordinates become +0)
+ *     row (t-1) mod m of G = c        (indices ascending)
+ *     u = (lambda I + (1/m) G^T G)^-1 x,  x = c (default) or a (EFCP_RHS_ACCUMULATOR),
+ * the last line evaluated as Eq. (2), a linear combination of the window rows with
+ * coefficients obtained from S (Section 2.1).
+ *   grad   device, d floats, read only.
+ *   update device, d floats, every element overwritten; must not alias grad.
+ *   stream a cudaStream_t (NULL = default stream).  All work is enqueued on it and
+ *          the call returns without waiting.  Learning rate, weight decay and the
+ *          parameter update (Algorithm 1 line 9) are left to the caller.
+ * Errors detected on the device (EFCP_ENUMERIC, ...) are sticky and reported by
+ * efcp_status or the next efcp_get_* call.
+ */
+int efcp_step(efcp_ctx* ctx, const float* grad, float* update, void* stream);
+
+/*
+ * efcp_step_host - the same step for callers whose gradient and update live in host
+ * memory (pinned memory gives the best copy rate): copies grad to the device, runs
+ * the step, copies the update back, all on `stream`, and waits for the stream.
+ *   grad, update: host, d floats each.
+ */
+int efcp_step_host(efcp_ctx* ctx, const float* grad, float* update, void* stream);
+
+/* Frees all device and host memory of the handle (waits for the device first). */
+int efcp_destroy(efcp_ctx* ctx);
+
+/*
+ * State inspection (parity tests, checkpointing).  Each call waits for all work
+ * queued on the handle's device, then copies to host memory:
+ *   efcp_get_error : xi, d floats.
+ *   efcp_get_row   : ring slot `slot` (0 <= slot < m): k ascending indices and the k
+ *                    values.  A slot never written reads as indices 0..k-1, values 0.
+ *   efcp_get_gram  : S = G G^T, m*m doubles, row-major, exactly symmetric
+ *                    (Section 2.1: row and column i are replaced together).
+ *   efcp_get_weights: the m fp64 weights w of the last step's linear combination
+ *                    (update = x/lambda*[mode] + sum_r w_r row_r; in the default mode
+ *                    update = sum_r w_r row_r).
+ * Returns the sticky device status if it is an error, else EFCP_OK.
+ */
+int efcp_get_error(efcp_ctx* ctx, float* host_e);
+int efcp_get_row(efcp_ctx* ctx, int32_t slot, int32_t* host_idx, float* host_val);
+int efcp_get_gram(efcp_ctx* ctx, double* host_S);
+int efcp_get_weights(efcp_ctx* ctx, double* host_w);
+
+/* Number of completed efcp_step calls on this handle (-1 for a NULL handle). */
+int64_t efcp_step_count(efcp_ctx* ctx);
+
+/* Waits for the device and returns the sticky status (EFCP_OK or an error code). */
+int efcp_status(efcp_ctx* ctx);
+
+/* The cudaError_t recorded with the last EFCP_ECUDA on this handle (0 if none). */
+int efcp_last_cuda_error(efcp_ctx* ctx);
+
+/*
+ * Relative residual |m e_i - (m lambda I + S) w| / m of the last step's m x m solve
+ * (fp64), a drift monitor for the incrementally updated inverse.  Waits for the device.
+ */
+double efcp_last_residual(efcp_ctx* ctx);
+
+/* Device bytes a handle for (d, m, k) allocates (state + scratch); -1 if invalid. */
+int64_t efcp_state_bytes(int64_t d, int32_t m, int64_t k);
+
+/* Number of kernels one efcp_step launches for this handle. */
+int32_t efcp_launches_per_step(efcp_ctx* ctx);
+
+/* Static description of an EFCP_* code. */
+const char* efcp_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EFCP_H_ */

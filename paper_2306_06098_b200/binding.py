@@ -1,0 +1,157 @@
+"""Thin ctypes binding over libefcp.so (argument marshalling only).
+
+The names mirror include/efcp.h.  PyTorch is used for device memory and streams; every
+step of the method runs inside the CUDA library.  Importing this module fails loudly
+when the library has not been built (there is no fallback path).
+"""
+import ctypes as C
+import os
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "csrc", "libefcp.so")
+
+OK, EINVAL, ENOMEM, ECUDA, ENUMERIC, ETIMEOUT, EINTERNAL = 0, -1, -2, -3, -4, -5, -6
+RHS_COMPRESSED, RHS_ACCUMULATOR = 0, 1
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is missing: build it with `python -m paper_2306_06098_b200.build` "
+        "(nvcc, sm_100a). There is no CPU fallback.")
+
+_lib = C.CDLL(LIB_PATH)
+_vp, _i32, _i64, _f32, _u32 = C.c_void_p, C.c_int32, C.c_int64, C.c_float, C.c_uint32
+
+EXPORTS = {
+    "efcp_create": ([C.POINTER(_vp), _i64, _i32, _i64, _f32], C.c_int),
+    "efcp_create_ex": ([C.POINTER(_vp), _i64, _i32, _i64, _f32, _u32], C.c_int),
+    "efcp_step": ([_vp, _vp, _vp, _vp], C.c_int),
+    "efcp_step_host": ([_vp, _vp, _vp, _vp], C.c_int),
+    "efcp_destroy": ([_vp], C.c_int),
+    "efcp_get_error": ([_vp, _vp], C.c_int),
+    "efcp_get_row": ([_vp, _i32, _vp, _vp], C.c_int),
+    "efcp_get_gram": ([_vp, _vp], C.c_int),
+    "efcp_get_weights": ([_vp, _vp], C.c_int),
+    "efcp_step_count": ([_vp], _i64),
+    "efcp_status": ([_vp], C.c_int),
+    "efcp_last_cuda_error": ([_vp], C.c_int),
+    "efcp_last_residual": ([_vp], C.c_double),
+    "efcp_state_bytes": ([_i64, _i32, _i64], _i64),
+    "efcp_launches_per_step": ([_vp], _i32),
+    "efcp_strerror": ([C.c_int], C.c_char_p),
+}
+for _name, (_args, _res) in EXPORTS.items():
+    _fn = getattr(_lib, _name)  # AttributeError here = header and library out of sync
+    _fn.argtypes = _args
+    _fn.restype = _res
+
+
+class EfcpError(RuntimeError):
+    def __init__(self, code, where, cuda=0):
+        self.code = code
+        msg = _lib.efcp_strerror(code).decode()
+        super().__init__(f"{where}: {msg} (code {code}" + (f", cudaError {cuda})" if cuda else ")"))
+
+
+def strerror(code: int) -> str:
+    return _lib.efcp_strerror(code).decode()
+
+
+def state_bytes(d: int, m: int, k: int) -> int:
+    return int(_lib.efcp_state_bytes(d, m, k))
+
+
+def paper_state_bytes(d: int, m: int, k: int, value_bytes: int = 4) -> int:
+    """Footprint of Sparse M-FAC as the paper's appendix "Memory savings" counts it:
+    indices 4mk, values value_bytes*mk, error feedback 4d, SP result 4m, LCG result 4d."""
+    return 4 * m * k + value_bytes * m * k + 4 * d + 4 * m + 4 * d
+
+
+def _np_ptr(a: np.ndarray):
+    return a.ctypes.data_as(C.c_void_p)
+
+
+class Efcp:
+    """One optimizer state (efcp_ctx) on the current CUDA device."""
+
+    def __init__(self, d: int, m: int, k: int, lam: float, flags: int = RHS_COMPRESSED):
+        self._h = None
+        self.d, self.m, self.k, self.lam, self.flags = int(d), int(m), int(k), float(lam), flags
+        h = _vp()
+        rc = _lib.efcp_create_ex(C.byref(h), self.d, self.m, self.k, self.lam, flags)
+        if rc != OK:
+            raise EfcpError(rc, "efcp_create_ex")
+        self._h = h
+
+    def close(self):
+        if self._h:
+            _lib.efcp_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        self.close()
+
+    def _check(self, rc, where):
+        if rc != OK:
+            raise EfcpError(rc, where, _lib.efcp_last_cuda_error(self._h))
+
+    def step(self, grad: torch.Tensor, update: torch.Tensor, stream=None):
+        """efcp_step on device tensors (fp32, contiguous, d elements); asynchronous."""
+        assert grad.is_cuda and update.is_cuda and grad.dtype == update.dtype == torch.float32
+        assert grad.is_contiguous() and update.is_contiguous()
+        assert grad.numel() == self.d and update.numel() == self.d
+        s = torch.cuda.current_stream() if stream is None else stream
+        self._check(_lib.efcp_step(self._h, grad.data_ptr(), update.data_ptr(), s.cuda_stream),
+                    "efcp_step")
+        return update
+
+    def step_ptr(self, grad_ptr: int, update_ptr: int, stream_ptr: int = 0):
+        self._check(_lib.efcp_step(self._h, grad_ptr, update_ptr, stream_ptr), "efcp_step")
+
+    def step_host(self, grad: torch.Tensor, update: torch.Tensor, stream=None):
+        """efcp_step_host on host tensors (pinned preferred); returns when update is ready."""
+        assert not grad.is_cuda and not update.is_cuda
+        assert grad.dtype == update.dtype == torch.float32
+        assert grad.is_contiguous() and update.is_contiguous()
+        assert grad.numel() == self.d and update.numel() == self.d
+        s = torch.cuda.current_stream() if stream is None else stream
+        self._check(_lib.efcp_step_host(self._h, grad.data_ptr(), update.data_ptr(),
+                                        s.cuda_stream), "efcp_step_host")
+        return update
+
+    @property
+    def step_count(self) -> int:
+        return int(_lib.efcp_step_count(self._h))
+
+    @property
+    def launches_per_step(self) -> int:
+        return int(_lib.efcp_launches_per_step(self._h))
+
+    def status(self) -> int:
+        return int(_lib.efcp_status(self._h))
+
+    def last_residual(self) -> float:
+        return float(_lib.efcp_last_residual(self._h))
+
+    def error(self) -> np.ndarray:
+        out = np.empty(self.d, np.float32)
+        self._check(_lib.efcp_get_error(self._h, _np_ptr(out)), "efcp_get_error")
+        return out
+
+    def row(self, slot: int):
+        idx = np.empty(self.k, np.int32)
+        val = np.empty(self.k, np.float32)
+        self._check(_lib.efcp_get_row(self._h, slot, _np_ptr(idx), _np_ptr(val)), "efcp_get_row")
+        return idx, val
+
+    def gram(self) -> np.ndarray:
+        out = np.empty((self.m, self.m), np.float64)
+        self._check(_lib.efcp_get_gram(self._h, _np_ptr(out)), "efcp_get_gram")
+        return out
+
+    def weights(self) -> np.ndarray:
+        out = np.empty(self.m, np.float64)
+        self._check(_lib.efcp_get_weights(self._h, _np_ptr(out)), "efcp_get_weights")
+        return out

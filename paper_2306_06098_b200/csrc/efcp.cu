@@ -1,0 +1,435 @@
+// Host side of the EFCP C ABI (see include/efcp.h): handle, allocation, and the kernel
+// sequence of one step.  Everything a step computes runs in the kernels of this
+// directory; there is no CPU fallback.
+#include "efcp.h"
+
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "efcp_common.cuh"
+#include "efcp_mxm.cuh"
+#include "efcp_topk.cuh"
+#include "efcp_window.cuh"
+
+using namespace efcp;
+
+struct efcp_ctx {
+  int64_t d = 0, k = 0;
+  int32_t m = 0;
+  float lambda = 0.f;
+  uint32_t flags = 0;
+  int device = 0;
+  int num_sms = 0;
+  int64_t t = 0;
+  int W = 0, n_slabs = 0, n_chunks = 0;
+  int grid_slab = 0;  // blocks of the slab kernels (SP partials are per block)
+  // state
+  float* e = nullptr;
+  int32_t* I = nullptr;
+  float* V = nullptr;
+  int32_t* offs = nullptr;
+  double* S = nullptr;
+  double* B = nullptr;
+  // scratch
+  uint32_t* hist = nullptr;  // kBins1 + kBins2 + kBins3
+  int32_t* chunk_off = nullptr;
+  int32_t* cand_idx = nullptr;
+  float* cand_val = nullptr;
+  int32_t* sel_gt = nullptr;
+  int32_t* sel_eq = nullptr;
+  Scalars* sc = nullptr;
+  double* partial = nullptr;
+  double* vecs = nullptr;  // 8 m-vectors: delta, aprime, y, bold, z, w, res, dw
+  float* wf = nullptr;
+  float* stage_g = nullptr;  // efcp_step_host staging
+  float* stage_u = nullptr;
+  int last_cuda = 0;
+  int launches = 0;
+  std::vector<void*> allocs;
+};
+
+namespace {
+
+struct Sizes {
+  int W, n_slabs, n_chunks, grid_slab;
+  int64_t total;
+};
+
+int pick_slab_width(int64_t d, int m, int num_sms) {
+  int W = 32768;
+  if (const char* env = getenv("EFCP_SLAB_W")) {
+    const int v = atoi(env);
+    if (v >= 256 && v <= 49152 && (v & 3) == 0) return v;
+  }
+  // shared memory: W*4 + 16*m must stay under the 227 KB per-block limit
+  while (size_t(W) * 4 + size_t(m) * 16 > 200 * 1024 && W > 1024) W >>= 1;
+  // enough slabs to give every SM several
+  while (W > 1024 && (d + W - 1) / W < int64_t(4) * num_sms) W >>= 1;
+  return W;
+}
+
+inline int64_t align256(int64_t b) { return (b + 255) & ~int64_t(255); }
+
+Sizes compute_sizes(int64_t d, int32_t m, int64_t k, int num_sms) {
+  Sizes z;
+  z.W = pick_slab_width(d, m, num_sms);
+  z.n_slabs = int((d + z.W - 1) / z.W);
+  z.n_chunks = int((d + kChunk - 1) / kChunk);
+  z.grid_slab = z.n_slabs < num_sms ? z.n_slabs : num_sms;
+  int64_t b = 0;
+  b += align256(d * 4);                                   // e
+  b += 2 * align256(int64_t(m) * k * 4);                  // I, V
+  b += align256(int64_t(z.n_slabs + 1) * m * 4);          // offs
+  b += 2 * align256(int64_t(m) * m * 8);                  // S, B
+  b += align256((kBins1 + kBins2 + kBins3) * 4);          // hist
+  b += 3 * align256(int64_t(z.n_chunks + 1) * 4);         // chunk_off, sel_gt, sel_eq
+  b += 2 * align256(d * 4);                               // cand_idx, cand_val
+  b += align256(sizeof(Scalars));
+  b += align256(int64_t(z.grid_slab) * m * 8);            // partial
+  b += align256(int64_t(8) * m * 8);                      // vecs
+  b += align256(int64_t(m) * 4);                          // wf
+  z.total = b;
+  return z;
+}
+
+bool valid_args(int64_t d, int32_t m, int64_t k) {
+  return d >= 1 && m >= 1 && m <= 4096 && k >= 1 && k <= d && d < (int64_t(1) << 31);
+}
+
+__global__ void k_init_rows(int32_t* __restrict__ I, int64_t k, int64_t total) {
+  for (int64_t i = int64_t(blockIdx.x) * blockDim.x + threadIdx.x; i < total;
+       i += int64_t(gridDim.x) * blockDim.x)
+    I[i] = int32_t(i % k);
+}
+
+#define EFCP_CUDA(call)                         \
+  do {                                          \
+    cudaError_t err__ = (call);                 \
+    if (err__ != cudaSuccess) {                 \
+      ctx->last_cuda = int(err__);              \
+      return EFCP_ECUDA;                        \
+    }                                           \
+  } while (0)
+
+#define EFCP_LAUNCHED()                         \
+  do {                                          \
+    ++ctx->launches;                            \
+    cudaError_t err__ = cudaGetLastError();     \
+    if (err__ != cudaSuccess) {                 \
+      ctx->last_cuda = int(err__);              \
+      return EFCP_ECUDA;                        \
+    }                                           \
+  } while (0)
+
+template <typename T>
+int dev_alloc(efcp_ctx* ctx, T** p, int64_t bytes) {
+  void* q = nullptr;
+  cudaError_t err = cudaMalloc(&q, size_t(align256(bytes)));
+  if (err != cudaSuccess) {
+    ctx->last_cuda = int(err);
+    (void)cudaGetLastError();
+    return EFCP_ENOMEM;
+  }
+  ctx->allocs.push_back(q);
+  *p = static_cast<T*>(q);
+  return EFCP_OK;
+}
+
+int status_to_code(uint32_t st) {
+  if (st & kStCount) return EFCP_EINTERNAL;
+  if (st & kStTimeout) return EFCP_ETIMEOUT;
+  if (st & (kStNonFinite | kStPivot)) return EFCP_ENUMERIC;
+  return EFCP_OK;
+}
+
+int sync_status(efcp_ctx* ctx) {
+  EFCP_CUDA(cudaSetDevice(ctx->device));
+  EFCP_CUDA(cudaDeviceSynchronize());
+  Scalars h;
+  EFCP_CUDA(cudaMemcpy(&h, ctx->sc, sizeof(h), cudaMemcpyDeviceToHost));
+  return status_to_code(h.status);
+}
+
+void free_all(efcp_ctx* ctx) {
+  for (void* p : ctx->allocs) cudaFree(p);
+  ctx->allocs.clear();
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* efcp_strerror(int code) {
+  switch (code) {
+    case EFCP_OK: return "ok";
+    case EFCP_EINVAL: return "invalid argument";
+    case EFCP_ENOMEM: return "out of memory";
+    case EFCP_ECUDA: return "CUDA runtime error (see efcp_last_cuda_error)";
+    case EFCP_ENUMERIC: return "non-finite input or non-positive pivot in the m x m update";
+    case EFCP_ETIMEOUT: return "bounded device-side wait expired";
+    case EFCP_EINTERNAL: return "internal consistency check failed";
+    default: return "unknown error code";
+  }
+}
+
+int64_t efcp_state_bytes(int64_t d, int32_t m, int64_t k) {
+  if (!valid_args(d, m, k)) return -1;
+  return compute_sizes(d, m, k, 148).total;
+}
+
+int efcp_create(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float lambda) {
+  return efcp_create_ex(out, d, m, k, lambda, EFCP_RHS_COMPRESSED);
+}
+
+int efcp_create_ex(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float lambda,
+                   uint32_t flags) {
+  if (!out) return EFCP_EINVAL;
+  *out = nullptr;
+  if (!valid_args(d, m, k) || !(lambda > 0.f) || !std::isfinite(lambda)) return EFCP_EINVAL;
+  if (flags & ~EFCP_RHS_ACCUMULATOR) return EFCP_EINVAL;
+  if (flags & EFCP_RHS_ACCUMULATOR) return EFCP_EINVAL;  // not built yet
+  efcp_ctx* ctx = new (std::nothrow) efcp_ctx();
+  if (!ctx) return EFCP_ENOMEM;
+  int rc = EFCP_OK;
+  auto fail = [&](int code) {
+    free_all(ctx);
+    delete ctx;
+    return code;
+  };
+  cudaError_t err = cudaGetDevice(&ctx->device);
+  if (err != cudaSuccess) { (void)cudaGetLastError(); return fail(EFCP_ECUDA); }
+  cudaDeviceProp prop;
+  err = cudaGetDeviceProperties(&prop, ctx->device);
+  if (err != cudaSuccess) { (void)cudaGetLastError(); return fail(EFCP_ECUDA); }
+  ctx->num_sms = prop.multiProcessorCount;
+  ctx->d = d; ctx->m = m; ctx->k = k; ctx->lambda = lambda; ctx->flags = flags;
+  const Sizes z = compute_sizes(d, m, k, ctx->num_sms);
+  ctx->W = z.W; ctx->n_slabs = z.n_slabs; ctx->n_chunks = z.n_chunks;
+  ctx->grid_slab = z.grid_slab;
+  const int64_t mk = int64_t(m) * k;
+  if ((rc = dev_alloc(ctx, &ctx->e, d * 4))) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->I, mk * 4))) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->V, mk * 4))) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->offs, int64_t(z.n_slabs + 1) * m * 4))) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->S, int64_t(m) * m * 8))) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->B, int64_t(m) * m * 8))) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->hist, (kBins1 + kBins2 + kBins3) * 4))) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->chunk_off, int64_t(z.n_chunks + 1) * 4))) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->sel_gt, int64_t(z.n_chunks + 1) * 4))) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->sel_eq, int64_t(z.n_chunks + 1) * 4))) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->cand_idx, d * 4))) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->cand_val, d * 4))) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->sc, sizeof(Scalars)))) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->partial, int64_t(z.grid_slab) * m * 8))) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->vecs, int64_t(8) * m * 8))) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->wf, int64_t(m) * 4))) return fail(rc);
+
+  bool ok = true;
+  ok &= cudaMemset(ctx->e, 0, size_t(d) * 4) == cudaSuccess;
+  ok &= cudaMemset(ctx->V, 0, size_t(mk) * 4) == cudaSuccess;
+  ok &= cudaMemset(ctx->offs, 0, size_t(z.n_slabs + 1) * m * 4) == cudaSuccess;
+  ok &= cudaMemset(ctx->S, 0, size_t(m) * m * 8) == cudaSuccess;
+  ok &= cudaMemset(ctx->hist, 0, (kBins1 + kBins2 + kBins3) * 4) == cudaSuccess;
+  ok &= cudaMemset(ctx->sc, 0, sizeof(Scalars)) == cudaSuccess;
+  ok &= cudaMemset(ctx->vecs, 0, size_t(8) * m * 8) == cudaSuccess;
+  ok &= cudaMemset(ctx->wf, 0, size_t(m) * 4) == cudaSuccess;
+  k_init_rows<<<ctx->num_sms * 4, 256>>>(ctx->I, k, mk);
+  k_init_identity<<<ctx->num_sms * 2, 256>>>(ctx->B, m, 1.0 / (double(m) * double(lambda)));
+  const size_t smem = slab_smem_bytes(z.W, m);
+  ok &= cudaFuncSetAttribute(k_sp_rows, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             int(smem)) == cudaSuccess;
+  ok &= cudaFuncSetAttribute(k_lcg<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             int(smem)) == cudaSuccess;
+  ok &= cudaFuncSetAttribute(k_lcg<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             int(smem)) == cudaSuccess;
+  ok &= cudaDeviceSynchronize() == cudaSuccess;
+  if (!ok) {
+    ctx->last_cuda = int(cudaGetLastError());
+    return fail(EFCP_ECUDA);
+  }
+  *out = ctx;
+  return EFCP_OK;
+}
+
+int efcp_destroy(efcp_ctx* ctx) {
+  if (!ctx) return EFCP_EINVAL;
+  cudaSetDevice(ctx->device);
+  cudaDeviceSynchronize();
+  free_all(ctx);
+  delete ctx;
+  return EFCP_OK;
+}
+
+int efcp_step(efcp_ctx* ctx, const float* grad, float* update, void* stream_) {
+  if (!ctx || !grad || !update || grad == update) return EFCP_EINVAL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream_);
+  const int64_t d = ctx->d, k = ctx->k;
+  const int m = ctx->m;
+  const int slot = int(ctx->t % m);
+  ctx->launches = 0;
+  uint32_t* hist1 = ctx->hist;
+  uint32_t* hist2 = ctx->hist + kBins1;
+  uint32_t* hist3 = ctx->hist + kBins1 + kBins2;
+  int32_t* row_idx = ctx->I + int64_t(slot) * k;
+  float* row_val = ctx->V + int64_t(slot) * k;
+  double* delta = ctx->vecs;
+  double* aprime = delta + m;
+  double* y = aprime + m;
+  double* bold = y + m;
+  double* z = bold + m;
+  double* w = z + m;
+  double* res = w + m;
+  double* dw = res + m;
+  const double mlambda = double(m) * double(ctx->lambda);
+
+  // a = xi + g, digit-1 histogram
+  const int ef_grid = ctx->num_sms * 2;
+  if ((reinterpret_cast<uintptr_t>(grad) & 15) == 0)
+    k_ef_hist1<true><<<ef_grid, 512, 0, st>>>(ctx->e, grad, d, hist1, ctx->sc);
+  else
+    k_ef_hist1<false><<<ef_grid, 512, 0, st>>>(ctx->e, grad, d, hist1, ctx->sc);
+  EFCP_LAUNCHED();
+  k_pick<kBins1, 1><<<1, 1024, 0, st>>>(hist1, ctx->sc, uint32_t(k));
+  EFCP_LAUNCHED();
+  // candidates: everything at or above the threshold bin, in index order
+  k_count_chunks<<<ctx->n_chunks, kChunkThreads, 0, st>>>(ctx->e, d, ctx->sc, ctx->chunk_off);
+  EFCP_LAUNCHED();
+  k_scan_counts<<<1, 1024, 0, st>>>(ctx->chunk_off, ctx->n_chunks, &ctx->sc->n_cand);
+  EFCP_LAUNCHED();
+  k_compact_cand<<<ctx->n_chunks, kChunkThreads, 0, st>>>(ctx->e, d, ctx->sc, ctx->chunk_off,
+                                                          ctx->cand_idx, ctx->cand_val, hist2);
+  EFCP_LAUNCHED();
+  k_pick<kBins2, 2><<<1, 1024, 0, st>>>(hist2, ctx->sc, uint32_t(k));
+  EFCP_LAUNCHED();
+  const int cand_grid = ctx->num_sms * 4;
+  k_hist3<<<cand_grid, 256, 0, st>>>(ctx->cand_val, ctx->sc, hist3);
+  EFCP_LAUNCHED();
+  k_pick<kBins3, 3><<<1, 1024, 0, st>>>(hist3, ctx->sc, uint32_t(k));
+  EFCP_LAUNCHED();
+  // exact selection, ring insert, residual
+  k_count_sel<<<cand_grid, kChunkThreads, 0, st>>>(ctx->cand_val, ctx->sc, ctx->sel_gt,
+                                                   ctx->sel_eq);
+  EFCP_LAUNCHED();
+  k_scan_sel<<<1, 1024, 0, st>>>(ctx->sel_gt, ctx->sel_eq, ctx->sc, uint32_t(k));
+  EFCP_LAUNCHED();
+  k_write_sel<<<cand_grid, kChunkThreads, 0, st>>>(ctx->cand_idx, ctx->cand_val, ctx->sc,
+                                                   ctx->sel_gt, ctx->sel_eq, row_idx, row_val,
+                                                   ctx->e, k);
+  EFCP_LAUNCHED();
+  k_build_offsets<<<(ctx->n_slabs + 1 + 255) / 256, 256, 0, st>>>(row_idx, k, ctx->W,
+                                                                  ctx->n_slabs, m, slot,
+                                                                  ctx->offs);
+  EFCP_LAUNCHED();
+  // scalar products with the new row, Gram row/column
+  const size_t smem = slab_smem_bytes(ctx->W, m);
+  k_sp_rows<<<ctx->grid_slab, 1024, smem, st>>>(ctx->I, ctx->V, ctx->offs, k, m, ctx->W,
+                                                ctx->n_slabs, slot, ctx->partial);
+  EFCP_LAUNCHED();
+  k_sp_finish<<<(m + 127) / 128, 128, 0, st>>>(ctx->partial, ctx->grid_slab, m, slot, delta,
+                                               ctx->S, aprime);
+  EFCP_LAUNCHED();
+  // m x m: remove-and-border update of the inverse, weights, one refinement step
+  const int gemv_grid = (m + 7) / 8;
+  k_gemv<<<gemv_grid, 256, 0, st>>>(ctx->B, aprime, y, m);
+  EFCP_LAUNCHED();
+  k_border_scalars<<<1, 1024, 0, st>>>(y, ctx->B + int64_t(slot) * m, delta, aprime, m, slot,
+                                       mlambda, bold, z, w, ctx->sc);
+  EFCP_LAUNCHED();
+  k_rank2<<<ctx->num_sms * 2, 256, 0, st>>>(ctx->B, bold, z, ctx->sc, m, slot);
+  EFCP_LAUNCHED();
+  k_residual<<<gemv_grid, 256, 0, st>>>(ctx->S, w, res, m, slot, mlambda);
+  EFCP_LAUNCHED();
+  k_gemv<<<gemv_grid, 256, 0, st>>>(ctx->B, res, dw, m);
+  EFCP_LAUNCHED();
+  k_refine_finish<<<1, 1024, 0, st>>>(w, dw, res, ctx->wf, m, ctx->sc);
+  EFCP_LAUNCHED();
+  // linear combination of the window rows
+  if ((reinterpret_cast<uintptr_t>(update) & 15) == 0)
+    k_lcg<true><<<ctx->grid_slab, 1024, smem, st>>>(ctx->I, ctx->V, ctx->offs, k, m, ctx->W,
+                                                    ctx->n_slabs, ctx->wf, update, d);
+  else
+    k_lcg<false><<<ctx->grid_slab, 1024, smem, st>>>(ctx->I, ctx->V, ctx->offs, k, m, ctx->W,
+                                                     ctx->n_slabs, ctx->wf, update, d);
+  EFCP_LAUNCHED();
+  ctx->t += 1;
+  return EFCP_OK;
+}
+
+int efcp_step_host(efcp_ctx* ctx, const float* grad, float* update, void* stream_) {
+  if (!ctx || !grad || !update) return EFCP_EINVAL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream_);
+  if (!ctx->stage_g) {
+    int rc;
+    if ((rc = dev_alloc(ctx, &ctx->stage_g, ctx->d * 4))) return rc;
+    if ((rc = dev_alloc(ctx, &ctx->stage_u, ctx->d * 4))) return rc;
+  }
+  EFCP_CUDA(cudaMemcpyAsync(ctx->stage_g, grad, size_t(ctx->d) * 4, cudaMemcpyHostToDevice, st));
+  const int rc = efcp_step(ctx, ctx->stage_g, ctx->stage_u, stream_);
+  if (rc != EFCP_OK) return rc;
+  EFCP_CUDA(cudaMemcpyAsync(update, ctx->stage_u, size_t(ctx->d) * 4, cudaMemcpyDeviceToHost, st));
+  EFCP_CUDA(cudaStreamSynchronize(st));
+  return EFCP_OK;
+}
+
+int efcp_get_error(efcp_ctx* ctx, float* host_e) {
+  if (!ctx || !host_e) return EFCP_EINVAL;
+  const int rc = sync_status(ctx);
+  if (rc == EFCP_ECUDA) return rc;
+  EFCP_CUDA(cudaMemcpy(host_e, ctx->e, size_t(ctx->d) * 4, cudaMemcpyDeviceToHost));
+  return rc;
+}
+
+int efcp_get_row(efcp_ctx* ctx, int32_t slot, int32_t* host_idx, float* host_val) {
+  if (!ctx || !host_idx || !host_val || slot < 0 || slot >= ctx->m) return EFCP_EINVAL;
+  const int rc = sync_status(ctx);
+  if (rc == EFCP_ECUDA) return rc;
+  const size_t bytes = size_t(ctx->k) * 4;
+  EFCP_CUDA(cudaMemcpy(host_idx, ctx->I + int64_t(slot) * ctx->k, bytes, cudaMemcpyDeviceToHost));
+  EFCP_CUDA(cudaMemcpy(host_val, ctx->V + int64_t(slot) * ctx->k, bytes, cudaMemcpyDeviceToHost));
+  return rc;
+}
+
+int efcp_get_gram(efcp_ctx* ctx, double* host_S) {
+  if (!ctx || !host_S) return EFCP_EINVAL;
+  const int rc = sync_status(ctx);
+  if (rc == EFCP_ECUDA) return rc;
+  EFCP_CUDA(cudaMemcpy(host_S, ctx->S, size_t(ctx->m) * ctx->m * 8, cudaMemcpyDeviceToHost));
+  return rc;
+}
+
+int efcp_get_weights(efcp_ctx* ctx, double* host_w) {
+  if (!ctx || !host_w) return EFCP_EINVAL;
+  const int rc = sync_status(ctx);
+  if (rc == EFCP_ECUDA) return rc;
+  EFCP_CUDA(cudaMemcpy(host_w, ctx->vecs + int64_t(5) * ctx->m, size_t(ctx->m) * 8,
+                       cudaMemcpyDeviceToHost));
+  return rc;
+}
+
+int64_t efcp_step_count(efcp_ctx* ctx) { return ctx ? ctx->t : -1; }
+
+int efcp_status(efcp_ctx* ctx) {
+  if (!ctx) return EFCP_EINVAL;
+  return sync_status(ctx);
+}
+
+int efcp_last_cuda_error(efcp_ctx* ctx) { return ctx ? ctx->last_cuda : 0; }
+
+double efcp_last_residual(efcp_ctx* ctx) {
+  if (!ctx) return -1.0;
+  if (cudaSetDevice(ctx->device) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess)
+    return -1.0;
+  Scalars h;
+  if (cudaMemcpy(&h, ctx->sc, sizeof(h), cudaMemcpyDeviceToHost) != cudaSuccess) return -1.0;
+  return h.resid;
+}
+
+int32_t efcp_launches_per_step(efcp_ctx* ctx) { return ctx ? ctx->launches : -1; }
+
+}  // extern "C"

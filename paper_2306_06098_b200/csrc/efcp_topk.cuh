@@ -1,0 +1,340 @@
+// Error feedback + exact global Top-k (Algorithm 1 lines 5-7, Section 3.1).
+//
+// Selection is a most-significant-digit radix select on the 31-bit magnitude key
+// (12 + 10 + 9 bits).  Digit 1 is histogrammed while a = xi + g is formed; every
+// entry at or above the threshold bin of digit 1 is then compacted, in index order,
+// into a candidate list, and digits 2 and 3 are resolved on that list only.  The
+// final ordered compaction writes the row (ascending indices) straight into the
+// ring slot and zeroes the kept coordinates of xi.  Ties at the threshold key are
+// taken in index order, so the result is the unique "first k of a sort by
+// (|a| descending, index ascending)".
+#pragma once
+
+#include "efcp_common.cuh"
+
+namespace efcp {
+
+// a = xi + g in place over xi, histogram of digit 1, non-finite detection.
+template <bool VEC>
+__global__ void __launch_bounds__(512) k_ef_hist1(float* __restrict__ e,
+                                                   const float* __restrict__ g, int64_t d,
+                                                   uint32_t* __restrict__ hist1, Scalars* sc) {
+  __shared__ uint32_t h[kBins1];
+  for (int i = threadIdx.x; i < kBins1; i += blockDim.x) h[i] = 0u;
+  __syncthreads();
+  bool bad = false;
+  const int64_t tid = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
+  const int64_t nth = int64_t(gridDim.x) * blockDim.x;
+  auto tally = [&](float a) {
+    const uint32_t key = mag_key(a);
+    atomicAdd(&h[key >> kShift1], 1u);
+    bad |= key >= 0x7F800000u;
+  };
+  int64_t scalar_from = 0;
+  if (VEC) {
+    const int64_t nv = d >> 2;
+    float4* e4 = reinterpret_cast<float4*>(e);
+    const float4* g4 = reinterpret_cast<const float4*>(g);
+    int64_t v = tid;
+    for (; v + nth < nv; v += 2 * nth) {
+      float4 e0 = e4[v], e1 = e4[v + nth];
+      const float4 g0 = __ldcs(g4 + v), g1 = __ldcs(g4 + v + nth);
+      e0.x = __fadd_rn(e0.x, g0.x); e0.y = __fadd_rn(e0.y, g0.y);
+      e0.z = __fadd_rn(e0.z, g0.z); e0.w = __fadd_rn(e0.w, g0.w);
+      e1.x = __fadd_rn(e1.x, g1.x); e1.y = __fadd_rn(e1.y, g1.y);
+      e1.z = __fadd_rn(e1.z, g1.z); e1.w = __fadd_rn(e1.w, g1.w);
+      e4[v] = e0; e4[v + nth] = e1;
+      tally(e0.x); tally(e0.y); tally(e0.z); tally(e0.w);
+      tally(e1.x); tally(e1.y); tally(e1.z); tally(e1.w);
+    }
+    for (; v < nv; v += nth) {
+      float4 e0 = e4[v];
+      const float4 g0 = __ldcs(g4 + v);
+      e0.x = __fadd_rn(e0.x, g0.x); e0.y = __fadd_rn(e0.y, g0.y);
+      e0.z = __fadd_rn(e0.z, g0.z); e0.w = __fadd_rn(e0.w, g0.w);
+      e4[v] = e0;
+      tally(e0.x); tally(e0.y); tally(e0.z); tally(e0.w);
+    }
+    scalar_from = nv << 2;
+  }
+  for (int64_t j = scalar_from + tid; j < d; j += nth) {
+    const float a = __fadd_rn(e[j], g[j]);
+    e[j] = a;
+    tally(a);
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < kBins1; i += blockDim.x) {
+    const uint32_t c = h[i];
+    if (c) atomicAdd(&hist1[i], c);
+  }
+  if (bad) atomicOr(&sc->status, kStNonFinite);
+}
+
+// Finds the threshold bin of one digit: the bin b with count(bins > b) < k_rem <=
+// count(bins >= b).  Clears the histogram for the next step.  One block of 1024.
+template <int NB, int LEVEL>
+__global__ void __launch_bounds__(1024) k_pick(uint32_t* __restrict__ hist, Scalars* sc,
+                                                uint32_t k_total) {
+  __shared__ uint32_t h[NB];
+  __shared__ uint32_t sm[33];
+  for (int i = threadIdx.x; i < NB; i += blockDim.x) {
+    h[i] = hist[i];
+    hist[i] = 0u;
+  }
+  __syncthreads();
+  const uint32_t k_rem = LEVEL == 1 ? k_total : (LEVEL == 2 ? sc->k1 : sc->k2);
+  constexpr int P = (NB + 1023) / 1024;
+  uint32_t mine = 0;
+#pragma unroll
+  for (int p = 0; p < P; ++p) {
+    const int pos = threadIdx.x * P + p;  // position counted from the highest bin
+    if (pos < NB) mine += h[NB - 1 - pos];
+  }
+  uint32_t total;
+  uint32_t above = block_excl_scan<uint32_t>(mine, &total, sm);
+#pragma unroll
+  for (int p = 0; p < P; ++p) {
+    const int pos = threadIdx.x * P + p;
+    if (pos < NB) {
+      const uint32_t bin = NB - 1 - pos;
+      const uint32_t c = h[bin];
+      if (above < k_rem && above + c >= k_rem) {
+        if (LEVEL == 1) { sc->b1 = bin; sc->k1 = k_rem - above; }
+        if (LEVEL == 2) { sc->b2 = bin; sc->k2 = k_rem - above; }
+        if (LEVEL == 3) {
+          sc->T = (sc->b1 << kShift1) | (sc->b2 << kShift2) | bin;
+          sc->n_eq = k_rem - above;
+        }
+      }
+      above += c;
+    }
+  }
+  if (threadIdx.x == 0 && total < k_rem) atomicOr(&sc->status, kStCount);
+}
+
+__device__ __forceinline__ void load_chunk8(const float* __restrict__ a, int64_t base, int64_t n,
+                                            float (&v)[kPerThread], bool (&ok)[kPerThread]) {
+  if (base + kPerThread <= n) {
+    const float4 x0 = *reinterpret_cast<const float4*>(a + base);
+    const float4 x1 = *reinterpret_cast<const float4*>(a + base + 4);
+    v[0] = x0.x; v[1] = x0.y; v[2] = x0.z; v[3] = x0.w;
+    v[4] = x1.x; v[5] = x1.y; v[6] = x1.z; v[7] = x1.w;
+#pragma unroll
+    for (int q = 0; q < kPerThread; ++q) ok[q] = true;
+  } else {
+#pragma unroll
+    for (int q = 0; q < kPerThread; ++q) {
+      ok[q] = base + q < n;
+      v[q] = ok[q] ? a[base + q] : 0.f;
+    }
+  }
+}
+
+// Per chunk of the accumulator: how many entries have digit 1 >= b1.
+__global__ void __launch_bounds__(kChunkThreads) k_count_chunks(const float* __restrict__ a,
+                                                                 int64_t d, const Scalars* sc,
+                                                                 int32_t* __restrict__ cnt) {
+  __shared__ int sm[33];
+  const uint32_t b1 = sc->b1;
+  const int64_t base = int64_t(blockIdx.x) * kChunk + threadIdx.x * kPerThread;
+  float v[kPerThread];
+  bool ok[kPerThread];
+  load_chunk8(a, base, d, v, ok);
+  int c = 0;
+#pragma unroll
+  for (int q = 0; q < kPerThread; ++q) c += (ok[q] && (mag_key(v[q]) >> kShift1) >= b1) ? 1 : 0;
+  int total;
+  (void)block_excl_scan<int>(c, &total, sm);
+  if (threadIdx.x == 0) cnt[blockIdx.x] = total;
+}
+
+// In-place exclusive scan of n chunk counts by one block; cnt[n] and *total_out get the sum.
+__global__ void __launch_bounds__(1024) k_scan_counts(int32_t* __restrict__ cnt, int n,
+                                                       int32_t* total_out) {
+  __shared__ int sm[33];
+  int carry = 0;
+  for (int base = 0; base < n; base += 1024) {
+    const int i = base + threadIdx.x;
+    const int v = i < n ? cnt[i] : 0;
+    int total;
+    const int ex = block_excl_scan<int>(v, &total, sm);
+    if (i < n) cnt[i] = carry + ex;
+    carry += total;
+  }
+  if (threadIdx.x == 0) {
+    cnt[n] = carry;
+    *total_out = carry;
+  }
+}
+
+// Ordered compaction of the candidates (digit 1 >= b1) and histogram of digit 2 over
+// the entries inside the threshold bin.
+__global__ void __launch_bounds__(kChunkThreads) k_compact_cand(
+    const float* __restrict__ a, int64_t d, const Scalars* sc, const int32_t* __restrict__ off,
+    int32_t* __restrict__ cand_idx, float* __restrict__ cand_val, uint32_t* __restrict__ hist2) {
+  __shared__ uint32_t h[kBins2];
+  __shared__ int sm[33];
+  for (int i = threadIdx.x; i < kBins2; i += blockDim.x) h[i] = 0u;
+  __syncthreads();
+  const uint32_t b1 = sc->b1;
+  const int64_t base = int64_t(blockIdx.x) * kChunk + threadIdx.x * kPerThread;
+  float v[kPerThread];
+  bool ok[kPerThread];
+  load_chunk8(a, base, d, v, ok);
+  int c = 0;
+#pragma unroll
+  for (int q = 0; q < kPerThread; ++q) {
+    ok[q] = ok[q] && (mag_key(v[q]) >> kShift1) >= b1;
+    c += ok[q] ? 1 : 0;
+  }
+  int total;
+  int pos = off[blockIdx.x] + block_excl_scan<int>(c, &total, sm);
+#pragma unroll
+  for (int q = 0; q < kPerThread; ++q) {
+    if (ok[q]) {
+      cand_idx[pos] = int32_t(base + q);
+      cand_val[pos] = v[q];
+      ++pos;
+      const uint32_t key = mag_key(v[q]);
+      if ((key >> kShift1) == b1) atomicAdd(&h[(key >> kShift2) & (kBins2 - 1)], 1u);
+    }
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < kBins2; i += blockDim.x) {
+    const uint32_t cc = h[i];
+    if (cc) atomicAdd(&hist2[i], cc);
+  }
+}
+
+// Histogram of digit 3 over the candidates whose digits 1 and 2 match the threshold.
+__global__ void __launch_bounds__(256) k_hist3(const float* __restrict__ cand_val,
+                                                const Scalars* sc, uint32_t* __restrict__ hist3) {
+  __shared__ uint32_t h[kBins3];
+  for (int i = threadIdx.x; i < kBins3; i += blockDim.x) h[i] = 0u;
+  __syncthreads();
+  const int n = sc->n_cand;
+  const uint32_t prefix = (sc->b1 << kBits2) | sc->b2;
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
+    const uint32_t key = mag_key(cand_val[i]);
+    if ((key >> kShift2) == prefix) atomicAdd(&h[key & (kBins3 - 1)], 1u);
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < kBins3; i += blockDim.x) {
+    const uint32_t c = h[i];
+    if (c) atomicAdd(&hist3[i], c);
+  }
+}
+
+// Per candidate chunk: entries above the threshold key and entries equal to it.
+__global__ void __launch_bounds__(kChunkThreads) k_count_sel(const float* __restrict__ cand_val,
+                                                              const Scalars* sc,
+                                                              int32_t* __restrict__ cnt_gt,
+                                                              int32_t* __restrict__ cnt_eq) {
+  __shared__ int sm[33];
+  const int n = sc->n_cand;
+  const uint32_t T = sc->T;
+  const int n_cc = (n + kChunk - 1) / kChunk;
+  for (int c = blockIdx.x; c < n_cc; c += gridDim.x) {
+    const int64_t base = int64_t(c) * kChunk + threadIdx.x * kPerThread;
+    float v[kPerThread];
+    bool ok[kPerThread];
+    load_chunk8(cand_val, base, n, v, ok);
+    int packed = 0;  // gt in the low half, eq in the high half (each <= 2048)
+#pragma unroll
+    for (int q = 0; q < kPerThread; ++q) {
+      const uint32_t key = mag_key(v[q]);
+      packed += (ok[q] && key > T) ? 1 : 0;
+      packed += (ok[q] && key == T) ? (1 << 16) : 0;
+    }
+    int total;
+    (void)block_excl_scan<int>(packed, &total, sm);
+    if (threadIdx.x == 0) {
+      cnt_gt[c] = total & 0xFFFF;
+      cnt_eq[c] = total >> 16;
+    }
+  }
+}
+
+// Exclusive scans of both per-chunk counts (one block) and the count check.
+__global__ void __launch_bounds__(1024) k_scan_sel(int32_t* __restrict__ cnt_gt,
+                                                    int32_t* __restrict__ cnt_eq, Scalars* sc,
+                                                    uint32_t k_total) {
+  __shared__ int sm[33];
+  const int n_cc = (sc->n_cand + kChunk - 1) / kChunk;
+  int carry_gt = 0, carry_eq = 0;
+  for (int base = 0; base < n_cc; base += 1024) {
+    const int i = base + threadIdx.x;
+    const int g = i < n_cc ? cnt_gt[i] : 0;
+    const int q = i < n_cc ? cnt_eq[i] : 0;
+    int tg, tq;
+    const int eg = block_excl_scan<int>(g, &tg, sm);
+    const int eq = block_excl_scan<int>(q, &tq, sm);
+    if (i < n_cc) {
+      cnt_gt[i] = carry_gt + eg;
+      cnt_eq[i] = carry_eq + eq;
+    }
+    carry_gt += tg;
+    carry_eq += tq;
+  }
+  if (threadIdx.x == 0) {
+    const uint32_t n_eq = sc->n_eq;
+    sc->n_sel = carry_gt + int32_t(n_eq);
+    if (uint32_t(carry_gt) + n_eq != k_total || uint32_t(carry_eq) < n_eq)
+      atomicOr(&sc->status, kStCount);
+  }
+}
+
+// Final ordered compaction: writes the kept (index, value) pairs into the ring slot in
+// ascending index order and sets the kept coordinates of xi to +0 (xi = a - c).
+__global__ void __launch_bounds__(kChunkThreads) k_write_sel(
+    const int32_t* __restrict__ cand_idx, const float* __restrict__ cand_val, const Scalars* sc,
+    const int32_t* __restrict__ off_gt, const int32_t* __restrict__ pre_eq,
+    int32_t* __restrict__ row_idx, float* __restrict__ row_val, float* __restrict__ e,
+    int64_t k_total) {
+  __shared__ int sm[33];
+  const int n = sc->n_cand;
+  const uint32_t T = sc->T;
+  const int n_eq = int(sc->n_eq);
+  const int n_cc = (n + kChunk - 1) / kChunk;
+  for (int c = blockIdx.x; c < n_cc; c += gridDim.x) {
+    const int64_t base = int64_t(c) * kChunk + threadIdx.x * kPerThread;
+    float v[kPerThread];
+    bool ok[kPerThread];
+    load_chunk8(cand_val, base, n, v, ok);
+    bool is_eq[kPerThread];
+    int my_eq = 0;
+#pragma unroll
+    for (int q = 0; q < kPerThread; ++q) {
+      const uint32_t key = mag_key(v[q]);
+      is_eq[q] = ok[q] && key == T;
+      ok[q] = ok[q] && key > T;
+      my_eq += is_eq[q] ? 1 : 0;
+    }
+    int tot;
+    const int eq_before_chunk = pre_eq[c];
+    int eq_rank = eq_before_chunk + block_excl_scan<int>(my_eq, &tot, sm);
+    int my_sel = 0;
+#pragma unroll
+    for (int q = 0; q < kPerThread; ++q) {
+      if (is_eq[q]) {
+        ok[q] = eq_rank < n_eq;
+        ++eq_rank;
+      }
+      my_sel += ok[q] ? 1 : 0;
+    }
+    int64_t pos = int64_t(off_gt[c]) + min(eq_before_chunk, n_eq) +
+                  block_excl_scan<int>(my_sel, &tot, sm);
+#pragma unroll
+    for (int q = 0; q < kPerThread; ++q) {
+      if (ok[q] && pos < k_total) {
+        const int32_t j = cand_idx[base + q];
+        row_idx[pos] = j;
+        row_val[pos] = v[q];
+        e[j] = 0.0f;
+        ++pos;
+      }
+    }
+  }
+}
+
+}  // namespace efcp

@@ -1,0 +1,218 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle, element by
+element on the same seeded inputs.  State (error buffer, ring rows) must be bit-exact at
+every step; the update must agree within 1e-4 relative L2 (the bound the benchmark
+definition states for fp32)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import ref
+from paper_2306_06098_b200 import gradgen
+
+pytestmark = pytest.mark.gpu
+
+U_TOL = 1e-4  # relative L2 on the update, fp32
+
+
+def _binding():
+    from paper_2306_06098_b200 import binding
+    return binding
+
+
+def bits(a):
+    return np.ascontiguousarray(a).view(np.uint32)
+
+
+def rel_l2(a, b):
+    a = np.asarray(a, np.float64)
+    b = np.asarray(b, np.float64)
+    return np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-300)
+
+
+def lincomb_amplification(cpu, u_ref):
+    """| |G|^T |w| | / |u| for the oracle's window and Eq. (2) weights: how much larger the
+    terms of the linear combination are than its result.  fp32 accumulation of the
+    combination (the precision the paper's LCG kernel uses) loses this factor times the
+    fp32 unit roundoff; it is ~1 for the benchmark workloads and large only when window
+    rows are nearly parallel (e.g. k = 1 with a repeated coordinate)."""
+    assert cpu.flags == ref.RHS_COMPRESSED
+    w = -cpu.coef()
+    w[(cpu.step_count - 1) % cpu.m] += 1.0 / np.float64(np.float32(cpu.lam))
+    acc = np.zeros(cpu.d)
+    for r in range(cpu.m):
+        idx, val = cpu.row(r)
+        np.add.at(acc, idx, np.abs(w[r]) * np.abs(val.astype(np.float64)))
+    return np.linalg.norm(acc) / max(np.linalg.norm(u_ref.astype(np.float64)), 1e-300)
+
+
+def run_parity(d, m, k, lam, grads, flags=0, check_rows="new", gram_every=0,
+               allow_amplified=False):
+    """grads: iterable of fp32 numpy arrays.  Returns the worst update error seen.
+
+    allow_amplified: for deliberately degenerate windows only - the bound becomes
+    U_TOL + 8 * 2^-24 * amplification (see lincomb_amplification)."""
+    B = _binding()
+    gpu = B.Efcp(d, m, k, lam, flags)
+    cpu = ref.RefEFCP(d, m, k, lam, flags)
+    g_dev = torch.empty(d, dtype=torch.float32, device="cuda")
+    u_dev = torch.empty(d, dtype=torch.float32, device="cuda")
+    worst = 0.0
+    for t, g in enumerate(grads):
+        g = np.ascontiguousarray(g, np.float32)
+        g_dev.copy_(torch.from_numpy(g))
+        u_dev.fill_(float("nan"))  # every element must be overwritten
+        gpu.step(g_dev, u_dev)
+        u_ref = cpu.step(g)
+        u = u_dev.cpu().numpy()
+        assert gpu.status() == 0, (t, gpu.status())
+        assert np.array_equal(bits(gpu.error()), bits(cpu.error())), f"error buffer differs at step {t}"
+        slot = t % m
+        gi, gv = gpu.row(slot)
+        ci, cv = cpu.row(slot)
+        assert np.array_equal(gi, ci), f"row indices differ at step {t}"
+        assert np.array_equal(bits(gv), bits(cv)), f"row values differ at step {t}"
+        assert np.isfinite(u).all(), f"update has unwritten / non-finite entries at step {t}"
+        err = rel_l2(u, u_ref)
+        worst = max(worst, err)
+        tol = U_TOL
+        if allow_amplified and err > U_TOL:
+            tol = U_TOL + 8 * 2.0 ** -24 * lincomb_amplification(cpu, u_ref)
+        assert err <= tol, f"update rel-L2 {err:.3e} (tol {tol:.3e}) at step {t}"
+        if gram_every and (t % gram_every == 0):
+            Sg, Sc = gpu.gram(), cpu.gram()
+            assert np.array_equal(Sg, Sg.T)
+            assert np.allclose(Sg, Sc, rtol=1e-12, atol=1e-12 * np.abs(Sc).max())
+    if check_rows == "all":
+        for s in range(m):
+            gi, gv = gpu.row(s)
+            ci, cv = cpu.row(s)
+            assert np.array_equal(gi, ci) and np.array_equal(bits(gv), bits(cv))
+    assert gpu.step_count == cpu.step_count
+    print(f"parity d={d} m={m} k={k}: worst update rel-L2 {worst:.3e}")
+    gpu.close()
+    cpu.close()
+    return worst
+
+
+def stream_grads(w, steps):
+    s = gradgen.GradStream.for_workload(w)
+    for _ in range(steps):
+        yield s.next().numpy()
+
+
+def test_c1_full_run():
+    w = gradgen.C1
+    run_parity(w.d, w.m, w.k, w.lam, stream_grads(w, w.steps), check_rows="all", gram_every=7)
+
+
+def test_c2_shape_first_steps():
+    w = gradgen.C2
+    run_parity(w.d, w.m, w.k, w.lam, stream_grads(w, 24), gram_every=8)
+
+
+@pytest.mark.parametrize("d,m,k,steps", [
+    (1, 1, 1, 3), (5, 2, 2, 6), (31, 3, 31, 7), (2049, 4, 100, 9), (4097, 8, 1, 20),
+    (100_003, 16, 1000, 40), (1_000_001, 8, 33_333, 12),
+])
+def test_ragged_sizes(d, m, k, steps):
+    rng = np.random.default_rng(d)
+    scale = np.exp(rng.standard_normal(d))
+    grads = ((scale * rng.standard_normal(d)).astype(np.float32) for _ in range(steps))
+    run_parity(d, m, k, 1e-3, grads, check_rows="all", gram_every=3, allow_amplified=(k == 1))
+
+
+def test_heavy_ties():
+    # values from a small set: most of the selection is decided by the index rule
+    d, m, k = 50_000, 4, 777
+    rng = np.random.default_rng(11)
+    grads = [rng.integers(-2, 3, d).astype(np.float32) for _ in range(6)]
+    run_parity(d, m, k, 1e-2, grads, check_rows="all")
+
+
+def test_all_equal_and_zero_gradients():
+    d, m, k = 10_000, 3, 100
+    grads = [np.full(d, 1.5, np.float32), np.zeros(d, np.float32), np.full(d, -1.5, np.float32),
+             np.zeros(d, np.float32), np.zeros(d, np.float32)]
+    run_parity(d, m, k, 1e-1, grads, check_rows="all")
+
+
+def test_denormals_are_ordered_not_flushed():
+    d, m, k = 4096, 2, 64
+    rng = np.random.default_rng(12)
+    g = (rng.integers(1, 1 << 20, d).astype(np.uint32)).view(np.float32)  # all denormal
+    g = g * np.where(rng.random(d) < 0.5, -1, 1).astype(np.float32)
+    big = g.copy()
+    big[::97] = 1.0
+    run_parity(d, m, k, 1.0, [g, big, g], check_rows="all")
+
+
+def test_unaligned_pointers():
+    B = _binding()
+    d, m, k = 70_001, 4, 500
+    rng = np.random.default_rng(13)
+    gpu = B.Efcp(d, m, k, 1e-3)
+    cpu = ref.RefEFCP(d, m, k, 1e-3)
+    gbuf = torch.empty(d + 3, dtype=torch.float32, device="cuda")
+    ubuf = torch.empty(d + 3, dtype=torch.float32, device="cuda")
+    for t in range(5):
+        g = rng.standard_normal(d).astype(np.float32)
+        gv, uv = gbuf[1:d + 1], ubuf[3:d + 3]
+        gv.copy_(torch.from_numpy(g))
+        gpu.step(gv, uv)
+        u_ref = cpu.step(g)
+        assert np.array_equal(bits(gpu.error()), bits(cpu.error()))
+        assert rel_l2(uv.cpu().numpy(), u_ref) <= U_TOL
+
+
+def test_large_d_short_window_wraps():
+    # large d with a short window so that the ring wraps at a size spanning many slabs
+    d, m, k = 3_000_017, 8, 30_000
+    rng = np.random.default_rng(14)
+    scale = np.exp(rng.standard_normal(d)).astype(np.float32)
+    grads = ((scale * rng.standard_normal(d).astype(np.float32)) for _ in range(19))
+    run_parity(d, m, k, 1e-4, grads, check_rows="all", gram_every=6)
+
+
+def test_nonfinite_gradient_sets_status():
+    B = _binding()
+    d = 1000
+    gpu = B.Efcp(d, 2, 10, 1e-3)
+    g = torch.randn(d, device="cuda")
+    g[17] = float("inf")
+    u = torch.empty_like(g)
+    gpu.step(g, u)
+    assert gpu.status() == B.ENUMERIC
+
+
+def test_argument_errors():
+    B = _binding()
+    for args in ((0, 1, 1, 1e-3), (4, 0, 1, 1e-3), (4, 1, 0, 1e-3), (4, 1, 5, 1e-3),
+                 (4, 1, 1, 0.0), (4, 1, 1, float("inf")), (2 ** 31, 1, 1, 1e-3), (4, 5000, 1, 1e-3)):
+        with pytest.raises(B.EfcpError) as ei:
+            B.Efcp(*args)
+        assert ei.value.code == B.EINVAL
+    gpu = B.Efcp(16, 2, 4, 1e-3)
+    g = torch.zeros(16, device="cuda")
+    with pytest.raises(B.EfcpError):
+        gpu.step_ptr(0, g.data_ptr())
+    with pytest.raises(B.EfcpError):
+        gpu.step_ptr(g.data_ptr(), g.data_ptr())  # update must not alias grad
+    assert B.state_bytes(0, 1, 1) == -1
+
+
+def test_host_entry_point_matches_device_entry_point():
+    B = _binding()
+    d, m, k = 200_000, 8, 2000
+    rng = np.random.default_rng(15)
+    a, b = B.Efcp(d, m, k, 1e-3), B.Efcp(d, m, k, 1e-3)
+    gh = torch.empty(d, dtype=torch.float32).pin_memory()
+    uh = torch.empty(d, dtype=torch.float32).pin_memory()
+    gd = torch.empty(d, dtype=torch.float32, device="cuda")
+    ud = torch.empty(d, dtype=torch.float32, device="cuda")
+    for t in range(10):
+        gh.copy_(torch.from_numpy(rng.standard_normal(d).astype(np.float32)))
+        gd.copy_(gh)
+        a.step(gd, ud)
+        b.step_host(gh, uh)
+        assert np.array_equal(bits(a.error()), bits(b.error()))
+        assert rel_l2(uh.numpy(), ud.cpu().numpy()) <= 1e-5
