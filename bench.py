@@ -1,0 +1,322 @@
+#!/usr/bin/env python
+"""EFCP optimizer-step benchmark (one JSON line on stdout, printed by rank 0).
+
+A "step" is one pass of the whole hot path over one synthetic gradient:
+error feedback -> exact Top-k -> residual -> ring insert -> scalar products ->
+m x m coefficients -> linear combination (one efcp_step call).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME]
+  python -m torch.distributed.run --nproc-per-node N ... bench.py --gpus N ...
+  python bench.py --impl reference ...        # the CPU oracle, timed on the host cores
+
+N > 1 runs N independent replicas (one optimizer state per GPU, no data-path
+collective): weak scaling.  Before timing, the ring window is filled completely
+(m untimed steps) so that the timed steps are steady-state steps.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2306_06098_b200 import gradgen  # noqa: E402
+
+METRIC = "efcp_steps_per_sec"
+UNIT = "steps/s"
+
+# DRAM traffic per launch of the dominant kernels from the ncu captures summarised under
+# profiles/ (dram__bytes_read.sum + dram__bytes_write.sum), keyed by workload; None until
+# a capture of that workload exists.  Scaled from a smaller capture where noted there.
+NCU_TRAFFIC_BYTES = {}
+
+
+def load_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    return 6650.0, "fallback (earlier pool measurement)"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU with nvidia-smi while timing."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, pw = [], [], []
+        reasons = set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in out.strip().splitlines():
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+                pw.append(float(parts[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(pw) if pw else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def dist_setup(n_gpus):
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        backend = "nccl" if torch.cuda.is_available() else "gloo"
+        dist.init_process_group(backend=backend)
+    return world, rank, local
+
+
+def barrier(world):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+
+
+def max_over_ranks(x, world, device):
+    if world == 1:
+        return x
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def oracle_steps_per_sec(w, grads_host, n_steps):
+    """Times the CPU oracle as it stands on `n_steps` gradients of workload w."""
+    from oracle import ref
+    o = ref.RefEFCP(w.d, w.m, w.k, w.lam)
+    t0 = time.perf_counter()
+    for i in range(n_steps):
+        o.step(grads_host[i % len(grads_host)])
+    dt = time.perf_counter() - t0
+    o.close()
+    return n_steps / dt, ref.num_threads(), dt
+
+
+def run_reference(args, world, rank):
+    """The reference arm: the CPU oracle on a bounded slice of the same workload."""
+    if rank != 0:
+        return
+    w = gradgen.WORKLOADS[args.workload]
+    # Oracle cost per step is close to linear in d (with k/d and m fixed).  Shrink d and k
+    # by `shrink` so that warmup + steps stay within a few minutes, report steps/s divided
+    # by the same factor.
+    est_full = 9e-8 * w.d + 1.3e-9 * w.m * w.k * 2 + 1.2e-10 * w.m ** 3  # seconds, 8 cores
+    budget = 150.0 / max(1, args.steps + args.warmup)
+    shrink = 1
+    while est_full / shrink > budget and w.d // (shrink * 2) >= 4096:
+        shrink *= 2
+    d, k = w.d // shrink, max(1, w.k // shrink)
+    small = gradgen.Workload(w.name, d, w.m, k, w.lam, w.steps, w.rank, w.scale_block, w.seed)
+    gs = gradgen.GradStream.for_workload(small, "cpu")
+    from oracle import ref
+    o = ref.RefEFCP(d, w.m, k, w.lam)
+    grads = [gs.next().numpy() for _ in range(min(4, args.steps + args.warmup))]
+    for i in range(args.warmup):
+        o.step(grads[i % len(grads)])
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        o.step(grads[(args.warmup + i) % len(grads)])
+    dt = time.perf_counter() - t0
+    value = args.steps / dt / shrink
+    sample = (f"oracle on d={d}, k={k}, m={w.m} (the workload with d and k divided by {shrink}); "
+              f"steps/s divided by {shrink} (cost is linear in d at fixed density and m)")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT,
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": 1e3 / value, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "d": w.d, "m": w.m, "k": w.k, "lambda": w.lam},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": ref.num_threads(),
+                         "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=40)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=gradgen.C4.name, choices=sorted(gradgen.WORKLOADS))
+    ap.add_argument("--prefill", type=int, default=-1,
+                    help="untimed steps before warm-up; -1 = m (fill the whole window)")
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--cpu-steps", type=int, default=2)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    world, rank, local = dist_setup(args.gpus)
+    if args.impl == "reference":
+        run_reference(args, world, rank)
+        return
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (no CPU fallback)")
+    from paper_2306_06098_b200 import binding  # fails loudly when the library is missing
+
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    w = gradgen.WORKLOADS[args.workload]
+    K, W = args.steps, args.warmup
+    gs = gradgen.GradStream(w.d, w.rank, w.seed + rank, w.scale_block, w.noise, str(device))
+    opt = binding.Efcp(w.d, w.m, w.k, w.lam)
+    gbuf = torch.empty(w.d, dtype=torch.float32, device=device)
+    ubuf = torch.empty(w.d, dtype=torch.float32, device=device)
+
+    prefill = w.m if args.prefill < 0 else args.prefill
+    for _ in range(prefill):
+        gs.next(out=gbuf)
+        opt.step(gbuf, ubuf)
+    torch.cuda.synchronize()
+    assert opt.status() == 0, binding.strerror(opt.status())
+
+    # inputs of the timed region: resident in HBM before it starts
+    pool_n = min(K + W, 128)
+    pool = [gs.next().clone() for _ in range(pool_n)]
+    del gs  # frees U
+    torch.cuda.empty_cache()
+
+    for i in range(W):
+        opt.step(pool[i % pool_n], ubuf)
+    torch.cuda.synchronize()
+    barrier(world)
+    try:  # nvidia-smi numbering ignores CUDA_VISIBLE_DEVICES: address the GPU by UUID
+        gpu_id = "GPU-" + str(torch.cuda.get_device_properties(local).uuid).replace("GPU-", "")
+    except Exception:
+        gpu_id = str(local)
+    sampler = ClockSampler(gpu_id)
+    sampler.start()
+    time.sleep(0.3)
+    stream = torch.cuda.current_stream()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    opt.profile_begin(K)
+    torch.cuda.synchronize()
+    ev0.record(stream)
+    for i in range(K):
+        opt.step(pool[(W + i) % pool_n], ubuf, stream)
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    barrier(world)
+    clocks = sampler.stop()
+    ms_total = max_over_ranks(ev0.elapsed_time(ev1), world, device)
+    stages, n_rec = opt.profile_end()
+    launches = opt.launches_per_step * K
+    assert opt.status() == 0, binding.strerror(opt.status())
+    ms_per_step = ms_total / K
+    value = world * K / (ms_total * 1e-3)
+
+    # end to end: host buffers, copies inside the timed region
+    e2e = None
+    if args.e2e_steps > 0:
+        gh = torch.empty(w.d, dtype=torch.float32).pin_memory()
+        uh = torch.empty(w.d, dtype=torch.float32).pin_memory()
+        gh.copy_(pool[0])
+        opt.step_host(gh, uh)  # allocates the staging buffers
+        barrier(world)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for i in range(args.e2e_steps):
+            opt.step_host(gh, uh)
+        torch.cuda.synchronize()
+        dt = max_over_ranks(time.perf_counter() - t0, world, device)
+        e2e = {"value": world * args.e2e_steps / dt, "unit": UNIT,
+               "h2d_bytes_per_step": 4 * w.d, "d2h_bytes_per_step": 4 * w.d,
+               "steps": args.e2e_steps}
+
+    # roofline of the dominant kernel (HBM bound): algorithmic bytes per launch / time
+    peak, peak_src = load_peak()
+    alg = {"sp": 8 * w.m * w.k, "lcg": 8 * w.m * w.k + 4 * w.d}
+    kern = max(("sp", "lcg"), key=lambda s: stages[s])
+    avg_ms = stages[kern] / max(n_rec, 1)
+    achieved = alg[kern] / (avg_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": {"sp": "k_sp_rows", "lcg": "k_lcg"}[kern],
+                "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "traffic": NCU_TRAFFIC_BYTES.get(w.name, {}).get(kern),
+                "peak_source": peak_src, "algorithmic_bytes_per_launch": alg[kern],
+                "avg_launch_ms": avg_ms}
+    step_bytes = 16 * w.m * w.k + 16 * w.d + 8 * w.k
+    step_gbs = step_bytes / (ms_per_step * 1e-3) / 1e9
+    stage_ms = {s: stages[s] / max(n_rec, 1) for s in stages}
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and args.cpu_steps > 0:
+        grads_host = [pool[i].cpu().numpy() for i in range(min(2, pool_n))]
+        v, cores, dt = oracle_steps_per_sec(w, grads_host, args.cpu_steps)
+        cpu_baseline = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
+                        "sample": f"{args.cpu_steps} full steps of {w.name} from an empty window "
+                                  f"(the oracle loops over all m rows whether written or not), "
+                                  f"{dt:.1f} s"}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K,
+            "warmup": W, "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": w.name, "d": w.d, "m": w.m, "k": w.k, "lambda": w.lam,
+                       "rhs": "compressed", "prefill_steps": prefill,
+                       "parallelism": f"replicas x{world}",
+                       "l2": "inputs larger than L2 (window %.2f GB, gradient %.2f GB)" % (
+                           8 * w.m * w.k / 1e9, 4 * w.d / 1e9)},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
+            "roofline": roofline,
+            "step_hbm": {"algorithmic_bytes_per_step": step_bytes, "achieved_gbs": step_gbs,
+                         "frac_of_peak": step_gbs / peak, "frac_of_8tbs": step_gbs / 8000.0},
+            "stage_ms": stage_ms,
+            "cpu_baseline": cpu_baseline,
+        }
+        print(json.dumps(line), flush=True)
+    opt.close()
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -123,6 +123,22 @@ int64_t efcp_state_bytes(int64_t d, int32_t m, int64_t k);
 /* Number of kernels one efcp_step launches for this handle. */
 int32_t efcp_launches_per_step(efcp_ctx* ctx);
 
+/*
+ * Stage timing with CUDA events recorded on the step's own stream.
+ *   efcp_profile_begin : from the next efcp_step on, record events around the four
+ *                        stages of a step, for at most max_steps steps (1..4096).
+ *   efcp_profile_end   : waits for the device, adds up the elapsed times of the steps
+ *                        recorded since efcp_profile_begin and stops recording.
+ *                        ms_out (host, 4 doubles) receives the totals in milliseconds:
+ *                        [0] error feedback + Top-k + ring insert (Algorithm 1 lines 5-7),
+ *                        [1] the scalar-product (SP) kernel alone,
+ *                        [2] the m x m stage,
+ *                        [3] the linear-combination (LCG) kernel alone;
+ *                        *steps_out (host) receives the number of steps recorded.
+ */
+int efcp_profile_begin(efcp_ctx* ctx, int32_t max_steps);
+int efcp_profile_end(efcp_ctx* ctx, double* ms_out, int32_t* steps_out);
+
 /* Static description of an EFCP_* code. */
 const char* efcp_strerror(int code);
 

@@ -40,6 +40,8 @@ EXPORTS = {
     "efcp_last_residual": ([_vp], C.c_double),
     "efcp_state_bytes": ([_i64, _i32, _i64], _i64),
     "efcp_launches_per_step": ([_vp], _i32),
+    "efcp_profile_begin": ([_vp, _i32], C.c_int),
+    "efcp_profile_end": ([_vp, _vp, _vp], C.c_int),
     "efcp_strerror": ([C.c_int], C.c_char_p),
 }
 for _name, (_args, _res) in EXPORTS.items():
@@ -134,6 +136,17 @@ class Efcp:
 
     def last_residual(self) -> float:
         return float(_lib.efcp_last_residual(self._h))
+
+    def profile_begin(self, max_steps: int):
+        self._check(_lib.efcp_profile_begin(self._h, max_steps), "efcp_profile_begin")
+
+    def profile_end(self):
+        """Returns ({stage: total ms}, steps recorded)."""
+        ms = (C.c_double * 4)()
+        n = C.c_int32()
+        self._check(_lib.efcp_profile_end(self._h, C.cast(ms, C.c_void_p),
+                                          C.cast(C.byref(n), C.c_void_p)), "efcp_profile_end")
+        return dict(zip(("ef_topk", "sp", "mxm", "lcg"), list(ms))), int(n.value)
 
     def error(self) -> np.ndarray:
         out = np.empty(self.d, np.float32)

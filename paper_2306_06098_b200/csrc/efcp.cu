@@ -51,6 +51,10 @@ struct efcp_ctx {
   float* stage_u = nullptr;
   int last_cuda = 0;
   int launches = 0;
+  // stage timing (efcp_profile_*): 5 events per recorded step
+  std::vector<cudaEvent_t> prof_ev;
+  int prof_cap = 0, prof_n = 0;
+  bool prof_on = false;
   std::vector<void*> allocs;
 };
 
@@ -159,6 +163,13 @@ int sync_status(efcp_ctx* ctx) {
 void free_all(efcp_ctx* ctx) {
   for (void* p : ctx->allocs) cudaFree(p);
   ctx->allocs.clear();
+  for (cudaEvent_t ev : ctx->prof_ev) cudaEventDestroy(ev);
+  ctx->prof_ev.clear();
+}
+
+inline void prof_mark(efcp_ctx* ctx, int which, cudaStream_t st) {
+  if (ctx->prof_on && ctx->prof_n < ctx->prof_cap)
+    cudaEventRecord(ctx->prof_ev[size_t(ctx->prof_n) * 5 + which], st);
 }
 
 }  // namespace
@@ -288,6 +299,7 @@ int efcp_step(efcp_ctx* ctx, const float* grad, float* update, void* stream_) {
   double* dw = res + m;
   const double mlambda = double(m) * double(ctx->lambda);
 
+  prof_mark(ctx, 0, st);
   // a = xi + g, digit-1 histogram
   const int ef_grid = ctx->num_sms * 2;
   if ((reinterpret_cast<uintptr_t>(grad) & 15) == 0)
@@ -328,9 +340,11 @@ int efcp_step(efcp_ctx* ctx, const float* grad, float* update, void* stream_) {
   EFCP_LAUNCHED();
   // scalar products with the new row, Gram row/column
   const size_t smem = slab_smem_bytes(ctx->W, m);
+  prof_mark(ctx, 1, st);
   k_sp_rows<<<ctx->grid_slab, 1024, smem, st>>>(ctx->I, ctx->V, ctx->offs, k, m, ctx->W,
                                                 ctx->n_slabs, slot, ctx->partial);
   EFCP_LAUNCHED();
+  prof_mark(ctx, 2, st);
   k_sp_finish<<<(m + 127) / 128, 128, 0, st>>>(ctx->partial, ctx->grid_slab, m, slot, delta,
                                                ctx->S, aprime);
   EFCP_LAUNCHED();
@@ -350,6 +364,7 @@ int efcp_step(efcp_ctx* ctx, const float* grad, float* update, void* stream_) {
   k_refine_finish<<<1, 1024, 0, st>>>(w, dw, res, ctx->wf, m, ctx->sc);
   EFCP_LAUNCHED();
   // linear combination of the window rows
+  prof_mark(ctx, 3, st);
   if ((reinterpret_cast<uintptr_t>(update) & 15) == 0)
     k_lcg<true><<<ctx->grid_slab, 1024, smem, st>>>(ctx->I, ctx->V, ctx->offs, k, m, ctx->W,
                                                     ctx->n_slabs, ctx->wf, update, d);
@@ -357,6 +372,8 @@ int efcp_step(efcp_ctx* ctx, const float* grad, float* update, void* stream_) {
     k_lcg<false><<<ctx->grid_slab, 1024, smem, st>>>(ctx->I, ctx->V, ctx->offs, k, m, ctx->W,
                                                      ctx->n_slabs, ctx->wf, update, d);
   EFCP_LAUNCHED();
+  prof_mark(ctx, 4, st);
+  if (ctx->prof_on && ctx->prof_n < ctx->prof_cap) ++ctx->prof_n;
   ctx->t += 1;
   return EFCP_OK;
 }
@@ -431,5 +448,38 @@ double efcp_last_residual(efcp_ctx* ctx) {
 }
 
 int32_t efcp_launches_per_step(efcp_ctx* ctx) { return ctx ? ctx->launches : -1; }
+
+int efcp_profile_begin(efcp_ctx* ctx, int32_t max_steps) {
+  if (!ctx || max_steps < 1 || max_steps > 4096) return EFCP_EINVAL;
+  EFCP_CUDA(cudaSetDevice(ctx->device));
+  while (int(ctx->prof_ev.size()) < max_steps * 5) {
+    cudaEvent_t ev;
+    EFCP_CUDA(cudaEventCreate(&ev));
+    ctx->prof_ev.push_back(ev);
+  }
+  ctx->prof_cap = max_steps;
+  ctx->prof_n = 0;
+  ctx->prof_on = true;
+  return EFCP_OK;
+}
+
+int efcp_profile_end(efcp_ctx* ctx, double* ms_out, int32_t* steps_out) {
+  if (!ctx || !ms_out || !steps_out) return EFCP_EINVAL;
+  ctx->prof_on = false;
+  EFCP_CUDA(cudaSetDevice(ctx->device));
+  EFCP_CUDA(cudaDeviceSynchronize());
+  for (int q = 0; q < 4; ++q) ms_out[q] = 0.0;
+  for (int i = 0; i < ctx->prof_n; ++i) {
+    for (int q = 0; q < 4; ++q) {
+      float ms = 0.f;
+      EFCP_CUDA(cudaEventElapsedTime(&ms, ctx->prof_ev[size_t(i) * 5 + q],
+                                     ctx->prof_ev[size_t(i) * 5 + q + 1]));
+      ms_out[q] += double(ms);
+    }
+  }
+  *steps_out = ctx->prof_n;
+  ctx->prof_n = 0;
+  return EFCP_OK;
+}
 
 }  // extern "C"
