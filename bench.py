@@ -192,10 +192,11 @@ def main():
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
-    world, rank, local = dist_setup(args.gpus)
     if args.impl == "reference":
-        run_reference(args, world, rank)
+        # rank 0 alone runs the oracle; no process group is needed for that
+        run_reference(args, int(os.environ.get("WORLD_SIZE", "1")), int(os.environ.get("RANK", "0")))
         return
+    world, rank, local = dist_setup(args.gpus)
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (no CPU fallback)")

@@ -1,0 +1,99 @@
+"""The C-ABI library against its header, and the host-side logic that needs no GPU."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+HEADER = os.path.join(ROOT, "include", "efcp.h")
+
+
+def declared_functions():
+    """Names of every function include/efcp.h declares (comments stripped first)."""
+    src = open(HEADER).read()
+    src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+    src = re.sub(r"^\s*#.*$", "", src, flags=re.M)
+    return sorted(set(re.findall(r"\b(efcp_[a-z0-9_]+)\s*\(", src)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2306_06098_b200 import build
+    return C.CDLL(build.build())
+
+
+def test_header_declares_the_problem_statement_calls():
+    names = declared_functions()
+    for must in ("efcp_create", "efcp_step", "efcp_destroy"):
+        assert must in names
+
+
+def test_library_exports_every_declared_symbol(lib):
+    missing = [n for n in declared_functions() if not hasattr(lib, n)]
+    assert not missing, missing
+
+
+def test_binding_covers_every_declared_symbol(lib):
+    from paper_2306_06098_b200 import binding
+    assert sorted(binding.EXPORTS) == declared_functions()
+
+
+def test_strerror_and_state_bytes_need_no_device(lib):
+    lib.efcp_strerror.restype = C.c_char_p
+    lib.efcp_strerror.argtypes = [C.c_int]
+    seen = {lib.efcp_strerror(c) for c in range(0, -7, -1)}
+    assert len(seen) == 7 and all(seen)
+    assert lib.efcp_strerror(-99) not in seen
+    lib.efcp_state_bytes.restype = C.c_int64
+    lib.efcp_state_bytes.argtypes = [C.c_int64, C.c_int32, C.c_int64]
+    for bad in ((0, 1, 1), (4, 0, 1), (4, 1, 0), (4, 1, 5), (2 ** 31, 1, 1), (4, 5000, 1)):
+        assert lib.efcp_state_bytes(*bad) == -1
+    d, m, k = 109_482_240, 1024, 1_094_822
+    b = lib.efcp_state_bytes(d, m, k)
+    # window (8mk) + error buffer (4d) are the floor; scratch stays within a few d-vectors
+    assert 8 * m * k + 4 * d <= b <= 8 * m * k + 4 * d + 16 * d + (64 << 20)
+
+
+def test_null_handles_are_rejected_without_a_device(lib):
+    lib.efcp_step_count.restype = C.c_int64
+    lib.efcp_step_count.argtypes = [C.c_void_p]
+    assert lib.efcp_step_count(None) == -1
+    lib.efcp_status.argtypes = [C.c_void_p]
+    assert lib.efcp_status(None) == -1
+    lib.efcp_destroy.argtypes = [C.c_void_p]
+    assert lib.efcp_destroy(None) == -1
+    lib.efcp_step.argtypes = [C.c_void_p] * 4
+    assert lib.efcp_step(None, None, None, None) == -1
+
+
+def golden_rows():
+    rows = {}
+    with open(os.path.join(ROOT, "tests", "golden", "memory_savings.txt")) as f:
+        for line in f:
+            line = line.split("#")[0].strip()
+            if line:
+                key, val = line.split("=")
+                rows[key.strip()] = float(val)
+    return rows
+
+
+def test_footprint_formula_reproduces_the_papers_memory_figures():
+    """Appendix "Memory savings" (m = 1024, k = d/100): ~90d bytes with fp32 values, ~70d
+    with bf16 values, 45.5x / 58.5x below the dense 4md; and the dense window of the
+    BERT-base run is the 417 GB the experiments section quotes."""
+    from paper_2306_06098_b200 import binding
+    gold = golden_rows()
+    d = 100_000_000
+    m, k = 1024, d // 100
+    f32 = binding.paper_state_bytes(d, m, k, 4)
+    b16 = binding.paper_state_bytes(d, m, k, 2)
+    assert abs(f32 / d - gold["sparse_bytes_per_d_fp32"]) < 0.01
+    assert abs(b16 / d - gold["sparse_bytes_per_d_bf16"]) < 0.01
+    dense = 4 * m * d
+    assert dense / d == gold["dense_bytes_per_d"]
+    # the paper rounds the footprints to 90d and 70d before dividing
+    assert abs(dense / (round(f32 / d, -1) * d) - gold["saving_fp32"]) < 0.05
+    assert abs(dense / (round(b16 / d, -1) * d) - gold["saving_bf16"]) < 0.05
+    from paper_2306_06098_b200 import gradgen
+    assert 4 * 1024 * gradgen.C4.d // 2 ** 30 == gold["bert_base_dense_window_gib"]  # 417.6
