@@ -30,6 +30,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
            "-gencode", "arch=compute_100a,code=sm_100a",
            "-Xcompiler", "-fPIC", "-shared", "-I", INCLUDE, "-I", CSRC,
            "-o", LIB + ".tmp"] + _sources()
+    cmd[1:1] = os.environ.get("EFCP_NVCC_FLAGS", "").split()  # e.g. -DEFCP_DEPTH=8
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")

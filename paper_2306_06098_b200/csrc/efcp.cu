@@ -5,11 +5,13 @@
 
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cmath>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
 #include <new>
+#include <utility>
 #include <vector>
 
 #include "efcp_common.cuh"
@@ -41,6 +43,8 @@ struct efcp_ctx {
   int32_t* chunk_off = nullptr;
   int32_t* cand_idx = nullptr;
   float* cand_val = nullptr;
+  int32_t* sel_idx = nullptr;  // the selection of the current step, ascending (k entries)
+  float* sel_val = nullptr;
   int32_t* sel_gt = nullptr;
   int32_t* sel_eq = nullptr;
   Scalars* sc = nullptr;
@@ -69,7 +73,7 @@ int pick_slab_width(int64_t d, int m, int num_sms) {
   int W = 32768;
   if (const char* env = getenv("EFCP_SLAB_W")) {
     const int v = atoi(env);
-    if (v >= 256 && v <= 49152 && (v & 3) == 0) return v;
+    if (v >= 256 && v <= 49152 && (v & 31) == 0) return v;
   }
   // shared memory: W*4 + 16*m must stay under the 227 KB per-block limit
   while (size_t(W) * 4 + size_t(m) * 16 > 200 * 1024 && W > 1024) W >>= 1;
@@ -94,6 +98,7 @@ Sizes compute_sizes(int64_t d, int32_t m, int64_t k, int num_sms) {
   b += align256((kBins1 + kBins2 + kBins3) * 4);          // hist
   b += 3 * align256(int64_t(z.n_chunks + 1) * 4);         // chunk_off, sel_gt, sel_eq
   b += 2 * align256(d * 4);                               // cand_idx, cand_val
+  b += 2 * align256(k * 4);                               // sel_idx, sel_val
   b += align256(sizeof(Scalars));
   b += align256(int64_t(z.grid_slab) * m * 8);            // partial
   b += align256(int64_t(8) * m * 8);                      // vecs
@@ -236,6 +241,8 @@ int efcp_create_ex(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float lambda
   if ((rc = dev_alloc(ctx, &ctx->sel_eq, int64_t(z.n_chunks + 1) * 4))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->cand_idx, d * 4))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->cand_val, d * 4))) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->sel_idx, k * 4))) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->sel_val, k * 4))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->sc, sizeof(Scalars)))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->partial, int64_t(z.grid_slab) * m * 8))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->vecs, int64_t(8) * m * 8))) return fail(rc);
@@ -331,17 +338,16 @@ int efcp_step(efcp_ctx* ctx, const float* grad, float* update, void* stream_) {
   k_scan_sel<<<1, 1024, 0, st>>>(ctx->sel_gt, ctx->sel_eq, ctx->sc, uint32_t(k));
   EFCP_LAUNCHED();
   k_write_sel<<<cand_grid, kChunkThreads, 0, st>>>(ctx->cand_idx, ctx->cand_val, ctx->sc,
-                                                   ctx->sel_gt, ctx->sel_eq, row_idx, row_val,
-                                                   ctx->e, k);
+                                                   ctx->sel_gt, ctx->sel_eq, ctx->sel_idx,
+                                                   ctx->sel_val, ctx->e, k);
   EFCP_LAUNCHED();
-  k_build_offsets<<<(ctx->n_slabs + 1 + 255) / 256, 256, 0, st>>>(row_idx, k, ctx->W,
-                                                                  ctx->n_slabs, m, slot,
-                                                                  ctx->offs);
+  k_layout_row<<<(ctx->n_slabs + kLayoutWarps) / kLayoutWarps, kLayoutWarps * 32, 0, st>>>(
+      ctx->sel_idx, ctx->sel_val, k, ctx->W, ctx->n_slabs, m, slot, ctx->offs, row_idx, row_val);
   EFCP_LAUNCHED();
   // scalar products with the new row, Gram row/column
   const size_t smem = slab_smem_bytes(ctx->W, m);
   prof_mark(ctx, 1, st);
-  k_sp_rows<<<ctx->grid_slab, 1024, smem, st>>>(ctx->I, ctx->V, ctx->offs, k, m, ctx->W,
+  k_sp_rows<<<ctx->grid_slab, kSlabThreads, smem, st>>>(ctx->I, ctx->V, ctx->offs, k, m, ctx->W,
                                                 ctx->n_slabs, slot, ctx->partial);
   EFCP_LAUNCHED();
   prof_mark(ctx, 2, st);
@@ -366,10 +372,10 @@ int efcp_step(efcp_ctx* ctx, const float* grad, float* update, void* stream_) {
   // linear combination of the window rows
   prof_mark(ctx, 3, st);
   if ((reinterpret_cast<uintptr_t>(update) & 15) == 0)
-    k_lcg<true><<<ctx->grid_slab, 1024, smem, st>>>(ctx->I, ctx->V, ctx->offs, k, m, ctx->W,
+    k_lcg<true><<<ctx->grid_slab, kSlabThreads, smem, st>>>(ctx->I, ctx->V, ctx->offs, k, m, ctx->W,
                                                     ctx->n_slabs, ctx->wf, update, d);
   else
-    k_lcg<false><<<ctx->grid_slab, 1024, smem, st>>>(ctx->I, ctx->V, ctx->offs, k, m, ctx->W,
+    k_lcg<false><<<ctx->grid_slab, kSlabThreads, smem, st>>>(ctx->I, ctx->V, ctx->offs, k, m, ctx->W,
                                                      ctx->n_slabs, ctx->wf, update, d);
   EFCP_LAUNCHED();
   prof_mark(ctx, 4, st);
@@ -409,6 +415,22 @@ int efcp_get_row(efcp_ctx* ctx, int32_t slot, int32_t* host_idx, float* host_val
   const size_t bytes = size_t(ctx->k) * 4;
   EFCP_CUDA(cudaMemcpy(host_idx, ctx->I + int64_t(slot) * ctx->k, bytes, cudaMemcpyDeviceToHost));
   EFCP_CUDA(cudaMemcpy(host_val, ctx->V + int64_t(slot) * ctx->k, bytes, cudaMemcpyDeviceToHost));
+  // the device keeps every slab segment of a row in a bank-interleaved order; callers get
+  // the row in ascending index order (indices within a row are distinct)
+  try {
+    std::vector<std::pair<int32_t, float>> tmp(static_cast<size_t>(ctx->k));
+    for (int64_t j = 0; j < ctx->k; ++j) tmp[size_t(j)] = {host_idx[j], host_val[j]};
+    std::sort(tmp.begin(), tmp.end(),
+              [](const std::pair<int32_t, float>& a, const std::pair<int32_t, float>& b) {
+                return a.first < b.first;
+              });
+    for (int64_t j = 0; j < ctx->k; ++j) {
+      host_idx[j] = tmp[size_t(j)].first;
+      host_val[j] = tmp[size_t(j)].second;
+    }
+  } catch (const std::bad_alloc&) {
+    return EFCP_ENOMEM;
+  }
   return rc;
 }
 

@@ -1,11 +1,11 @@
 // Sparse ring-buffer window G = (I, V) and its two primitives (Section 3.1, "Sparse
 // Scalar Products" and "Sparse LCG"; Appendix "CUDA Kernels").
 //
-// Layout: I (int32) and V (fp32) are m x k row-major, one row per ring slot, every row
-// sorted by ascending index.  The coordinate range [0, d) is cut into slabs of W
-// coordinates; offs[s * m + r] is the position inside row r of its first entry with
-// index >= s * W (offs has n_slabs + 1 slab rows), so the entries of row r that fall in
-// slab s are the contiguous range [offs[s][r], offs[s+1][r]).
+// Layout: I (int32) and V (fp32) are m x k row-major, one row per ring slot.  The
+// coordinate range [0, d) is cut into slabs of W coordinates (W a multiple of 32);
+// offs[s * m + r] is the number of entries of row r with index < s * W (offs has
+// n_slabs + 1 slab rows), so the entries of row r that fall in slab s are the contiguous
+// range [offs[s][r], offs[s+1][r]) of the row: its segment in that slab.
 //
 // Both primitives are slab-major: a block owns a slab, keeps the dense slab of the
 // right-hand side (SP) or of the output (LCG) in shared memory, and streams the
@@ -14,25 +14,98 @@
 // replaces the paper's block-wise Top-k (which fixes the segment boundaries by
 // construction) with a small table written when a row is inserted, so Top-k can stay
 // global.
+//
+// Order inside a segment.  A warp takes 32 consecutive entries of a segment at a time and
+// uses their indices as shared-memory addresses, so what matters for speed is how many
+// of the 32 fall into the same bank (index mod 32).  Neither primitive depends on the
+// order of the entries inside a segment, so the insert kernel stores every chunk of 512
+// entries (counted from the segment start) sorted by (occurrence number of the entry's
+// bank, bank): the first entry of every bank, then the second of every bank, and so on.
+// Every aligned group of 32 then holds mostly distinct banks.  efcp_get_row returns rows
+// in ascending index order again.
 #pragma once
 
 #include "efcp_common.cuh"
 
 namespace efcp {
 
-// offs[s][slot] = lower_bound(row, s * W) for s = 0..n_slabs.
-__global__ void __launch_bounds__(256) k_build_offsets(const int32_t* __restrict__ row_idx,
-                                                        int64_t k, int W, int n_slabs, int m,
-                                                        int slot, int32_t* __restrict__ offs) {
-  const int s = blockIdx.x * blockDim.x + threadIdx.x;
+constexpr int kLayoutChunk = 512;   // entries permuted together (a multiple of 32)
+constexpr int kLayoutWarps = 8;     // warps (= slabs) per block of k_layout_row
+
+// Insert of the new row: from the ascending (index, value) list of the selection,
+//   offs[s][slot] = lower_bound(row, s * W) for s = 0..n_slabs, and
+//   ring slot <- the row, every segment in the bank-interleaved order described above.
+// One warp per slab.
+__global__ void __launch_bounds__(kLayoutWarps * 32) k_layout_row(
+    const int32_t* __restrict__ src_idx, const float* __restrict__ src_val, int64_t k, int W,
+    int n_slabs, int m, int slot, int32_t* __restrict__ offs, int32_t* __restrict__ dst_idx,
+    float* __restrict__ dst_val) {
+  __shared__ int32_t s_idx[kLayoutWarps][kLayoutChunk];
+  __shared__ float s_val[kLayoutWarps][kLayoutChunk];
+  __shared__ uint16_t s_q[kLayoutWarps][kLayoutChunk];
+  __shared__ int s_cnt[kLayoutWarps][32];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int s = blockIdx.x * kLayoutWarps + warp;
   if (s > n_slabs) return;
-  const int64_t target = int64_t(s) * W;
-  int64_t lo = 0, hi = k;
-  while (lo < hi) {
-    const int64_t mid = (lo + hi) >> 1;
-    if (int64_t(row_idx[mid]) < target) lo = mid + 1; else hi = mid;
+  // lane 0 finds the segment start, lane 1 its end
+  int64_t bound = 0;
+  if (lane < 2) {
+    const int64_t target = int64_t(s + lane) * W;
+    int64_t lo = 0, hi = k;
+    while (lo < hi) {
+      const int64_t mid = (lo + hi) >> 1;
+      if (int64_t(src_idx[mid]) < target) lo = mid + 1; else hi = mid;
+    }
+    bound = lo;
   }
-  offs[int64_t(s) * m + slot] = int32_t(lo);
+  const int seg_b = int(__shfl_sync(0xFFFFFFFFu, bound, 0));
+  const int seg_e = s < n_slabs ? int(__shfl_sync(0xFFFFFFFFu, bound, 1)) : seg_b;
+  if (lane == 0) offs[int64_t(s) * m + slot] = seg_b;
+  int32_t* ci = s_idx[warp];
+  float* cv = s_val[warp];
+  uint16_t* cq = s_q[warp];
+  int* cnt = s_cnt[warp];
+  for (int c0 = seg_b; c0 < seg_e; c0 += kLayoutChunk) {
+    const int n = min(kLayoutChunk, seg_e - c0);
+    cnt[lane] = 0;
+    __syncwarp();
+    // occurrence number of every entry within its bank, in ascending index order
+    for (int a0 = 0; a0 < n; a0 += 32) {
+      const int a = a0 + lane;
+      const bool on = a < n;
+      int idx = 0;
+      if (on) {
+        idx = src_idx[c0 + a];
+        ci[a] = idx;
+        cv[a] = src_val[c0 + a];
+      }
+      const int bank = idx & 31;
+      const unsigned same = __match_any_sync(0xFFFFFFFFu, on ? bank : 32 + lane);
+      const int before = on ? cnt[bank] : 0;
+      __syncwarp();
+      if (on) {
+        cq[a] = uint16_t(before + __popc(same & ((1u << lane) - 1u)));
+        if ((same & ((1u << lane) - 1u)) == 0u) cnt[bank] = before + __popc(same);
+      }
+      __syncwarp();
+    }
+    // position in the (occurrence, bank) order
+    for (int a0 = 0; a0 < n; a0 += 32) {
+      const int a = a0 + lane;
+      if (a < n) {
+        const int idx = ci[a], bank = idx & 31, q = cq[a];
+        int pos = 0;
+#pragma unroll 8
+        for (int bb = 0; bb < 32; ++bb) {
+          const int c = cnt[bb];
+          pos += min(c, q) + ((bb < bank && c > q) ? 1 : 0);
+        }
+        dst_idx[c0 + pos] = idx;
+        dst_val[c0 + pos] = cv[a];
+      }
+    }
+    __syncwarp();
+  }
 }
 
 // Shared-memory layout of the slab kernels: float slab[W]; double/float per-row
@@ -41,10 +114,19 @@ __host__ __device__ inline size_t slab_smem_bytes(int W, int m) {
   return size_t(W) * 4 + size_t(m) * 8 + size_t(m) * 8;
 }
 
+#ifndef EFCP_SLAB_THREADS
+#define EFCP_SLAB_THREADS 1024
+#endif
+#ifndef EFCP_DEPTH
+#define EFCP_DEPTH 8
+#endif
+constexpr int kSlabThreads = EFCP_SLAB_THREADS;  // threads of a slab-kernel block (one block per SM)
+constexpr int kDepth = EFCP_DEPTH;               // groups of 32 entries a warp loads per pass
+
 // Scalar products of every window row with the newest row (x = dens(c_t)):
 //   partial[block][r] = sum over this block's slabs of <row_r, x> restricted to the slab
 // accumulated in fp64 (every fp32 x fp32 product is exact in fp64).
-__global__ void __launch_bounds__(1024, 1) k_sp_rows(
+__global__ void __launch_bounds__(kSlabThreads, 1) k_sp_rows(
     const int32_t* __restrict__ I, const float* __restrict__ V, const int32_t* __restrict__ offs,
     int64_t k, int m, int W, int n_slabs, int slot, double* __restrict__ partial) {
   extern __shared__ __align__(16) unsigned char smraw[];
@@ -76,20 +158,20 @@ __global__ void __launch_bounds__(1024, 1) k_sp_rows(
       const int32_t* Ir = I + int64_t(r) * k;
       const float* Vr = V + int64_t(r) * k;
       double acc = 0.0;
-      for (int j = b + lane; j < e; j += 128) {
-        const int j1 = j + 32, j2 = j + 64, j3 = j + 96;
-        const int i0 = __ldcs(Ir + j);
-        const float v0 = __ldcs(Vr + j);
-        const int i1 = j1 < e ? __ldcs(Ir + j1) : base;
-        const float v1 = j1 < e ? __ldcs(Vr + j1) : 0.f;
-        const int i2 = j2 < e ? __ldcs(Ir + j2) : base;
-        const float v2 = j2 < e ? __ldcs(Vr + j2) : 0.f;
-        const int i3 = j3 < e ? __ldcs(Ir + j3) : base;
-        const float v3 = j3 < e ? __ldcs(Vr + j3) : 0.f;
-        acc += double(v0) * double(xs[i0 - base]);
-        acc += double(v1) * double(xs[i1 - base]);
-        acc += double(v2) * double(xs[i2 - base]);
-        acc += double(v3) * double(xs[i3 - base]);
+      // kDepth groups of 32 entries per pass: all loads of a pass are issued before the
+      // first use
+      for (int j0 = b + lane; j0 < e; j0 += 32 * kDepth) {
+        int ii[kDepth];
+        float vv[kDepth];
+#pragma unroll
+        for (int q = 0; q < kDepth; ++q) {
+          const int j = j0 + 32 * q;
+          const bool on = j < e;
+          ii[q] = on ? __ldcs(Ir + j) : base;
+          vv[q] = on ? __ldcs(Vr + j) : 0.f;
+        }
+#pragma unroll
+        for (int q = 0; q < kDepth; ++q) acc += double(vv[q]) * double(xs[ii[q] - base]);
       }
       acc = warp_sum(acc);
       if (lane == 0) ds[r] += acc;
@@ -119,7 +201,7 @@ __global__ void __launch_bounds__(128) k_sp_finish(const double* __restrict__ pa
 // shared-memory accumulator (Eq. (2) in the form that has no x/lambda term, see
 // efcp_mxm.cuh).  Every element of u is written exactly once.
 template <bool VEC>
-__global__ void __launch_bounds__(1024, 1) k_lcg(
+__global__ void __launch_bounds__(kSlabThreads, 1) k_lcg(
     const int32_t* __restrict__ I, const float* __restrict__ V, const int32_t* __restrict__ offs,
     int64_t k, int m, int W, int n_slabs, const float* __restrict__ wf, float* __restrict__ u,
     int64_t d) {
@@ -145,20 +227,19 @@ __global__ void __launch_bounds__(1024, 1) k_lcg(
       if (b >= e || c == 0.f) continue;
       const int32_t* Ir = I + int64_t(r) * k;
       const float* Vr = V + int64_t(r) * k;
-      for (int j = b + lane; j < e; j += 128) {
-        const int j1 = j + 32, j2 = j + 64, j3 = j + 96;
-        const int i0 = __ldcs(Ir + j);
-        const float v0 = __ldcs(Vr + j);
-        const int i1 = j1 < e ? __ldcs(Ir + j1) : -1;
-        const float v1 = j1 < e ? __ldcs(Vr + j1) : 0.f;
-        const int i2 = j2 < e ? __ldcs(Ir + j2) : -1;
-        const float v2 = j2 < e ? __ldcs(Vr + j2) : 0.f;
-        const int i3 = j3 < e ? __ldcs(Ir + j3) : -1;
-        const float v3 = j3 < e ? __ldcs(Vr + j3) : 0.f;
-        atomicAdd(&acc[i0 - base], c * v0);
-        if (i1 >= 0) atomicAdd(&acc[i1 - base], c * v1);
-        if (i2 >= 0) atomicAdd(&acc[i2 - base], c * v2);
-        if (i3 >= 0) atomicAdd(&acc[i3 - base], c * v3);
+      for (int j0 = b + lane; j0 < e; j0 += 32 * kDepth) {
+        int ii[kDepth];
+        float vv[kDepth];
+#pragma unroll
+        for (int q = 0; q < kDepth; ++q) {
+          const int j = j0 + 32 * q;
+          const bool on = j < e;
+          ii[q] = on ? __ldcs(Ir + j) : -1;
+          vv[q] = on ? __ldcs(Vr + j) : 0.f;
+        }
+#pragma unroll
+        for (int q = 0; q < kDepth; ++q)
+          if (ii[q] >= 0) atomicAdd(&acc[ii[q] - base], c * vv[q]);
       }
     }
     __syncthreads();
