@@ -34,7 +34,14 @@ UNIT = "steps/s"
 # DRAM traffic per launch of the dominant kernels from the ncu captures summarised under
 # profiles/ (dram__bytes_read.sum + dram__bytes_write.sum), keyed by workload; None until
 # a capture of that workload exists.  Scaled from a smaller capture where noted there.
-NCU_TRAFFIC_BYTES = {}
+# Captured on c3_resnet18 (same kernels, window 0.96 GB); DRAM traffic is proportional to
+# the bytes streamed, so the C4 figures are the C3 traffic / C3 algorithmic bytes ratio
+# (k_sp_rows 1.009, k_lcg 0.981) times the C4 algorithmic bytes per launch.
+NCU_TRAFFIC_BYTES = {
+    "c3_resnet18": {"sp": 966_382_848, "lcg": 984_982_528},
+    "c4_bert_base": {"sp": int(1.0092 * 8 * 1024 * 1_094_822),
+                     "lcg": int(0.9807 * (8 * 1024 * 1_094_822 + 4 * 109_482_240))},
+}
 
 
 def load_peak():
