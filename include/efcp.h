@@ -36,6 +36,7 @@ typedef struct efcp_ctx efcp_ctx;
                              m x m update (window numerically singular for this lambda)  */
 #define EFCP_ETIMEOUT -5  /* a bounded device-side wait gave up                            */
 #define EFCP_EINTERNAL -6 /* an internal consistency check failed (selection count != k)  */
+#define EFCP_ETOOBIG  -7  /* size beyond the fixed capacity of an allocation-free entry point */
 
 /* flags for efcp_create_ex */
 #define EFCP_RHS_COMPRESSED  0u /* u_t = A(c_t): precondition the compressed accumulator
@@ -138,6 +139,33 @@ int32_t efcp_launches_per_step(efcp_ctx* ctx);
  */
 int efcp_profile_begin(efcp_ctx* ctx, int32_t max_steps);
 int efcp_profile_end(efcp_ctx* ctx, double* ms_out, int32_t* steps_out);
+
+/*
+ * efcp_topk_static - the exact Top-k selection of efcp_step (k largest magnitudes, ties to
+ * the lower index, pairs in ascending index order) as a stand-alone call that allocates
+ * nothing.  The paper has no counterpart of this call; it exists for callers that must
+ * not allocate device memory: code running while a memory pool or another framework owns
+ * all free device memory, code inside a region where cudaMalloc's implicit device-wide
+ * synchronisation is not acceptable, and start-up paths that must not fail with
+ * out-of-memory.  efcp_create, by contrast, calls cudaMalloc.
+ *
+ * The scratch memory of the selection (histograms, chunk counters and the candidate list,
+ * 8 bytes per element of `a`) lives in one fixed array inside the library image,
+ * EFCP_TOPK_STATIC_MAX_D elements long: about 8.1 MiB that every GPU which loads the
+ * library holds until the process exits.
+ *   a      device, d floats, read only.
+ *   idx    device, k int32: receives the kept indices, ascending.
+ *   val    device, k floats: receives a[idx[j]].
+ *   stream a cudaStream_t (NULL = default stream); the work is enqueued, not awaited.
+ * Returns EFCP_EINVAL for null pointers or k outside 1..d, EFCP_ETOOBIG when
+ * d > EFCP_TOPK_STATIC_MAX_D (nothing is enqueued), EFCP_ECUDA when a runtime call fails.
+ * The first call on each device looks up the array's device address and the SM count;
+ * make that first call outside any stream capture.  All calls on a device share the one
+ * array: the call clears the parts that must start at zero, and two calls whose GPU work
+ * overlaps (different streams, different host threads) race on it - serialise them.
+ */
+#define EFCP_TOPK_STATIC_MAX_D (1 << 20)
+int efcp_topk_static(const float* a, int64_t d, int64_t k, int32_t* idx, float* val, void* stream);
 
 /* Static description of an EFCP_* code. */
 const char* efcp_strerror(int code);

@@ -13,7 +13,8 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "csrc", "libefcp.so")
 
-OK, EINVAL, ENOMEM, ECUDA, ENUMERIC, ETIMEOUT, EINTERNAL = 0, -1, -2, -3, -4, -5, -6
+OK, EINVAL, ENOMEM, ECUDA, ENUMERIC, ETIMEOUT, EINTERNAL, ETOOBIG = 0, -1, -2, -3, -4, -5, -6, -7
+TOPK_STATIC_MAX_D = 1 << 20
 RHS_COMPRESSED, RHS_ACCUMULATOR = 0, 1
 
 if not os.path.exists(LIB_PATH):
@@ -42,6 +43,7 @@ EXPORTS = {
     "efcp_launches_per_step": ([_vp], _i32),
     "efcp_profile_begin": ([_vp, _i32], C.c_int),
     "efcp_profile_end": ([_vp, _vp, _vp], C.c_int),
+    "efcp_topk_static": ([_vp, _i64, _i64, _vp, _vp, _vp], C.c_int),
     "efcp_strerror": ([C.c_int], C.c_char_p),
 }
 for _name, (_args, _res) in EXPORTS.items():
@@ -69,6 +71,22 @@ def paper_state_bytes(d: int, m: int, k: int, value_bytes: int = 4) -> int:
     """Footprint of Sparse M-FAC as the paper's appendix "Memory savings" counts it:
     indices 4mk, values value_bytes*mk, error feedback 4d, SP result 4m, LCG result 4d."""
     return 4 * m * k + value_bytes * m * k + 4 * d + 4 * m + 4 * d
+
+
+def topk_static(a: torch.Tensor, k: int, idx: torch.Tensor, val: torch.Tensor, stream=None):
+    """efcp_topk_static: exact Top-k of the device vector `a` into the device tensors `idx`
+    (int32, k) and `val` (fp32, k), ascending indices, using no allocation at all (the
+    scratch memory is a fixed array inside the library; at most TOPK_STATIC_MAX_D elements).
+    For callers that must not allocate device memory; asynchronous on `stream`."""
+    assert a.is_cuda and idx.is_cuda and val.is_cuda
+    assert a.dtype == torch.float32 and val.dtype == torch.float32 and idx.dtype == torch.int32
+    assert a.is_contiguous() and idx.is_contiguous() and val.is_contiguous()
+    assert idx.numel() >= k and val.numel() >= k
+    s = torch.cuda.current_stream() if stream is None else stream
+    rc = _lib.efcp_topk_static(a.data_ptr(), a.numel(), int(k), idx.data_ptr(), val.data_ptr(),
+                               s.cuda_stream)
+    if rc != OK:
+        raise EfcpError(rc, "efcp_topk_static")
 
 
 def _np_ptr(a: np.ndarray):

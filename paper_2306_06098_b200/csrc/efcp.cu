@@ -10,6 +10,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <utility>
 #include <vector>
@@ -83,6 +84,7 @@ int pick_slab_width(int64_t d, int m, int num_sms) {
 }
 
 inline int64_t align256(int64_t b) { return (b + 255) & ~int64_t(255); }
+constexpr int64_t align256c(int64_t b) { return (b + 255) & ~int64_t(255); }
 
 Sizes compute_sizes(int64_t d, int32_t m, int64_t k, int num_sms) {
   Sizes z;
@@ -190,6 +192,7 @@ const char* efcp_strerror(int code) {
     case EFCP_ENUMERIC: return "non-finite input or non-positive pivot in the m x m update";
     case EFCP_ETIMEOUT: return "bounded device-side wait expired";
     case EFCP_EINTERNAL: return "internal consistency check failed";
+    case EFCP_ETOOBIG: return "size exceeds the fixed scratch capacity of the allocation-free entry point";
     default: return "unknown error code";
   }
 }
@@ -505,3 +508,160 @@ int efcp_profile_end(efcp_ctx* ctx, double* ms_out, int32_t* steps_out) {
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------
+// efcp_topk_static: the Top-k selection with its scratch memory in a fixed array of the
+// library image, for callers that cannot allocate (see include/efcp.h).
+namespace {
+
+constexpr int64_t kStaticMaxD = EFCP_TOPK_STATIC_MAX_D;
+constexpr int64_t kStaticMaxChunks = (kStaticMaxD + kChunk - 1) / kChunk;
+// layout of the array (every part 256-byte aligned)
+constexpr int64_t kOffHist = 0;                                            // 3 histograms
+constexpr int64_t kOffScalars = kOffHist + align256c((kBins1 + kBins2 + kBins3) * 4);
+constexpr int64_t kOffChunk = kOffScalars + align256c(int64_t(sizeof(Scalars)));
+constexpr int64_t kOffSelGt = kOffChunk + align256c((kStaticMaxChunks + 1) * 4);
+constexpr int64_t kOffSelEq = kOffSelGt + align256c((kStaticMaxChunks + 1) * 4);
+constexpr int64_t kOffCandIdx = kOffSelEq + align256c((kStaticMaxChunks + 1) * 4);
+constexpr int64_t kOffCandVal = kOffCandIdx + align256c(kStaticMaxD * 4);
+constexpr int64_t kStaticBytes = kOffCandVal + align256c(kStaticMaxD * 4);
+
+// In host code this name is only a handle for cudaGetSymbolAddress, never an address.
+static __device__ __align__(256) unsigned char g_topk_scratch[kStaticBytes];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mu;
+unsigned char* g_static_ptr[kMaxDevices] = {};  // device address of the array, per device
+int g_static_sms[kMaxDevices] = {};
+
+// Digit-1 histogram of the magnitude keys of a (the part of k_ef_hist1 that does not
+// touch an error buffer).
+__global__ void __launch_bounds__(512) k_hist1_only(const float* __restrict__ a, int64_t d,
+                                                    uint32_t* __restrict__ hist1) {
+  __shared__ uint32_t h[kBins1];
+  for (int i = threadIdx.x; i < kBins1; i += blockDim.x) h[i] = 0u;
+  __syncthreads();
+  for (int64_t j = int64_t(blockIdx.x) * blockDim.x + threadIdx.x; j < d;
+       j += int64_t(gridDim.x) * blockDim.x)
+    atomicAdd(&h[mag_key(a[j]) >> kShift1], 1u);
+  __syncthreads();
+  for (int i = threadIdx.x; i < kBins1; i += blockDim.x) {
+    const uint32_t c = h[i];
+    if (c) atomicAdd(&hist1[i], c);
+  }
+}
+
+// Final ordered compaction of k_write_sel without the error-buffer update: the kept
+// (index, value) pairs in ascending index order.
+__global__ void __launch_bounds__(kChunkThreads) k_write_sel_only(
+    const int32_t* __restrict__ cand_idx, const float* __restrict__ cand_val, const Scalars* sc,
+    const int32_t* __restrict__ off_gt, const int32_t* __restrict__ pre_eq,
+    int32_t* __restrict__ out_idx, float* __restrict__ out_val, int64_t k_total) {
+  __shared__ int sm[33];
+  const int n = sc->n_cand;
+  const uint32_t T = sc->T;
+  const int n_eq = int(sc->n_eq);
+  const int n_cc = (n + kChunk - 1) / kChunk;
+  for (int c = blockIdx.x; c < n_cc; c += gridDim.x) {
+    const int64_t base = int64_t(c) * kChunk + threadIdx.x * kPerThread;
+    float v[kPerThread];
+    bool ok[kPerThread];
+    load_chunk8(cand_val, base, n, v, ok);
+    bool is_eq[kPerThread];
+    int my_eq = 0;
+#pragma unroll
+    for (int q = 0; q < kPerThread; ++q) {
+      const uint32_t key = mag_key(v[q]);
+      is_eq[q] = ok[q] && key == T;
+      ok[q] = ok[q] && key > T;
+      my_eq += is_eq[q] ? 1 : 0;
+    }
+    int tot;
+    const int eq_before_chunk = pre_eq[c];
+    int eq_rank = eq_before_chunk + block_excl_scan<int>(my_eq, &tot, sm);
+    int my_sel = 0;
+#pragma unroll
+    for (int q = 0; q < kPerThread; ++q) {
+      if (is_eq[q]) {
+        ok[q] = eq_rank < n_eq;
+        ++eq_rank;
+      }
+      my_sel += ok[q] ? 1 : 0;
+    }
+    int64_t pos = int64_t(off_gt[c]) + min(eq_before_chunk, n_eq) +
+                  block_excl_scan<int>(my_sel, &tot, sm);
+#pragma unroll
+    for (int q = 0; q < kPerThread; ++q) {
+      if (ok[q] && pos < k_total) {
+        out_idx[pos] = cand_idx[base + q];
+        out_val[pos] = v[q];
+        ++pos;
+      }
+    }
+  }
+}
+
+}  // namespace
+
+extern "C" int efcp_topk_static(const float* a, int64_t d, int64_t k, int32_t* idx, float* val,
+                                void* stream_) {
+  if (!a || !idx || !val || d < 1 || k < 1 || k > d) return EFCP_EINVAL;
+  if (d > kStaticMaxD) return EFCP_ETOOBIG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream_);
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+    (void)cudaGetLastError();
+    return EFCP_ECUDA;
+  }
+  unsigned char* base = nullptr;
+  int sms = 0;
+  {
+    // set-up, once per device, with that device current: the device address of the array
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    if (!g_static_ptr[dev]) {
+      unsigned char* p = nullptr;
+      int n = 0;
+      if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_topk_scratch) != cudaSuccess ||
+          cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+          !p || n < 1) {
+        (void)cudaGetLastError();
+        return EFCP_ECUDA;
+      }
+      g_static_ptr[dev] = p;
+      g_static_sms[dev] = n;
+    }
+    base = g_static_ptr[dev];
+    sms = g_static_sms[dev];
+  }
+  uint32_t* hist1 = reinterpret_cast<uint32_t*>(base + kOffHist);
+  uint32_t* hist2 = hist1 + kBins1;
+  uint32_t* hist3 = hist2 + kBins2;
+  Scalars* sc = reinterpret_cast<Scalars*>(base + kOffScalars);
+  int32_t* chunk_off = reinterpret_cast<int32_t*>(base + kOffChunk);
+  int32_t* sel_gt = reinterpret_cast<int32_t*>(base + kOffSelGt);
+  int32_t* sel_eq = reinterpret_cast<int32_t*>(base + kOffSelEq);
+  int32_t* cand_idx = reinterpret_cast<int32_t*>(base + kOffCandIdx);
+  float* cand_val = reinterpret_cast<float*>(base + kOffCandVal);
+  const int n_chunks = int((d + kChunk - 1) / kChunk);
+  // the array keeps the last call's contents: histograms and scalars must start at zero
+  if (cudaMemsetAsync(base + kOffHist, 0, size_t(kOffChunk - kOffHist), st) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return EFCP_ECUDA;
+  }
+  const int cand_grid = sms * 4;
+  k_hist1_only<<<sms * 2, 512, 0, st>>>(a, d, hist1);
+  k_pick<kBins1, 1><<<1, 1024, 0, st>>>(hist1, sc, uint32_t(k));
+  k_count_chunks<<<n_chunks, kChunkThreads, 0, st>>>(a, d, sc, chunk_off);
+  k_scan_counts<<<1, 1024, 0, st>>>(chunk_off, n_chunks, &sc->n_cand);
+  k_compact_cand<<<n_chunks, kChunkThreads, 0, st>>>(a, d, sc, chunk_off, cand_idx, cand_val,
+                                                     hist2);
+  k_pick<kBins2, 2><<<1, 1024, 0, st>>>(hist2, sc, uint32_t(k));
+  k_hist3<<<cand_grid, 256, 0, st>>>(cand_val, sc, hist3);
+  k_pick<kBins3, 3><<<1, 1024, 0, st>>>(hist3, sc, uint32_t(k));
+  k_count_sel<<<cand_grid, kChunkThreads, 0, st>>>(cand_val, sc, sel_gt, sel_eq);
+  k_scan_sel<<<1, 1024, 0, st>>>(sel_gt, sel_eq, sc, uint32_t(k));
+  k_write_sel_only<<<cand_grid, kChunkThreads, 0, st>>>(cand_idx, cand_val, sc, sel_gt, sel_eq,
+                                                        idx, val, k);
+  if (cudaGetLastError() != cudaSuccess) return EFCP_ECUDA;
+  return EFCP_OK;
+}
