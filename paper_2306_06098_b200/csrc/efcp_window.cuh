@@ -157,10 +157,28 @@ __global__ void __launch_bounds__(kSlabThreads, 1) k_sp_rows(
       if (b >= e) continue;
       const int32_t* Ir = I + int64_t(r) * k;
       const float* Vr = V + int64_t(r) * k;
-      double acc = 0.0;
+      double acc = 0.0, acc2 = 0.0;
       // kDepth groups of 32 entries per pass: all loads of a pass are issued before the
-      // first use
-      for (int j0 = b + lane; j0 < e; j0 += 32 * kDepth) {
+      // first use.  Full passes need no bounds checks and address every load by a
+      // constant offset from one pointer pair.
+      int j0 = b + lane;
+      for (; j0 + 32 * (kDepth - 1) < e - 31 + lane; j0 += 32 * kDepth) {
+        const int32_t* pi = Ir + j0;
+        const float* pv = Vr + j0;
+        int ii[kDepth];
+        float vv[kDepth];
+#pragma unroll
+        for (int q = 0; q < kDepth; ++q) {
+          ii[q] = __ldcs(pi + 32 * q);
+          vv[q] = __ldcs(pv + 32 * q);
+        }
+#pragma unroll
+        for (int q = 0; q < kDepth; q += 2) {
+          acc += double(vv[q]) * double(xs[ii[q] - base]);
+          acc2 += double(vv[q + 1]) * double(xs[ii[q + 1] - base]);
+        }
+      }
+      if (j0 - lane < e) {  // the last, partial pass (warp-uniform condition)
         int ii[kDepth];
         float vv[kDepth];
 #pragma unroll
@@ -171,8 +189,12 @@ __global__ void __launch_bounds__(kSlabThreads, 1) k_sp_rows(
           vv[q] = on ? __ldcs(Vr + j) : 0.f;
         }
 #pragma unroll
-        for (int q = 0; q < kDepth; ++q) acc += double(vv[q]) * double(xs[ii[q] - base]);
+        for (int q = 0; q < kDepth; q += 2) {
+          acc += double(vv[q]) * double(xs[ii[q] - base]);
+          acc2 += double(vv[q + 1]) * double(xs[ii[q + 1] - base]);
+        }
       }
+      acc += acc2;
       acc = warp_sum(acc);
       if (lane == 0) ds[r] += acc;
     }
@@ -227,7 +249,21 @@ __global__ void __launch_bounds__(kSlabThreads, 1) k_lcg(
       if (b >= e || c == 0.f) continue;
       const int32_t* Ir = I + int64_t(r) * k;
       const float* Vr = V + int64_t(r) * k;
-      for (int j0 = b + lane; j0 < e; j0 += 32 * kDepth) {
+      int j0 = b + lane;
+      for (; j0 + 32 * (kDepth - 1) < e - 31 + lane; j0 += 32 * kDepth) {  // full passes
+        const int32_t* pi = Ir + j0;
+        const float* pv = Vr + j0;
+        int ii[kDepth];
+        float vv[kDepth];
+#pragma unroll
+        for (int q = 0; q < kDepth; ++q) {
+          ii[q] = __ldcs(pi + 32 * q);
+          vv[q] = __ldcs(pv + 32 * q);
+        }
+#pragma unroll
+        for (int q = 0; q < kDepth; ++q) atomicAdd(&acc[ii[q] - base], c * vv[q]);
+      }
+      if (j0 - lane < e) {  // the last, partial pass
         int ii[kDepth];
         float vv[kDepth];
 #pragma unroll
