@@ -49,9 +49,11 @@ struct efcp_ctx {
   int32_t* sel_gt = nullptr;
   int32_t* sel_eq = nullptr;
   Scalars* sc = nullptr;
-  double* partial = nullptr;
+  double* slab_part = nullptr;  // SP: one partial sum per (slab, row)
+  double* partial = nullptr;    // SP: kSpParts x m sums of slab partials
   double* vecs = nullptr;  // 8 m-vectors: delta, aprime, y, bold, z, w, res, dw
   float* wf = nullptr;
+  int* slab_ctr = nullptr;   // work counters of the slab kernels (SP, LCG)
   float* stage_g = nullptr;  // efcp_step_host staging
   float* stage_u = nullptr;
   int last_cuda = 0;
@@ -65,19 +67,21 @@ struct efcp_ctx {
 
 namespace {
 
+constexpr int kSpParts = 32;  // second-level partial sums of the scalar products
+
 struct Sizes {
   int W, n_slabs, n_chunks, grid_slab;
   int64_t total;
 };
 
 int pick_slab_width(int64_t d, int m, int num_sms) {
-  int W = 32768;
+  int W = (32768 / kSlabBlocksPerSM) & ~31;
   if (const char* env = getenv("EFCP_SLAB_W")) {
     const int v = atoi(env);
     if (v >= 256 && v <= 49152 && (v & 31) == 0) return v;
   }
   // shared memory: W*4 + 16*m must stay under the 227 KB per-block limit
-  while (size_t(W) * 4 + size_t(m) * 16 > 200 * 1024 && W > 1024) W >>= 1;
+  while ((size_t(W) * 4 + size_t(m) * 16) * kSlabBlocksPerSM > 200 * 1024 && W > 1024) W >>= 1;
   // enough slabs to give every SM several
   while (W > 1024 && (d + W - 1) / W < int64_t(4) * num_sms) W >>= 1;
   return W;
@@ -91,7 +95,7 @@ Sizes compute_sizes(int64_t d, int32_t m, int64_t k, int num_sms) {
   z.W = pick_slab_width(d, m, num_sms);
   z.n_slabs = int((d + z.W - 1) / z.W);
   z.n_chunks = int((d + kChunk - 1) / kChunk);
-  z.grid_slab = z.n_slabs < num_sms ? z.n_slabs : num_sms;
+  z.grid_slab = z.n_slabs < num_sms * kSlabBlocksPerSM ? z.n_slabs : num_sms * kSlabBlocksPerSM;
   int64_t b = 0;
   b += align256(d * 4);                                   // e
   b += 2 * align256(int64_t(m) * k * 4);                  // I, V
@@ -102,7 +106,8 @@ Sizes compute_sizes(int64_t d, int32_t m, int64_t k, int num_sms) {
   b += 2 * align256(d * 4);                               // cand_idx, cand_val
   b += 2 * align256(k * 4);                               // sel_idx, sel_val
   b += align256(sizeof(Scalars));
-  b += align256(int64_t(z.grid_slab) * m * 8);            // partial
+  b += align256(int64_t(z.n_slabs) * m * 8);              // slab_part
+  b += align256(int64_t(kSpParts) * m * 8);               // partial
   b += align256(int64_t(8) * m * 8);                      // vecs
   b += align256(int64_t(m) * 4);                          // wf
   z.total = b;
@@ -247,9 +252,12 @@ int efcp_create_ex(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float lambda
   if ((rc = dev_alloc(ctx, &ctx->sel_idx, k * 4))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->sel_val, k * 4))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->sc, sizeof(Scalars)))) return fail(rc);
-  if ((rc = dev_alloc(ctx, &ctx->partial, int64_t(z.grid_slab) * m * 8))) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->slab_part, int64_t(z.n_slabs) * m * 8))) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->partial, int64_t(kSpParts) * m * 8))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->vecs, int64_t(8) * m * 8))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->wf, int64_t(m) * 4))) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->slab_ctr, 256))) return fail(rc);
+
 
   bool ok = true;
   ok &= cudaMemset(ctx->e, 0, size_t(d) * 4) == cudaSuccess;
@@ -345,16 +353,21 @@ int efcp_step(efcp_ctx* ctx, const float* grad, float* update, void* stream_) {
                                                    ctx->sel_val, ctx->e, k);
   EFCP_LAUNCHED();
   k_layout_row<<<(ctx->n_slabs + kLayoutWarps) / kLayoutWarps, kLayoutWarps * 32, 0, st>>>(
-      ctx->sel_idx, ctx->sel_val, k, ctx->W, ctx->n_slabs, m, slot, ctx->offs, row_idx, row_val);
+      ctx->sel_idx, ctx->sel_val, k, ctx->W, ctx->n_slabs, m, slot, ctx->offs, row_idx, row_val,
+      ctx->slab_ctr);
   EFCP_LAUNCHED();
   // scalar products with the new row, Gram row/column
   const size_t smem = slab_smem_bytes(ctx->W, m);
   prof_mark(ctx, 1, st);
   k_sp_rows<<<ctx->grid_slab, kSlabThreads, smem, st>>>(ctx->I, ctx->V, ctx->offs, k, m, ctx->W,
-                                                ctx->n_slabs, slot, ctx->partial);
+                                                ctx->n_slabs, slot, ctx->slab_part, ctx->slab_ctr);
   EFCP_LAUNCHED();
   prof_mark(ctx, 2, st);
-  k_sp_finish<<<(m + 127) / 128, 128, 0, st>>>(ctx->partial, ctx->grid_slab, m, slot, delta,
+  const int sp_parts = ctx->n_slabs < kSpParts ? ctx->n_slabs : kSpParts;
+  k_sp_reduce<<<dim3((m + 127) / 128, sp_parts), 128, 0, st>>>(ctx->slab_part, ctx->n_slabs, m,
+                                                               ctx->partial);
+  EFCP_LAUNCHED();
+  k_sp_finish<<<(m + 127) / 128, 128, 0, st>>>(ctx->partial, sp_parts, m, slot, delta,
                                                ctx->S, aprime);
   EFCP_LAUNCHED();
   // m x m: remove-and-border update of the inverse, weights, one refinement step
@@ -376,10 +389,10 @@ int efcp_step(efcp_ctx* ctx, const float* grad, float* update, void* stream_) {
   prof_mark(ctx, 3, st);
   if ((reinterpret_cast<uintptr_t>(update) & 15) == 0)
     k_lcg<true><<<ctx->grid_slab, kSlabThreads, smem, st>>>(ctx->I, ctx->V, ctx->offs, k, m, ctx->W,
-                                                    ctx->n_slabs, ctx->wf, update, d);
+                                                    ctx->n_slabs, ctx->wf, update, d, ctx->slab_ctr + 1);
   else
     k_lcg<false><<<ctx->grid_slab, kSlabThreads, smem, st>>>(ctx->I, ctx->V, ctx->offs, k, m, ctx->W,
-                                                     ctx->n_slabs, ctx->wf, update, d);
+                                                     ctx->n_slabs, ctx->wf, update, d, ctx->slab_ctr + 1);
   EFCP_LAUNCHED();
   prof_mark(ctx, 4, st);
   if (ctx->prof_on && ctx->prof_n < ctx->prof_cap) ++ctx->prof_n;

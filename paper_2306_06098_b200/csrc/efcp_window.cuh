@@ -39,12 +39,13 @@ constexpr int kLayoutWarps = 8;     // warps (= slabs) per block of k_layout_row
 __global__ void __launch_bounds__(kLayoutWarps * 32) k_layout_row(
     const int32_t* __restrict__ src_idx, const float* __restrict__ src_val, int64_t k, int W,
     int n_slabs, int m, int slot, int32_t* __restrict__ offs, int32_t* __restrict__ dst_idx,
-    float* __restrict__ dst_val) {
+    float* __restrict__ dst_val, int* __restrict__ slab_ctr) {
   __shared__ int32_t s_idx[kLayoutWarps][kLayoutChunk];
   __shared__ float s_val[kLayoutWarps][kLayoutChunk];
   __shared__ uint16_t s_q[kLayoutWarps][kLayoutChunk];
   __shared__ int s_cnt[kLayoutWarps][32];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (blockIdx.x == 0 && threadIdx.x < 2) slab_ctr[threadIdx.x] = 0;  // SP and LCG work counters
   const int s = blockIdx.x * kLayoutWarps + warp;
   if (s > n_slabs) return;
   // lane 0 finds the segment start, lane 1 its end
@@ -117,28 +118,53 @@ __host__ __device__ inline size_t slab_smem_bytes(int W, int m) {
 #ifndef EFCP_SLAB_THREADS
 #define EFCP_SLAB_THREADS 1024
 #endif
+#ifndef EFCP_SLAB_BLOCKS
+#define EFCP_SLAB_BLOCKS 1
+#endif
+constexpr int kSlabBlocksPerSM = EFCP_SLAB_BLOCKS;  // resident blocks of a slab kernel per SM
 #ifndef EFCP_DEPTH
 #define EFCP_DEPTH 8
 #endif
 constexpr int kSlabThreads = EFCP_SLAB_THREADS;  // threads of a slab-kernel block (one block per SM)
 constexpr int kDepth = EFCP_DEPTH;               // groups of 32 entries a warp loads per pass
 
+// Asks L2 for the lines of entries [b, e) of a row's index and value streams (at most 16
+// lines of each; longer segments are covered at their start only).  Issued one row ahead
+// of use, so that the loads of the next row find their data in L2 instead of waiting for
+// HBM.
+__device__ __forceinline__ void prefetch_segment(const int32_t* Ir, const float* Vr, int b, int e,
+                                                 int lane) {
+  const int half = lane & 15;
+  const char* p = (lane < 16) ? reinterpret_cast<const char*>(Ir + b)
+                              : reinterpret_cast<const char*>(Vr + b);
+  const int bytes = (e - b) * 4;
+  if (half * 128 < bytes) asm volatile("prefetch.global.L2 [%0];" ::"l"(p + half * 128));
+}
+
+// Slab scheduling of the two slab kernels.  Slabs differ in weight (the kept entries
+// cluster where the gradient is large), so blocks do not take a fixed share: block b starts
+// with slab b and then draws the next unprocessed slab from a counter in global memory
+// (cleared by k_layout_row earlier in the step).  The draw for the next slab is issued at
+// the start of the current one, so its latency is hidden.  Results do not depend on which
+// block processes which slab: LCG slabs are disjoint outputs, and SP writes one partial
+// sum per (slab, row) that is reduced afterwards in slab order.
+
 // Scalar products of every window row with the newest row (x = dens(c_t)):
-//   partial[block][r] = sum over this block's slabs of <row_r, x> restricted to the slab
+//   slab_part[s][r] = <row_r, x> restricted to slab s
 // accumulated in fp64 (every fp32 x fp32 product is exact in fp64).
-__global__ void __launch_bounds__(kSlabThreads, 1) k_sp_rows(
+__global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_sp_rows(
     const int32_t* __restrict__ I, const float* __restrict__ V, const int32_t* __restrict__ offs,
-    int64_t k, int m, int W, int n_slabs, int slot, double* __restrict__ partial) {
+    int64_t k, int m, int W, int n_slabs, int slot, double* __restrict__ slab_part, int* ctr) {
   extern __shared__ __align__(16) unsigned char smraw[];
   float* xs = reinterpret_cast<float*>(smraw);
-  double* ds = reinterpret_cast<double*>(smraw + size_t(W) * 4);
   int32_t* seg = reinterpret_cast<int32_t*>(smraw + size_t(W) * 4 + size_t(m) * 8);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
-  for (int r = tid; r < m; r += blockDim.x) ds[r] = 0.0;
   const int32_t* Inew = I + int64_t(slot) * k;
   const float* Vnew = V + int64_t(slot) * k;
-  for (int s = blockIdx.x; s < n_slabs; s += gridDim.x) {
+  __shared__ int s_next;
+  for (int s = blockIdx.x; s < n_slabs;) {
     __syncthreads();
+    if (tid == 0) s_next = int(gridDim.x) + atomicAdd(ctr, 1);
     float4* xs4 = reinterpret_cast<float4*>(xs);
     for (int i = tid; i < (W >> 2); i += blockDim.x) xs4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int r = tid; r < m; r += blockDim.x) {
@@ -152,11 +178,19 @@ __global__ void __launch_bounds__(kSlabThreads, 1) k_sp_rows(
       for (int j = b + tid; j < e; j += blockDim.x) xs[Inew[j] - base] = Vnew[j];
     }
     __syncthreads();
+    double* out = slab_part + int64_t(s) * m;
     for (int r = warp; r < m; r += nwarps) {
       const int b = seg[r], e = seg[m + r];
-      if (b >= e) continue;
+      if (b >= e) {
+        if (lane == 0) out[r] = 0.0;
+        continue;
+      }
       const int32_t* Ir = I + int64_t(r) * k;
       const float* Vr = V + int64_t(r) * k;
+      if (r + nwarps < m) {
+        const int rn = r + nwarps;
+        prefetch_segment(I + int64_t(rn) * k, V + int64_t(rn) * k, seg[rn], seg[m + rn], lane);
+      }
       double acc = 0.0, acc2 = 0.0;
       // kDepth groups of 32 entries per pass: all loads of a pass are issued before the
       // first use.  Full passes need no bounds checks and address every load by a
@@ -196,11 +230,29 @@ __global__ void __launch_bounds__(kSlabThreads, 1) k_sp_rows(
       }
       acc += acc2;
       acc = warp_sum(acc);
-      if (lane == 0) ds[r] += acc;
+      if (lane == 0) out[r] = acc;
     }
+    s = s_next;
   }
-  __syncthreads();
-  for (int r = tid; r < m; r += blockDim.x) partial[int64_t(blockIdx.x) * m + r] = ds[r];
+}
+
+// part2[y][r] = sum of slab_part[s][r] over s = y, y + gridDim.y, ... in increasing s.
+__global__ void __launch_bounds__(128) k_sp_reduce(const double* __restrict__ slab_part,
+                                                    int n_slabs, int m,
+                                                    double* __restrict__ part2) {
+  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r >= m) return;
+  const int step = gridDim.y;
+  double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
+  int s = blockIdx.y;
+  for (; s + 3 * step < n_slabs; s += 4 * step) {
+    a0 += slab_part[int64_t(s) * m + r];
+    a1 += slab_part[int64_t(s + step) * m + r];
+    a2 += slab_part[int64_t(s + 2 * step) * m + r];
+    a3 += slab_part[int64_t(s + 3 * step) * m + r];
+  }
+  for (; s < n_slabs; s += step) a0 += slab_part[int64_t(s) * m + r];
+  part2[int64_t(blockIdx.y) * m + r] = (a0 + a1) + (a2 + a3);
 }
 
 // delta[r] = sum of the per-block partials in block order; S row/column `slot` := delta
@@ -223,20 +275,22 @@ __global__ void __launch_bounds__(128) k_sp_finish(const double* __restrict__ pa
 // shared-memory accumulator (Eq. (2) in the form that has no x/lambda term, see
 // efcp_mxm.cuh).  Every element of u is written exactly once.
 template <bool VEC>
-__global__ void __launch_bounds__(kSlabThreads, 1) k_lcg(
+__global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_lcg(
     const int32_t* __restrict__ I, const float* __restrict__ V, const int32_t* __restrict__ offs,
     int64_t k, int m, int W, int n_slabs, const float* __restrict__ wf, float* __restrict__ u,
-    int64_t d) {
+    int64_t d, int* ctr) {
   extern __shared__ __align__(16) unsigned char smraw[];
   float* acc = reinterpret_cast<float*>(smraw);
   float* wc = reinterpret_cast<float*>(smraw + size_t(W) * 4);
   int32_t* seg = reinterpret_cast<int32_t*>(smraw + size_t(W) * 4 + size_t(m) * 8);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
   for (int r = tid; r < m; r += blockDim.x) wc[r] = wf[r];
-  for (int s = blockIdx.x; s < n_slabs; s += gridDim.x) {
+  float4* acc4 = reinterpret_cast<float4*>(acc);
+  for (int i = tid; i < (W >> 2); i += blockDim.x) acc4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+  __shared__ int s_next;
+  for (int s = blockIdx.x; s < n_slabs;) {
     __syncthreads();
-    float4* acc4 = reinterpret_cast<float4*>(acc);
-    for (int i = tid; i < (W >> 2); i += blockDim.x) acc4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (tid == 0) s_next = int(gridDim.x) + atomicAdd(ctr, 1);
     for (int r = tid; r < m; r += blockDim.x) {
       seg[r] = offs[int64_t(s) * m + r];
       seg[m + r] = offs[int64_t(s + 1) * m + r];
@@ -249,6 +303,10 @@ __global__ void __launch_bounds__(kSlabThreads, 1) k_lcg(
       if (b >= e || c == 0.f) continue;
       const int32_t* Ir = I + int64_t(r) * k;
       const float* Vr = V + int64_t(r) * k;
+      if (r + nwarps < m) {
+        const int rn = r + nwarps;
+        prefetch_segment(I + int64_t(rn) * k, V + int64_t(rn) * k, seg[rn], seg[m + rn], lane);
+      }
       int j0 = b + lane;
       for (; j0 + 32 * (kDepth - 1) < e - 31 + lane; j0 += 32 * kDepth) {  // full passes
         const int32_t* pi = Ir + j0;
@@ -261,7 +319,9 @@ __global__ void __launch_bounds__(kSlabThreads, 1) k_lcg(
           vv[q] = __ldcs(pv + 32 * q);
         }
 #pragma unroll
-        for (int q = 0; q < kDepth; ++q) atomicAdd(&acc[ii[q] - base], c * vv[q]);
+        for (int q = 0; q < kDepth; ++q) ii[q] -= base;
+#pragma unroll
+        for (int q = 0; q < kDepth; ++q) atomicAdd(&acc[ii[q]], c * vv[q]);
       }
       if (j0 - lane < e) {  // the last, partial pass
         int ii[kDepth];
@@ -270,25 +330,36 @@ __global__ void __launch_bounds__(kSlabThreads, 1) k_lcg(
         for (int q = 0; q < kDepth; ++q) {
           const int j = j0 + 32 * q;
           const bool on = j < e;
-          ii[q] = on ? __ldcs(Ir + j) : -1;
+          ii[q] = on ? __ldcs(Ir + j) - base : -1;
           vv[q] = on ? __ldcs(Vr + j) : 0.f;
         }
 #pragma unroll
         for (int q = 0; q < kDepth; ++q)
-          if (ii[q] >= 0) atomicAdd(&acc[ii[q] - base], c * vv[q]);
+          if (ii[q] >= 0) atomicAdd(&acc[ii[q]], c * vv[q]);
       }
     }
     __syncthreads();
+    // write the slab out and clear it for the next one
     const int64_t gbase = int64_t(s) * W;
     const int n = int(min(int64_t(W), d - gbase));
     if (VEC) {
       float4* u4 = reinterpret_cast<float4*>(u + gbase);
       const int nv = n >> 2;
-      for (int i = tid; i < nv; i += blockDim.x) __stcs(u4 + i, acc4[i]);
-      for (int i = (nv << 2) + tid; i < n; i += blockDim.x) u[gbase + i] = acc[i];
+      for (int i = tid; i < nv; i += blockDim.x) {
+        __stcs(u4 + i, acc4[i]);
+        acc4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+      for (int i = (nv << 2) + tid; i < n; i += blockDim.x) {
+        u[gbase + i] = acc[i];
+        acc[i] = 0.f;
+      }
     } else {
-      for (int i = tid; i < n; i += blockDim.x) u[gbase + i] = acc[i];
+      for (int i = tid; i < n; i += blockDim.x) {
+        u[gbase + i] = acc[i];
+        acc[i] = 0.f;
+      }
     }
+    s = s_next;
   }
 }
 
