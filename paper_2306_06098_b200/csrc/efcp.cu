@@ -328,12 +328,15 @@ int efcp_step(efcp_ctx* ctx, const float* grad, float* update, void* stream_) {
   k_pick<kBins1, 1><<<1, 1024, 0, st>>>(hist1, ctx->sc, uint32_t(k));
   EFCP_LAUNCHED();
   // candidates: everything at or above the threshold bin, in index order
-  k_count_chunks<<<ctx->n_chunks, kChunkThreads, 0, st>>>(ctx->e, d, ctx->sc, ctx->chunk_off);
+  const int chunk_grid = ctx->n_chunks < ctx->num_sms * 8 ? ctx->n_chunks : ctx->num_sms * 8;
+  k_count_chunks<<<chunk_grid, kChunkThreads, 0, st>>>(ctx->e, d, ctx->sc, ctx->chunk_off,
+                                                       ctx->n_chunks);
   EFCP_LAUNCHED();
   k_scan_counts<<<1, 1024, 0, st>>>(ctx->chunk_off, ctx->n_chunks, &ctx->sc->n_cand);
   EFCP_LAUNCHED();
-  k_compact_cand<<<ctx->n_chunks, kChunkThreads, 0, st>>>(ctx->e, d, ctx->sc, ctx->chunk_off,
-                                                          ctx->cand_idx, ctx->cand_val, hist2);
+  k_compact_cand<<<chunk_grid, kChunkThreads, 0, st>>>(ctx->e, d, ctx->sc, ctx->chunk_off,
+                                                       ctx->cand_idx, ctx->cand_val, hist2,
+                                                       ctx->n_chunks);
   EFCP_LAUNCHED();
   k_pick<kBins2, 2><<<1, 1024, 0, st>>>(hist2, ctx->sc, uint32_t(k));
   EFCP_LAUNCHED();
@@ -352,7 +355,10 @@ int efcp_step(efcp_ctx* ctx, const float* grad, float* update, void* stream_) {
                                                    ctx->sel_gt, ctx->sel_eq, ctx->sel_idx,
                                                    ctx->sel_val, ctx->e, k);
   EFCP_LAUNCHED();
-  k_layout_row<<<(ctx->n_slabs + kLayoutWarps) / kLayoutWarps, kLayoutWarps * 32, 0, st>>>(
+  k_row_offsets<<<ctx->num_sms * 4, 256, 0, st>>>(ctx->sel_idx, k, ctx->W, ctx->n_slabs, m, slot,
+                                                  ctx->offs);
+  EFCP_LAUNCHED();
+  k_layout_row<<<(ctx->n_slabs + kLayoutWarps - 1) / kLayoutWarps, kLayoutWarps * 32, 0, st>>>(
       ctx->sel_idx, ctx->sel_val, k, ctx->W, ctx->n_slabs, m, slot, ctx->offs, row_idx, row_val,
       ctx->slab_ctr);
   EFCP_LAUNCHED();
@@ -664,10 +670,10 @@ extern "C" int efcp_topk_static(const float* a, int64_t d, int64_t k, int32_t* i
   const int cand_grid = sms * 4;
   k_hist1_only<<<sms * 2, 512, 0, st>>>(a, d, hist1);
   k_pick<kBins1, 1><<<1, 1024, 0, st>>>(hist1, sc, uint32_t(k));
-  k_count_chunks<<<n_chunks, kChunkThreads, 0, st>>>(a, d, sc, chunk_off);
+  k_count_chunks<<<n_chunks, kChunkThreads, 0, st>>>(a, d, sc, chunk_off, n_chunks);
   k_scan_counts<<<1, 1024, 0, st>>>(chunk_off, n_chunks, &sc->n_cand);
   k_compact_cand<<<n_chunks, kChunkThreads, 0, st>>>(a, d, sc, chunk_off, cand_idx, cand_val,
-                                                     hist2);
+                                                     hist2, n_chunks);
   k_pick<kBins2, 2><<<1, 1024, 0, st>>>(hist2, sc, uint32_t(k));
   k_hist3<<<cand_grid, 256, 0, st>>>(cand_val, sc, hist3);
   k_pick<kBins3, 3><<<1, 1024, 0, st>>>(hist3, sc, uint32_t(k));

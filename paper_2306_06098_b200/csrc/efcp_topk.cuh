@@ -130,35 +130,70 @@ __device__ __forceinline__ void load_chunk8(const float* __restrict__ a, int64_t
   }
 }
 
-// Per chunk of the accumulator: how many entries have digit 1 >= b1.
+// Per chunk of the accumulator: how many entries have digit 1 >= b1.  Blocks stride over
+// the chunks.
 __global__ void __launch_bounds__(kChunkThreads) k_count_chunks(const float* __restrict__ a,
                                                                  int64_t d, const Scalars* sc,
-                                                                 int32_t* __restrict__ cnt) {
+                                                                 int32_t* __restrict__ cnt,
+                                                                 int n_chunks) {
   __shared__ int sm[33];
   const uint32_t b1 = sc->b1;
-  const int64_t base = int64_t(blockIdx.x) * kChunk + threadIdx.x * kPerThread;
-  float v[kPerThread];
-  bool ok[kPerThread];
-  load_chunk8(a, base, d, v, ok);
-  int c = 0;
+  for (int ch = blockIdx.x; ch < n_chunks; ch += gridDim.x) {
+    const int64_t base = int64_t(ch) * kChunk + threadIdx.x * kPerThread;
+    float v[kPerThread];
+    bool ok[kPerThread];
+    load_chunk8(a, base, d, v, ok);
+    int c = 0;
 #pragma unroll
-  for (int q = 0; q < kPerThread; ++q) c += (ok[q] && (mag_key(v[q]) >> kShift1) >= b1) ? 1 : 0;
-  int total;
-  (void)block_excl_scan<int>(c, &total, sm);
-  if (threadIdx.x == 0) cnt[blockIdx.x] = total;
+    for (int q = 0; q < kPerThread; ++q) c += (ok[q] && (mag_key(v[q]) >> kShift1) >= b1) ? 1 : 0;
+    int total;
+    (void)block_excl_scan<int>(c, &total, sm);
+    if (threadIdx.x == 0) cnt[ch] = total;
+  }
 }
 
 // In-place exclusive scan of n chunk counts by one block; cnt[n] and *total_out get the sum.
+// Tiles of 16384 counts: every thread scans 16 consecutive counts (vector loads), the
+// thread sums are scanned across the block.
 __global__ void __launch_bounds__(1024) k_scan_counts(int32_t* __restrict__ cnt, int n,
                                                        int32_t* total_out) {
   __shared__ int sm[33];
+  constexpr int kPer = 16;  // counts per thread and tile
   int carry = 0;
-  for (int base = 0; base < n; base += 1024) {
-    const int i = base + threadIdx.x;
-    const int v = i < n ? cnt[i] : 0;
+  for (int base = 0; base < n; base += 1024 * kPer) {
+    const int lo = base + int(threadIdx.x) * kPer;
+    int v[kPer];
+    if (lo + kPer <= n) {
+      const int4* p = reinterpret_cast<const int4*>(cnt + lo);  // cnt is 256-byte aligned
+#pragma unroll
+      for (int q = 0; q < kPer / 4; ++q) {
+        const int4 x = p[q];
+        v[4 * q] = x.x; v[4 * q + 1] = x.y; v[4 * q + 2] = x.z; v[4 * q + 3] = x.w;
+      }
+    } else {
+#pragma unroll
+      for (int q = 0; q < kPer; ++q) v[q] = lo + q < n ? cnt[lo + q] : 0;
+    }
+    int mine = 0;
+#pragma unroll
+    for (int q = 0; q < kPer; ++q) mine += v[q];
     int total;
-    const int ex = block_excl_scan<int>(v, &total, sm);
-    if (i < n) cnt[i] = carry + ex;
+    int run = carry + block_excl_scan<int>(mine, &total, sm);
+#pragma unroll
+    for (int q = 0; q < kPer; ++q) {
+      const int x = v[q];
+      v[q] = run;
+      run += x;
+    }
+    if (lo + kPer <= n) {
+      int4* p = reinterpret_cast<int4*>(cnt + lo);
+#pragma unroll
+      for (int q = 0; q < kPer / 4; ++q) p[q] = make_int4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+    } else {
+#pragma unroll
+      for (int q = 0; q < kPer; ++q)
+        if (lo + q < n) cnt[lo + q] = v[q];
+    }
     carry += total;
   }
   if (threadIdx.x == 0) {
@@ -169,34 +204,38 @@ __global__ void __launch_bounds__(1024) k_scan_counts(int32_t* __restrict__ cnt,
 
 // Ordered compaction of the candidates (digit 1 >= b1) and histogram of digit 2 over
 // the entries inside the threshold bin.
-__global__ void __launch_bounds__(kChunkThreads) k_compact_cand(
+__global__ void __launch_bounds__(kChunkThreads, 8) k_compact_cand(
     const float* __restrict__ a, int64_t d, const Scalars* sc, const int32_t* __restrict__ off,
-    int32_t* __restrict__ cand_idx, float* __restrict__ cand_val, uint32_t* __restrict__ hist2) {
+    int32_t* __restrict__ cand_idx, float* __restrict__ cand_val, uint32_t* __restrict__ hist2,
+    int n_chunks) {
   __shared__ uint32_t h[kBins2];
   __shared__ int sm[33];
   for (int i = threadIdx.x; i < kBins2; i += blockDim.x) h[i] = 0u;
   __syncthreads();
   const uint32_t b1 = sc->b1;
-  const int64_t base = int64_t(blockIdx.x) * kChunk + threadIdx.x * kPerThread;
-  float v[kPerThread];
-  bool ok[kPerThread];
-  load_chunk8(a, base, d, v, ok);
-  int c = 0;
+  for (int ch = blockIdx.x; ch < n_chunks; ch += gridDim.x) {
+    if (off[ch + 1] == off[ch]) continue;  // no candidate in this chunk (block-uniform)
+    const int64_t base = int64_t(ch) * kChunk + threadIdx.x * kPerThread;
+    float v[kPerThread];
+    bool ok[kPerThread];
+    load_chunk8(a, base, d, v, ok);
+    int c = 0;
 #pragma unroll
-  for (int q = 0; q < kPerThread; ++q) {
-    ok[q] = ok[q] && (mag_key(v[q]) >> kShift1) >= b1;
-    c += ok[q] ? 1 : 0;
-  }
-  int total;
-  int pos = off[blockIdx.x] + block_excl_scan<int>(c, &total, sm);
+    for (int q = 0; q < kPerThread; ++q) {
+      ok[q] = ok[q] && (mag_key(v[q]) >> kShift1) >= b1;
+      c += ok[q] ? 1 : 0;
+    }
+    int total;
+    int pos = off[ch] + block_excl_scan<int>(c, &total, sm);
 #pragma unroll
-  for (int q = 0; q < kPerThread; ++q) {
-    if (ok[q]) {
-      cand_idx[pos] = int32_t(base + q);
-      cand_val[pos] = v[q];
-      ++pos;
-      const uint32_t key = mag_key(v[q]);
-      if ((key >> kShift1) == b1) atomicAdd(&h[(key >> kShift2) & (kBins2 - 1)], 1u);
+    for (int q = 0; q < kPerThread; ++q) {
+      if (ok[q]) {
+        cand_idx[pos] = int32_t(base + q);
+        cand_val[pos] = v[q];
+        ++pos;
+        const uint32_t key = mag_key(v[q]);
+        if ((key >> kShift1) == b1) atomicAdd(&h[(key >> kShift2) & (kBins2 - 1)], 1u);
+      }
     }
   }
   __syncthreads();

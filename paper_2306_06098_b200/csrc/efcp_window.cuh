@@ -32,14 +32,29 @@ namespace efcp {
 constexpr int kLayoutChunk = 512;   // entries permuted together (a multiple of 32)
 constexpr int kLayoutWarps = 8;     // warps (= slabs) per block of k_layout_row
 
+// offs[s][slot] for the new row from its ascending index list: entry `pos` starts every
+// slab between its predecessor's slab (exclusive) and its own (inclusive); the last entry
+// also closes all slabs behind it.  One thread per entry, no searches.
+__global__ void __launch_bounds__(256) k_row_offsets(const int32_t* __restrict__ idx, int64_t k,
+                                                      int W, int n_slabs, int m, int slot,
+                                                      int32_t* __restrict__ offs) {
+  for (int64_t pos = int64_t(blockIdx.x) * blockDim.x + threadIdx.x; pos < k;
+       pos += int64_t(gridDim.x) * blockDim.x) {
+    const int s1 = idx[pos] / W;
+    const int s0 = pos > 0 ? idx[pos - 1] / W : -1;
+    for (int s = s0 + 1; s <= s1; ++s) offs[int64_t(s) * m + slot] = int32_t(pos);
+    if (pos == k - 1)
+      for (int s = s1 + 1; s <= n_slabs; ++s) offs[int64_t(s) * m + slot] = int32_t(k);
+  }
+}
+
 // Insert of the new row: from the ascending (index, value) list of the selection,
-//   offs[s][slot] = lower_bound(row, s * W) for s = 0..n_slabs, and
-//   ring slot <- the row, every segment in the bank-interleaved order described above.
-// One warp per slab.
+//   ring slot <- the row, every segment [offs[s][slot], offs[s+1][slot]) in the
+//   bank-interleaved order described above.  One warp per slab.
 __global__ void __launch_bounds__(kLayoutWarps * 32) k_layout_row(
     const int32_t* __restrict__ src_idx, const float* __restrict__ src_val, int64_t k, int W,
-    int n_slabs, int m, int slot, int32_t* __restrict__ offs, int32_t* __restrict__ dst_idx,
-    float* __restrict__ dst_val, int* __restrict__ slab_ctr) {
+    int n_slabs, int m, int slot, const int32_t* __restrict__ offs,
+    int32_t* __restrict__ dst_idx, float* __restrict__ dst_val, int* __restrict__ slab_ctr) {
   __shared__ int32_t s_idx[kLayoutWarps][kLayoutChunk];
   __shared__ float s_val[kLayoutWarps][kLayoutChunk];
   __shared__ uint16_t s_q[kLayoutWarps][kLayoutChunk];
@@ -47,21 +62,9 @@ __global__ void __launch_bounds__(kLayoutWarps * 32) k_layout_row(
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   if (blockIdx.x == 0 && threadIdx.x < 2) slab_ctr[threadIdx.x] = 0;  // SP and LCG work counters
   const int s = blockIdx.x * kLayoutWarps + warp;
-  if (s > n_slabs) return;
-  // lane 0 finds the segment start, lane 1 its end
-  int64_t bound = 0;
-  if (lane < 2) {
-    const int64_t target = int64_t(s + lane) * W;
-    int64_t lo = 0, hi = k;
-    while (lo < hi) {
-      const int64_t mid = (lo + hi) >> 1;
-      if (int64_t(src_idx[mid]) < target) lo = mid + 1; else hi = mid;
-    }
-    bound = lo;
-  }
-  const int seg_b = int(__shfl_sync(0xFFFFFFFFu, bound, 0));
-  const int seg_e = s < n_slabs ? int(__shfl_sync(0xFFFFFFFFu, bound, 1)) : seg_b;
-  if (lane == 0) offs[int64_t(s) * m + slot] = seg_b;
+  if (s >= n_slabs) return;
+  const int seg_b = offs[int64_t(s) * m + slot];
+  const int seg_e = offs[int64_t(s + 1) * m + slot];
   int32_t* ci = s_idx[warp];
   float* cv = s_val[warp];
   uint16_t* cq = s_q[warp];
@@ -70,17 +73,17 @@ __global__ void __launch_bounds__(kLayoutWarps * 32) k_layout_row(
     const int n = min(kLayoutChunk, seg_e - c0);
     cnt[lane] = 0;
     __syncwarp();
-    // occurrence number of every entry within its bank, in ascending index order
+    // stage the chunk (all loads in flight together), then number every entry within its
+    // bank in ascending index order
+    for (int a = lane; a < n; a += 32) {
+      ci[a] = src_idx[c0 + a];
+      cv[a] = src_val[c0 + a];
+    }
+    __syncwarp();
     for (int a0 = 0; a0 < n; a0 += 32) {
       const int a = a0 + lane;
       const bool on = a < n;
-      int idx = 0;
-      if (on) {
-        idx = src_idx[c0 + a];
-        ci[a] = idx;
-        cv[a] = src_val[c0 + a];
-      }
-      const int bank = idx & 31;
+      const int bank = on ? (ci[a] & 31) : 0;
       const unsigned same = __match_any_sync(0xFFFFFFFFu, on ? bank : 32 + lane);
       const int before = on ? cnt[bank] : 0;
       __syncwarp();
