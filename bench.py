@@ -146,7 +146,7 @@ def run_reference(args, world, rank):
     """The reference arm: the CPU oracle on a bounded slice of the same workload."""
     if rank != 0:
         return
-    w = gradgen.WORKLOADS[args.workload]
+    w = get_workload(args.workload)
     # Oracle cost per step is close to linear in d (with k/d and m fixed).  Shrink d and k
     # by `shrink` so that warmup + steps stay within a few minutes, report steps/s divided
     # by the same factor.
@@ -184,13 +184,23 @@ def run_reference(args, world, rank):
     print(json.dumps(line), flush=True)
 
 
+def get_workload(name):
+    if name.startswith("custom:"):
+        f = name.split(":", 1)[1].split(",")
+        return gradgen.Workload(name, int(f[0]), int(f[1]), int(f[2]), float(f[3]), 200, int(f[4]),
+                                int(f[5]) if len(f) > 5 else None)
+    return gradgen.WORKLOADS[name]
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=40)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default=gradgen.C4.name, choices=sorted(gradgen.WORKLOADS))
+    ap.add_argument("--workload", default=gradgen.C4.name,
+                    help="one of %s, or custom:d,m,k,lambda,rank[,scale_block] (profiling cases)"
+                    % ", ".join(sorted(gradgen.WORKLOADS)))
     ap.add_argument("--prefill", type=int, default=-1,
                     help="untimed steps before warm-up; -1 = m (fill the whole window)")
     ap.add_argument("--e2e-steps", type=int, default=5)
@@ -211,7 +221,7 @@ def main():
 
     torch.cuda.set_device(local)
     device = torch.device("cuda", local)
-    w = gradgen.WORKLOADS[args.workload]
+    w = get_workload(args.workload)
     K, W = args.steps, args.warmup
     gs = gradgen.GradStream(w.d, w.rank, w.seed + rank, w.scale_block, w.noise, str(device))
     opt = binding.Efcp(w.d, w.m, w.k, w.lam)

@@ -54,6 +54,8 @@ struct efcp_ctx {
   double* vecs = nullptr;  // 8 m-vectors: delta, aprime, y, bold, z, w, res, dw
   float* wf = nullptr;
   int* slab_ctr = nullptr;   // work counters of the slab kernels (SP, LCG)
+  int64_t* colsum = nullptr; // n_slabs + 1 column sums of offs
+  int32_t* order = nullptr;  // n_slabs slabs, heavy first
   float* stage_g = nullptr;  // efcp_step_host staging
   float* stage_u = nullptr;
   int last_cuda = 0;
@@ -107,6 +109,7 @@ Sizes compute_sizes(int64_t d, int32_t m, int64_t k, int num_sms) {
   b += 2 * align256(k * 4);                               // sel_idx, sel_val
   b += align256(sizeof(Scalars));
   b += align256(int64_t(z.n_slabs) * m * 8);              // slab_part
+  b += align256(int64_t(z.n_slabs + 1) * 8) + align256(int64_t(z.n_slabs) * 4);  // colsum, order
   b += align256(int64_t(kSpParts) * m * 8);               // partial
   b += align256(int64_t(8) * m * 8);                      // vecs
   b += align256(int64_t(m) * 4);                          // wf
@@ -257,6 +260,8 @@ int efcp_create_ex(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float lambda
   if ((rc = dev_alloc(ctx, &ctx->vecs, int64_t(8) * m * 8))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->wf, int64_t(m) * 4))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->slab_ctr, 256))) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->colsum, int64_t(z.n_slabs + 1) * 8))) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->order, int64_t(z.n_slabs) * 4))) return fail(rc);
 
 
   bool ok = true;
@@ -264,6 +269,7 @@ int efcp_create_ex(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float lambda
   ok &= cudaMemset(ctx->V, 0, size_t(mk) * 4) == cudaSuccess;
   ok &= cudaMemset(ctx->offs, 0, size_t(z.n_slabs + 1) * m * 4) == cudaSuccess;
   ok &= cudaMemset(ctx->S, 0, size_t(m) * m * 8) == cudaSuccess;
+  ok &= cudaMemset(ctx->colsum, 0, size_t(z.n_slabs + 1) * 8) == cudaSuccess;
   ok &= cudaMemset(ctx->hist, 0, (kBins1 + kBins2 + kBins3) * 4) == cudaSuccess;
   ok &= cudaMemset(ctx->sc, 0, sizeof(Scalars)) == cudaSuccess;
   ok &= cudaMemset(ctx->vecs, 0, size_t(8) * m * 8) == cudaSuccess;
@@ -356,7 +362,9 @@ int efcp_step(efcp_ctx* ctx, const float* grad, float* update, void* stream_) {
                                                    ctx->sel_val, ctx->e, k);
   EFCP_LAUNCHED();
   k_row_offsets<<<ctx->num_sms * 4, 256, 0, st>>>(ctx->sel_idx, k, ctx->W, ctx->n_slabs, m, slot,
-                                                  ctx->offs);
+                                                  ctx->offs, ctx->colsum);
+  EFCP_LAUNCHED();
+  k_slab_order<<<1, 1024, 0, st>>>(ctx->colsum, ctx->n_slabs, ctx->order);
   EFCP_LAUNCHED();
   k_layout_row<<<(ctx->n_slabs + kLayoutWarps - 1) / kLayoutWarps, kLayoutWarps * 32, 0, st>>>(
       ctx->sel_idx, ctx->sel_val, k, ctx->W, ctx->n_slabs, m, slot, ctx->offs, row_idx, row_val,
@@ -366,7 +374,8 @@ int efcp_step(efcp_ctx* ctx, const float* grad, float* update, void* stream_) {
   const size_t smem = slab_smem_bytes(ctx->W, m);
   prof_mark(ctx, 1, st);
   k_sp_rows<<<ctx->grid_slab, kSlabThreads, smem, st>>>(ctx->I, ctx->V, ctx->offs, k, m, ctx->W,
-                                                ctx->n_slabs, slot, ctx->slab_part, ctx->slab_ctr);
+                                                ctx->n_slabs, slot, ctx->slab_part, ctx->slab_ctr,
+                                                ctx->order);
   EFCP_LAUNCHED();
   prof_mark(ctx, 2, st);
   const int sp_parts = ctx->n_slabs < kSpParts ? ctx->n_slabs : kSpParts;
@@ -395,10 +404,12 @@ int efcp_step(efcp_ctx* ctx, const float* grad, float* update, void* stream_) {
   prof_mark(ctx, 3, st);
   if ((reinterpret_cast<uintptr_t>(update) & 15) == 0)
     k_lcg<true><<<ctx->grid_slab, kSlabThreads, smem, st>>>(ctx->I, ctx->V, ctx->offs, k, m, ctx->W,
-                                                    ctx->n_slabs, ctx->wf, update, d, ctx->slab_ctr + 1);
+                                                    ctx->n_slabs, ctx->wf, update, d, ctx->slab_ctr + 1,
+                                                    ctx->order);
   else
     k_lcg<false><<<ctx->grid_slab, kSlabThreads, smem, st>>>(ctx->I, ctx->V, ctx->offs, k, m, ctx->W,
-                                                     ctx->n_slabs, ctx->wf, update, d, ctx->slab_ctr + 1);
+                                                     ctx->n_slabs, ctx->wf, update, d, ctx->slab_ctr + 1,
+                                                    ctx->order);
   EFCP_LAUNCHED();
   prof_mark(ctx, 4, st);
   if (ctx->prof_on && ctx->prof_n < ctx->prof_cap) ++ctx->prof_n;

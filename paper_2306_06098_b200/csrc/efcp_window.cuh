@@ -34,18 +34,52 @@ constexpr int kLayoutWarps = 8;     // warps (= slabs) per block of k_layout_row
 
 // offs[s][slot] for the new row from its ascending index list: entry `pos` starts every
 // slab between its predecessor's slab (exclusive) and its own (inclusive); the last entry
-// also closes all slabs behind it.  One thread per entry, no searches.
+// also closes all slabs behind it.  One thread per entry, no searches.  colsum[s] =
+// sum over the rows of offs[s][.] is kept up to date (one writer per s), so that
+// colsum[s + 1] - colsum[s] is the number of window entries in slab s.
 __global__ void __launch_bounds__(256) k_row_offsets(const int32_t* __restrict__ idx, int64_t k,
                                                       int W, int n_slabs, int m, int slot,
-                                                      int32_t* __restrict__ offs) {
+                                                      int32_t* __restrict__ offs,
+                                                      int64_t* __restrict__ colsum) {
+  auto put = [&](int s, int32_t v) {
+    int32_t* p = offs + int64_t(s) * m + slot;
+    colsum[s] += int64_t(v) - int64_t(*p);
+    *p = v;
+  };
   for (int64_t pos = int64_t(blockIdx.x) * blockDim.x + threadIdx.x; pos < k;
        pos += int64_t(gridDim.x) * blockDim.x) {
     const int s1 = idx[pos] / W;
     const int s0 = pos > 0 ? idx[pos - 1] / W : -1;
-    for (int s = s0 + 1; s <= s1; ++s) offs[int64_t(s) * m + slot] = int32_t(pos);
+    for (int s = s0 + 1; s <= s1; ++s) put(s, int32_t(pos));
     if (pos == k - 1)
-      for (int s = s1 + 1; s <= n_slabs; ++s) offs[int64_t(s) * m + slot] = int32_t(k);
+      for (int s = s1 + 1; s <= n_slabs; ++s) put(s, int32_t(k));
   }
+}
+
+// order[] = the slabs, heaviest first up to a factor 2^(1/4): a counting sort on the top
+// bits of the slab weight colsum[s + 1] - colsum[s].  The slab kernels hand out slabs in
+// this order, so the heavy slabs are never the last ones a block starts.  The order inside
+// a weight class is arbitrary; no result depends on it.  One block.
+constexpr int kOrderBins = 1024;
+__global__ void __launch_bounds__(1024) k_slab_order(const int64_t* __restrict__ colsum,
+                                                      int n_slabs, int32_t* __restrict__ order) {
+  __shared__ int cnt[kOrderBins];
+  __shared__ int sm[33];
+  for (int i = threadIdx.x; i < kOrderBins; i += blockDim.x) cnt[i] = 0;
+  __syncthreads();
+  auto bin_of = [&](int s) {
+    const float w = float(colsum[s + 1] - colsum[s]);           // >= 0
+    const int key = int(__float_as_uint(w) >> 21);               // exponent and 2 mantissa bits
+    return kOrderBins - 1 - min(key, kOrderBins - 1);            // heavy slabs first
+  };
+  for (int s = threadIdx.x; s < n_slabs; s += blockDim.x) atomicAdd(&cnt[bin_of(s)], 1);
+  __syncthreads();
+  int total;
+  const int mine = cnt[threadIdx.x];
+  const int start = block_excl_scan<int>(mine, &total, sm);
+  cnt[threadIdx.x] = start;
+  __syncthreads();
+  for (int s = threadIdx.x; s < n_slabs; s += blockDim.x) order[atomicAdd(&cnt[bin_of(s)], 1)] = s;
 }
 
 // Insert of the new row: from the ascending (index, value) list of the selection,
@@ -149,7 +183,7 @@ __device__ __forceinline__ void prefetch_segment(const int32_t* Ir, const float*
 // with slab b and then draws the next unprocessed slab from a counter in global memory
 // (cleared by k_layout_row earlier in the step).  The draw for the next slab is issued at
 // the start of the current one, so its latency is hidden.  Results do not depend on which
-// block processes which slab: LCG slabs are disjoint outputs, and SP writes one partial
+// block processes which slab, nor on the order k_slab_order puts the slabs in: LCG slabs are disjoint outputs, and SP writes one partial
 // sum per (slab, row) that is reduced afterwards in slab order.
 
 // Scalar products of every window row with the newest row (x = dens(c_t)):
@@ -157,7 +191,8 @@ __device__ __forceinline__ void prefetch_segment(const int32_t* Ir, const float*
 // accumulated in fp64 (every fp32 x fp32 product is exact in fp64).
 __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_sp_rows(
     const int32_t* __restrict__ I, const float* __restrict__ V, const int32_t* __restrict__ offs,
-    int64_t k, int m, int W, int n_slabs, int slot, double* __restrict__ slab_part, int* ctr) {
+    int64_t k, int m, int W, int n_slabs, int slot, double* __restrict__ slab_part, int* ctr,
+    const int32_t* __restrict__ order) {
   extern __shared__ __align__(16) unsigned char smraw[];
   float* xs = reinterpret_cast<float*>(smraw);
   int32_t* seg = reinterpret_cast<int32_t*>(smraw + size_t(W) * 4 + size_t(m) * 8);
@@ -165,7 +200,8 @@ __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_sp_rows(
   const int32_t* Inew = I + int64_t(slot) * k;
   const float* Vnew = V + int64_t(slot) * k;
   __shared__ int s_next;
-  for (int s = blockIdx.x; s < n_slabs;) {
+  for (int t = blockIdx.x; t < n_slabs;) {  // t: position in the hand-out order
+    const int s = order[t];
     __syncthreads();
     if (tid == 0) s_next = int(gridDim.x) + atomicAdd(ctr, 1);
     float4* xs4 = reinterpret_cast<float4*>(xs);
@@ -235,7 +271,7 @@ __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_sp_rows(
       acc = warp_sum(acc);
       if (lane == 0) out[r] = acc;
     }
-    s = s_next;
+    t = s_next;
   }
 }
 
@@ -281,7 +317,7 @@ template <bool VEC>
 __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_lcg(
     const int32_t* __restrict__ I, const float* __restrict__ V, const int32_t* __restrict__ offs,
     int64_t k, int m, int W, int n_slabs, const float* __restrict__ wf, float* __restrict__ u,
-    int64_t d, int* ctr) {
+    int64_t d, int* ctr, const int32_t* __restrict__ order) {
   extern __shared__ __align__(16) unsigned char smraw[];
   float* acc = reinterpret_cast<float*>(smraw);
   float* wc = reinterpret_cast<float*>(smraw + size_t(W) * 4);
@@ -291,7 +327,8 @@ __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_lcg(
   float4* acc4 = reinterpret_cast<float4*>(acc);
   for (int i = tid; i < (W >> 2); i += blockDim.x) acc4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
   __shared__ int s_next;
-  for (int s = blockIdx.x; s < n_slabs;) {
+  for (int t = blockIdx.x; t < n_slabs;) {  // t: position in the hand-out order
+    const int s = order[t];
     __syncthreads();
     if (tid == 0) s_next = int(gridDim.x) + atomicAdd(ctr, 1);
     for (int r = tid; r < m; r += blockDim.x) {
@@ -362,7 +399,7 @@ __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_lcg(
         acc[i] = 0.f;
       }
     }
-    s = s_next;
+    t = s_next;
   }
 }
 
