@@ -201,6 +201,8 @@ def main():
     ap.add_argument("--workload", default=gradgen.C4.name,
                     help="one of %s, or custom:d,m,k,lambda,rank[,scale_block] (profiling cases)"
                     % ", ".join(sorted(gradgen.WORKLOADS)))
+    ap.add_argument("--rhs", default="compressed", choices=["compressed", "accumulator"],
+                    help="precondition c_t (Algorithm 1, default) or the whole accumulator a_t")
     ap.add_argument("--prefill", type=int, default=-1,
                     help="untimed steps before warm-up; -1 = m (fill the whole window)")
     ap.add_argument("--e2e-steps", type=int, default=5)
@@ -224,7 +226,9 @@ def main():
     w = get_workload(args.workload)
     K, W = args.steps, args.warmup
     gs = gradgen.GradStream(w.d, w.rank, w.seed + rank, w.scale_block, w.noise, str(device))
-    opt = binding.Efcp(w.d, w.m, w.k, w.lam)
+    acc = args.rhs == "accumulator"
+    opt = binding.Efcp(w.d, w.m, w.k, w.lam,
+                       binding.RHS_ACCUMULATOR if acc else binding.RHS_COMPRESSED)
     gbuf = torch.empty(w.d, dtype=torch.float32, device=device)
     ubuf = torch.empty(w.d, dtype=torch.float32, device=device)
 
@@ -290,16 +294,18 @@ def main():
 
     # roofline of the dominant kernel (HBM bound): algorithmic bytes per launch / time
     peak, peak_src = load_peak()
-    alg = {"sp": 8 * w.m * w.k, "lcg": 8 * w.m * w.k + 4 * w.d}
+    # x = a_t adds one read of xi to SP and one to LCG
+    alg = {"sp": 8 * w.m * w.k + (4 * w.d if acc else 0),
+           "lcg": 8 * w.m * w.k + 4 * w.d + (4 * w.d if acc else 0)}
     kern = max(("sp", "lcg"), key=lambda s: stages[s])
     avg_ms = stages[kern] / max(n_rec, 1)
     achieved = alg[kern] / (avg_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": {"sp": "k_sp_rows", "lcg": "k_lcg"}[kern],
                 "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": NCU_TRAFFIC_BYTES.get(w.name, {}).get(kern),
+                "traffic": None if acc else NCU_TRAFFIC_BYTES.get(w.name, {}).get(kern),
                 "peak_source": peak_src, "algorithmic_bytes_per_launch": alg[kern],
                 "avg_launch_ms": avg_ms}
-    step_bytes = 16 * w.m * w.k + 16 * w.d + 8 * w.k
+    step_bytes = 16 * w.m * w.k + 16 * w.d + 8 * w.k + (8 * w.d if acc else 0)
     step_gbs = step_bytes / (ms_per_step * 1e-3) / 1e9
     stage_ms = {s: stages[s] / max(n_rec, 1) for s in stages}
 
@@ -318,7 +324,7 @@ def main():
             "warmup": W, "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": w.name, "d": w.d, "m": w.m, "k": w.k, "lambda": w.lam,
-                       "rhs": "compressed", "prefill_steps": prefill,
+                       "rhs": args.rhs, "prefill_steps": prefill,
                        "parallelism": f"replicas x{world}",
                        "l2": "inputs larger than L2 (window %.2f GB, gradient %.2f GB)" % (
                            8 * w.m * w.k / 1e9, 4 * w.d / 1e9)},

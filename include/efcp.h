@@ -41,7 +41,8 @@ typedef struct efcp_ctx efcp_ctx;
 /* flags for efcp_create_ex */
 #define EFCP_RHS_COMPRESSED  0u /* u_t = A(c_t): precondition the compressed accumulator
                                    (Algorithm 1, line 8) - the default                    */
-#define EFCP_RHS_ACCUMULATOR 1u /* precondition the full accumulator a_t = xi_t + c_t     */
+#define EFCP_RHS_ACCUMULATOR 1u /* precondition the full accumulator a_t = xi_t + c_t
+                                   (u = F^-1 a_t; costs one more read of xi in SP and LCG)  */
 
 /*
  * efcp_create / efcp_create_ex - Algorithm 1 lines 1-2: set up an empty window and
@@ -93,9 +94,9 @@ int efcp_destroy(efcp_ctx* ctx);
  *                    values.  A slot never written reads as indices 0..k-1, values 0.
  *   efcp_get_gram  : S = G G^T, m*m doubles, row-major, exactly symmetric
  *                    (Section 2.1: row and column i are replaced together).
- *   efcp_get_weights: the m fp64 weights w of the last step's linear combination
- *                    (update = x/lambda*[mode] + sum_r w_r row_r; in the default mode
- *                    update = sum_r w_r row_r).
+ *   efcp_get_weights: the m fp64 weights w of the last step's linear combination:
+ *                    update = sum_r w_r row_r in the default mode,
+ *                    update = xi/lambda + sum_r w_r row_r with EFCP_RHS_ACCUMULATOR.
  * Returns the sticky device status if it is an error, else EFCP_OK.
  */
 int efcp_get_error(efcp_ctx* ctx, float* host_e);

@@ -51,7 +51,7 @@ struct efcp_ctx {
   Scalars* sc = nullptr;
   double* slab_part = nullptr;  // SP: one partial sum per (slab, row)
   double* partial = nullptr;    // SP: kSpParts x m sums of slab partials
-  double* vecs = nullptr;  // 8 m-vectors: delta, aprime, y, bold, z, w, res, dw
+  double* vecs = nullptr;  // 9 m-vectors: delta, aprime, y, bold, z, w, res, dw, rhs
   float* wf = nullptr;
   int* slab_ctr = nullptr;   // work counters of the slab kernels (SP, LCG)
   int64_t* colsum = nullptr; // n_slabs + 1 column sums of offs
@@ -83,7 +83,7 @@ int pick_slab_width(int64_t d, int m, int num_sms) {
     if (v >= 256 && v <= 49152 && (v & 31) == 0) return v;
   }
   // shared memory: W*4 + 16*m must stay under the 227 KB per-block limit
-  while ((size_t(W) * 4 + size_t(m) * 16) * kSlabBlocksPerSM > 200 * 1024 && W > 1024) W >>= 1;
+  while (slab_smem_bytes(W, m) * kSlabBlocksPerSM > 200 * 1024 && W > 1024) W >>= 1;
   // enough slabs to give every SM several
   while (W > 1024 && (d + W - 1) / W < int64_t(4) * num_sms) W >>= 1;
   return W;
@@ -111,7 +111,7 @@ Sizes compute_sizes(int64_t d, int32_t m, int64_t k, int num_sms) {
   b += align256(int64_t(z.n_slabs) * m * 8);              // slab_part
   b += align256(int64_t(z.n_slabs + 1) * 8) + align256(int64_t(z.n_slabs) * 4);  // colsum, order
   b += align256(int64_t(kSpParts) * m * 8);               // partial
-  b += align256(int64_t(8) * m * 8);                      // vecs
+  b += align256(int64_t(9) * m * 8);                      // vecs
   b += align256(int64_t(m) * 4);                          // wf
   z.total = b;
   return z;
@@ -220,7 +220,6 @@ int efcp_create_ex(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float lambda
   *out = nullptr;
   if (!valid_args(d, m, k) || !(lambda > 0.f) || !std::isfinite(lambda)) return EFCP_EINVAL;
   if (flags & ~EFCP_RHS_ACCUMULATOR) return EFCP_EINVAL;
-  if (flags & EFCP_RHS_ACCUMULATOR) return EFCP_EINVAL;  // not built yet
   efcp_ctx* ctx = new (std::nothrow) efcp_ctx();
   if (!ctx) return EFCP_ENOMEM;
   int rc = EFCP_OK;
@@ -255,9 +254,10 @@ int efcp_create_ex(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float lambda
   if ((rc = dev_alloc(ctx, &ctx->sel_idx, k * 4))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->sel_val, k * 4))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->sc, sizeof(Scalars)))) return fail(rc);
-  if ((rc = dev_alloc(ctx, &ctx->slab_part, int64_t(z.n_slabs) * m * 8))) return fail(rc);
-  if ((rc = dev_alloc(ctx, &ctx->partial, int64_t(kSpParts) * m * 8))) return fail(rc);
-  if ((rc = dev_alloc(ctx, &ctx->vecs, int64_t(8) * m * 8))) return fail(rc);
+  const int64_t sums = (flags & EFCP_RHS_ACCUMULATOR) ? 2 : 1;
+  if ((rc = dev_alloc(ctx, &ctx->slab_part, int64_t(z.n_slabs) * m * 8 * sums))) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->partial, int64_t(kSpParts) * m * 8 * sums))) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->vecs, int64_t(9) * m * 8))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->wf, int64_t(m) * 4))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->slab_ctr, 256))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->colsum, int64_t(z.n_slabs + 1) * 8))) return fail(rc);
@@ -272,17 +272,18 @@ int efcp_create_ex(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float lambda
   ok &= cudaMemset(ctx->colsum, 0, size_t(z.n_slabs + 1) * 8) == cudaSuccess;
   ok &= cudaMemset(ctx->hist, 0, (kBins1 + kBins2 + kBins3) * 4) == cudaSuccess;
   ok &= cudaMemset(ctx->sc, 0, sizeof(Scalars)) == cudaSuccess;
-  ok &= cudaMemset(ctx->vecs, 0, size_t(8) * m * 8) == cudaSuccess;
+  ok &= cudaMemset(ctx->vecs, 0, size_t(9) * m * 8) == cudaSuccess;
   ok &= cudaMemset(ctx->wf, 0, size_t(m) * 4) == cudaSuccess;
   k_init_rows<<<ctx->num_sms * 4, 256>>>(ctx->I, k, mk);
   k_init_identity<<<ctx->num_sms * 2, 256>>>(ctx->B, m, 1.0 / (double(m) * double(lambda)));
   const size_t smem = slab_smem_bytes(z.W, m);
-  ok &= cudaFuncSetAttribute(k_sp_rows, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             int(smem)) == cudaSuccess;
-  ok &= cudaFuncSetAttribute(k_lcg<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             int(smem)) == cudaSuccess;
-  ok &= cudaFuncSetAttribute(k_lcg<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             int(smem)) == cudaSuccess;
+  const auto attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
+  ok &= cudaFuncSetAttribute(k_sp_rows<false>, attr, int(smem)) == cudaSuccess;
+  ok &= cudaFuncSetAttribute(k_sp_rows<true>, attr, int(smem)) == cudaSuccess;
+  ok &= cudaFuncSetAttribute(k_lcg<true, false>, attr, int(smem)) == cudaSuccess;
+  ok &= cudaFuncSetAttribute(k_lcg<false, false>, attr, int(smem)) == cudaSuccess;
+  ok &= cudaFuncSetAttribute(k_lcg<true, true>, attr, int(smem)) == cudaSuccess;
+  ok &= cudaFuncSetAttribute(k_lcg<false, true>, attr, int(smem)) == cudaSuccess;
   ok &= cudaDeviceSynchronize() == cudaSuccess;
   if (!ok) {
     ctx->last_cuda = int(cudaGetLastError());
@@ -371,19 +372,28 @@ int efcp_step(efcp_ctx* ctx, const float* grad, float* update, void* stream_) {
       ctx->slab_ctr);
   EFCP_LAUNCHED();
   // scalar products with the new row, Gram row/column
+  const bool acc_mode = (ctx->flags & EFCP_RHS_ACCUMULATOR) != 0;
+  const int m2 = acc_mode ? 2 * m : m;  // sums per slab: <row, c> and, for x = a, <row, xi>
+  double* rhs = dw + m;
   const size_t smem = slab_smem_bytes(ctx->W, m);
   prof_mark(ctx, 1, st);
-  k_sp_rows<<<ctx->grid_slab, kSlabThreads, smem, st>>>(ctx->I, ctx->V, ctx->offs, k, m, ctx->W,
-                                                ctx->n_slabs, slot, ctx->slab_part, ctx->slab_ctr,
-                                                ctx->order);
+  if (acc_mode)
+    k_sp_rows<true><<<ctx->grid_slab, kSlabThreads, smem, st>>>(
+        ctx->I, ctx->V, ctx->offs, k, m, ctx->W, ctx->n_slabs, slot, ctx->slab_part, ctx->slab_ctr,
+        ctx->order, ctx->e, d);
+  else
+    k_sp_rows<false><<<ctx->grid_slab, kSlabThreads, smem, st>>>(
+        ctx->I, ctx->V, ctx->offs, k, m, ctx->W, ctx->n_slabs, slot, ctx->slab_part, ctx->slab_ctr,
+        ctx->order, ctx->e, d);
   EFCP_LAUNCHED();
   prof_mark(ctx, 2, st);
   const int sp_parts = ctx->n_slabs < kSpParts ? ctx->n_slabs : kSpParts;
-  k_sp_reduce<<<dim3((m + 127) / 128, sp_parts), 128, 0, st>>>(ctx->slab_part, ctx->n_slabs, m,
-                                                               ctx->partial);
+  k_sp_reduce<<<dim3((m2 + 127) / 128, sp_parts), 128, 0, st>>>(ctx->slab_part, ctx->n_slabs, m2,
+                                                                ctx->partial);
   EFCP_LAUNCHED();
-  k_sp_finish<<<(m + 127) / 128, 128, 0, st>>>(ctx->partial, sp_parts, m, slot, delta,
-                                               ctx->S, aprime);
+  k_sp_finish<<<(m + 127) / 128, 128, 0, st>>>(ctx->partial, sp_parts, m, slot, delta, ctx->S,
+                                               aprime, acc_mode ? rhs : nullptr,
+                                               double(ctx->lambda));
   EFCP_LAUNCHED();
   // m x m: remove-and-border update of the inverse, weights, one refinement step
   const int gemv_grid = (m + 7) / 8;
@@ -394,7 +404,12 @@ int efcp_step(efcp_ctx* ctx, const float* grad, float* update, void* stream_) {
   EFCP_LAUNCHED();
   k_rank2<<<ctx->num_sms * 2, 256, 0, st>>>(ctx->B, bold, z, ctx->sc, m, slot);
   EFCP_LAUNCHED();
-  k_residual<<<gemv_grid, 256, 0, st>>>(ctx->S, w, res, m, slot, mlambda);
+  if (acc_mode) {  // w = B' rhs replaces the column of B' that k_border_scalars wrote
+    k_gemv<<<gemv_grid, 256, 0, st>>>(ctx->B, rhs, w, m);
+    EFCP_LAUNCHED();
+  }
+  k_residual<<<gemv_grid, 256, 0, st>>>(ctx->S, w, res, m, slot, mlambda,
+                                        acc_mode ? rhs : nullptr);
   EFCP_LAUNCHED();
   k_gemv<<<gemv_grid, 256, 0, st>>>(ctx->B, res, dw, m);
   EFCP_LAUNCHED();
@@ -402,14 +417,18 @@ int efcp_step(efcp_ctx* ctx, const float* grad, float* update, void* stream_) {
   EFCP_LAUNCHED();
   // linear combination of the window rows
   prof_mark(ctx, 3, st);
-  if ((reinterpret_cast<uintptr_t>(update) & 15) == 0)
-    k_lcg<true><<<ctx->grid_slab, kSlabThreads, smem, st>>>(ctx->I, ctx->V, ctx->offs, k, m, ctx->W,
-                                                    ctx->n_slabs, ctx->wf, update, d, ctx->slab_ctr + 1,
-                                                    ctx->order);
-  else
-    k_lcg<false><<<ctx->grid_slab, kSlabThreads, smem, st>>>(ctx->I, ctx->V, ctx->offs, k, m, ctx->W,
-                                                     ctx->n_slabs, ctx->wf, update, d, ctx->slab_ctr + 1,
-                                                    ctx->order);
+  const bool uvec = (reinterpret_cast<uintptr_t>(update) & 15) == 0;
+  const float inv_lambda = 1.0f / ctx->lambda;
+#define EFCP_LCG_LAUNCH(VEC, ACC)                                                              \
+  k_lcg<VEC, ACC><<<ctx->grid_slab, kSlabThreads, smem, st>>>(                                 \
+      ctx->I, ctx->V, ctx->offs, k, m, ctx->W, ctx->n_slabs, ctx->wf, update, d,               \
+      ctx->slab_ctr + 1, ctx->order, ctx->e, inv_lambda)
+  if (acc_mode) {
+    if (uvec) EFCP_LCG_LAUNCH(true, true); else EFCP_LCG_LAUNCH(false, true);
+  } else {
+    if (uvec) EFCP_LCG_LAUNCH(true, false); else EFCP_LCG_LAUNCH(false, false);
+  }
+#undef EFCP_LCG_LAUNCH
   EFCP_LAUNCHED();
   prof_mark(ctx, 4, st);
   if (ctx->prof_on && ctx->prof_n < ctx->prof_cap) ++ctx->prof_n;

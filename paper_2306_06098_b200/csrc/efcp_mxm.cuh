@@ -16,6 +16,12 @@
 //      B' = C + z z^T / s,  B'[:, i] = B'[i, :] = -z/s,  B'[i][i] = 1/s.
 // Then w = m B'[:, i], followed by one step of iterative refinement against A itself
 // (r = m e_i - A w, w += B' r), which squares whatever error B has accumulated.
+//
+// When the right-hand side is the whole accumulator a = xi + c (xi: the error buffer after
+// the step, zero on the support of c), the c part is treated as above and the xi part
+// literally: F^-1 xi = xi/lambda - G^T A^-1 (G xi)/lambda.  Together
+//     u = xi/lambda + G^T w,   w = A^-1 (m e_i - q/lambda),   q = G xi,
+// one product with B' and the same refinement step against A.
 // All kernels are BLAS-2 shaped and L2 resident (8 MB at m = 1024): no tensor cores.
 #pragma once
 
@@ -99,11 +105,11 @@ __global__ void __launch_bounds__(256) k_rank2(double* __restrict__ B, const dou
   }
 }
 
-// res = m e_slot - (m lambda I + S) w ; one warp per row.  Also tracks max |res| / m.
+// res = rhs - (m lambda I + S) w with rhs = m e_slot when `rhs` is null; one warp per row.
 __global__ void __launch_bounds__(256) k_residual(const double* __restrict__ S,
                                                    const double* __restrict__ w,
                                                    double* __restrict__ res, int m, int slot,
-                                                   double mlambda) {
+                                                   double mlambda, const double* __restrict__ rhs) {
   const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (row >= m) return;
@@ -111,7 +117,10 @@ __global__ void __launch_bounds__(256) k_residual(const double* __restrict__ S,
   double acc = 0.0;
   for (int c = lane; c < m; c += 32) acc += Sr[c] * w[c];
   acc = warp_sum(acc);
-  if (lane == 0) res[row] = (row == slot ? double(m) : 0.0) - (mlambda * w[row] + acc);
+  if (lane == 0) {
+    const double b = rhs ? rhs[row] : (row == slot ? double(m) : 0.0);
+    res[row] = b - (mlambda * w[row] + acc);
+  }
 }
 
 // w += dw ; wf = float(w) ; sc->resid = max |res| / m.  One block.

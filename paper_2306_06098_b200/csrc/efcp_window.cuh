@@ -149,7 +149,7 @@ __global__ void __launch_bounds__(kLayoutWarps * 32) k_layout_row(
 // Shared-memory layout of the slab kernels: float slab[W]; double/float per-row
 // scratch; int32 seg[2 * m] (segment begin / end of every row in the current slab).
 __host__ __device__ inline size_t slab_smem_bytes(int W, int m) {
-  return size_t(W) * 4 + size_t(m) * 8 + size_t(m) * 8;
+  return size_t(W) * 4 + size_t(m) * 8 + size_t(m) * 8 + size_t(W) / 8;  // + bit mask (SP, x = a)
 }
 
 #ifndef EFCP_SLAB_THREADS
@@ -186,42 +186,63 @@ __device__ __forceinline__ void prefetch_segment(const int32_t* Ir, const float*
 // block processes which slab, nor on the order k_slab_order puts the slabs in: LCG slabs are disjoint outputs, and SP writes one partial
 // sum per (slab, row) that is reduced afterwards in slab order.
 
-// Scalar products of every window row with the newest row (x = dens(c_t)):
-//   slab_part[s][r] = <row_r, x> restricted to slab s
-// accumulated in fp64 (every fp32 x fp32 product is exact in fp64).
+// Scalar products of every window row with the newest row c_t:
+//   slab_part[s][r] = <row_r, c_t> restricted to slab s                      (both modes)
+// and, when the right-hand side is the whole accumulator a_t = xi_t + c_t (ACC):
+//   slab_part[s][m + r] = <row_r, xi_t> restricted to slab s,
+// accumulated in fp64 (every fp32 x fp32 product is exact in fp64).  In ACC mode the slab in
+// shared memory holds a_t (xi_t with the kept coordinates, which are zero in xi_t, filled
+// in from c_t) and a bit mask says which coordinates belong to c_t, so that one gather
+// serves both sums.  `stride` is the row length of slab_part (m or 2 m).
+template <bool ACC>
 __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_sp_rows(
     const int32_t* __restrict__ I, const float* __restrict__ V, const int32_t* __restrict__ offs,
     int64_t k, int m, int W, int n_slabs, int slot, double* __restrict__ slab_part, int* ctr,
-    const int32_t* __restrict__ order) {
+    const int32_t* __restrict__ order, const float* __restrict__ e, int64_t d) {
   extern __shared__ __align__(16) unsigned char smraw[];
   float* xs = reinterpret_cast<float*>(smraw);
   int32_t* seg = reinterpret_cast<int32_t*>(smraw + size_t(W) * 4 + size_t(m) * 8);
+  uint32_t* mask = reinterpret_cast<uint32_t*>(smraw + size_t(W) * 4 + size_t(m) * 16);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
   const int32_t* Inew = I + int64_t(slot) * k;
   const float* Vnew = V + int64_t(slot) * k;
+  const int stride = ACC ? 2 * m : m;
   __shared__ int s_next;
   for (int t = blockIdx.x; t < n_slabs;) {  // t: position in the hand-out order
     const int s = order[t];
+    const int base = s * W;
     __syncthreads();
     if (tid == 0) s_next = int(gridDim.x) + atomicAdd(ctr, 1);
-    float4* xs4 = reinterpret_cast<float4*>(xs);
-    for (int i = tid; i < (W >> 2); i += blockDim.x) xs4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (ACC) {
+      const int n = int(min(int64_t(W), d - base));
+      for (int i = tid; i < W; i += blockDim.x) xs[i] = i < n ? e[int64_t(base) + i] : 0.f;
+      for (int i = tid; i < (W >> 5); i += blockDim.x) mask[i] = 0u;
+    } else {
+      float4* xs4 = reinterpret_cast<float4*>(xs);
+      for (int i = tid; i < (W >> 2); i += blockDim.x) xs4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
     for (int r = tid; r < m; r += blockDim.x) {
       seg[r] = offs[int64_t(s) * m + r];
       seg[m + r] = offs[int64_t(s + 1) * m + r];
     }
     __syncthreads();
-    const int base = s * W;
     {
-      const int b = seg[slot], e = seg[m + slot];
-      for (int j = b + tid; j < e; j += blockDim.x) xs[Inew[j] - base] = Vnew[j];
+      const int b = seg[slot], e2 = seg[m + slot];
+      for (int j = b + tid; j < e2; j += blockDim.x) {
+        const int i = Inew[j] - base;
+        xs[i] = Vnew[j];
+        if (ACC) atomicOr(&mask[i >> 5], 1u << (i & 31));
+      }
     }
     __syncthreads();
-    double* out = slab_part + int64_t(s) * m;
+    double* out = slab_part + int64_t(s) * stride;
     for (int r = warp; r < m; r += nwarps) {
-      const int b = seg[r], e = seg[m + r];
-      if (b >= e) {
-        if (lane == 0) out[r] = 0.0;
+      const int b = seg[r], e2 = seg[m + r];
+      if (b >= e2) {
+        if (lane == 0) {
+          out[r] = 0.0;
+          if (ACC) out[m + r] = 0.0;
+        }
         continue;
       }
       const int32_t* Ir = I + int64_t(r) * k;
@@ -230,12 +251,24 @@ __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_sp_rows(
         const int rn = r + nwarps;
         prefetch_segment(I + int64_t(rn) * k, V + int64_t(rn) * k, seg[rn], seg[m + rn], lane);
       }
-      double acc = 0.0, acc2 = 0.0;
+      double acc = 0.0, acc2 = 0.0;  // COMPRESSED: two chains of <row, c>; ACC: <row, c>, <row, xi>
+      auto use = [&](int q, int i, float v) {
+        const double p = double(v) * double(xs[i]);
+        if (ACC) {
+          const bool in_c = (mask[i >> 5] >> (i & 31)) & 1u;
+          acc += in_c ? p : 0.0;
+          acc2 += in_c ? 0.0 : p;
+        } else if (q & 1) {
+          acc2 += p;
+        } else {
+          acc += p;
+        }
+      };
       // kDepth groups of 32 entries per pass: all loads of a pass are issued before the
       // first use.  Full passes need no bounds checks and address every load by a
       // constant offset from one pointer pair.
       int j0 = b + lane;
-      for (; j0 + 32 * (kDepth - 1) < e - 31 + lane; j0 += 32 * kDepth) {
+      for (; j0 + 32 * (kDepth - 1) < e2 - 31 + lane; j0 += 32 * kDepth) {
         const int32_t* pi = Ir + j0;
         const float* pv = Vr + j0;
         int ii[kDepth];
@@ -246,30 +279,32 @@ __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_sp_rows(
           vv[q] = __ldcs(pv + 32 * q);
         }
 #pragma unroll
-        for (int q = 0; q < kDepth; q += 2) {
-          acc += double(vv[q]) * double(xs[ii[q] - base]);
-          acc2 += double(vv[q + 1]) * double(xs[ii[q + 1] - base]);
-        }
+        for (int q = 0; q < kDepth; ++q) use(q, ii[q] - base, vv[q]);
       }
-      if (j0 - lane < e) {  // the last, partial pass (warp-uniform condition)
+      if (j0 - lane < e2) {  // the last, partial pass (warp-uniform condition)
         int ii[kDepth];
         float vv[kDepth];
 #pragma unroll
         for (int q = 0; q < kDepth; ++q) {
           const int j = j0 + 32 * q;
-          const bool on = j < e;
+          const bool on = j < e2;
           ii[q] = on ? __ldcs(Ir + j) : base;
           vv[q] = on ? __ldcs(Vr + j) : 0.f;
         }
 #pragma unroll
-        for (int q = 0; q < kDepth; q += 2) {
-          acc += double(vv[q]) * double(xs[ii[q] - base]);
-          acc2 += double(vv[q + 1]) * double(xs[ii[q + 1] - base]);
-        }
+        for (int q = 0; q < kDepth; ++q) use(q, ii[q] - base, vv[q]);
       }
-      acc += acc2;
-      acc = warp_sum(acc);
-      if (lane == 0) out[r] = acc;
+      if (ACC) {
+        acc = warp_sum(acc);
+        acc2 = warp_sum(acc2);
+        if (lane == 0) {
+          out[r] = acc;
+          out[m + r] = acc2;
+        }
+      } else {
+        acc = warp_sum(acc + acc2);
+        if (lane == 0) out[r] = acc;
+      }
     }
     t = s_next;
   }
@@ -296,28 +331,40 @@ __global__ void __launch_bounds__(128) k_sp_reduce(const double* __restrict__ sl
 
 // delta[r] = sum of the per-block partials in block order; S row/column `slot` := delta
 // (Section 2.1: S_{i,:} = S_{:,i} = G g); aprime = delta with entry `slot` cleared.
+// With rhs != null (x = a_t): `partial` rows are 2 m long, the second half sums to
+// q = G xi_t, and rhs = m e_slot - q / lambda (the right-hand side of the weights, see
+// efcp_mxm.cuh).
 __global__ void __launch_bounds__(128) k_sp_finish(const double* __restrict__ partial, int nparts,
                                                     int m, int slot, double* __restrict__ delta,
                                                     double* __restrict__ S,
-                                                    double* __restrict__ aprime) {
+                                                    double* __restrict__ aprime,
+                                                    double* __restrict__ rhs, double lambda) {
   const int r = blockIdx.x * blockDim.x + threadIdx.x;
   if (r >= m) return;
+  const int stride = rhs ? 2 * m : m;
   double s = 0.0;
-  for (int p = 0; p < nparts; ++p) s += partial[int64_t(p) * m + r];
+  for (int p = 0; p < nparts; ++p) s += partial[int64_t(p) * stride + r];
   delta[r] = s;
   S[int64_t(slot) * m + r] = s;
   S[int64_t(r) * m + slot] = s;
   aprime[r] = r == slot ? 0.0 : s;
+  if (rhs) {
+    double q = 0.0;
+    for (int p = 0; p < nparts; ++p) q += partial[int64_t(p) * stride + m + r];
+    rhs[r] = (r == slot ? double(m) : 0.0) - q / lambda;
+  }
 }
 
 // Linear combination of the window rows, u = sum_r w_r row_r, one slab at a time in a
 // shared-memory accumulator (Eq. (2) in the form that has no x/lambda term, see
 // efcp_mxm.cuh).  Every element of u is written exactly once.
-template <bool VEC>
+// With ACC (x = a_t) the accumulator of a slab starts from xi_t / lambda instead of zero.
+template <bool VEC, bool ACC>
 __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_lcg(
     const int32_t* __restrict__ I, const float* __restrict__ V, const int32_t* __restrict__ offs,
     int64_t k, int m, int W, int n_slabs, const float* __restrict__ wf, float* __restrict__ u,
-    int64_t d, int* ctr, const int32_t* __restrict__ order) {
+    int64_t d, int* ctr, const int32_t* __restrict__ order, const float* __restrict__ xi,
+    float inv_lambda) {
   extern __shared__ __align__(16) unsigned char smraw[];
   float* acc = reinterpret_cast<float*>(smraw);
   float* wc = reinterpret_cast<float*>(smraw + size_t(W) * 4);
@@ -335,8 +382,12 @@ __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_lcg(
       seg[r] = offs[int64_t(s) * m + r];
       seg[m + r] = offs[int64_t(s + 1) * m + r];
     }
-    __syncthreads();
     const int base = s * W;
+    if (ACC) {
+      const int n = int(min(int64_t(W), d - base));
+      for (int i = tid; i < n; i += blockDim.x) acc[i] = xi[int64_t(base) + i] * inv_lambda;
+    }
+    __syncthreads();
     for (int r = warp; r < m; r += nwarps) {
       const int b = seg[r], e = seg[m + r];
       const float c = wc[r];

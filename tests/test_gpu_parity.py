@@ -121,6 +121,29 @@ def test_ragged_sizes(d, m, k, steps):
     run_parity(d, m, k, 1e-3, grads, check_rows="all", gram_every=3, allow_amplified=(k == 1))
 
 
+# ---- right-hand side = the whole accumulator a_t (EFCP_RHS_ACCUMULATOR)
+def test_accumulator_rhs_c1_full_run():
+    w = gradgen.C1
+    run_parity(w.d, w.m, w.k, w.lam, stream_grads(w, w.steps), flags=ref.RHS_ACCUMULATOR,
+               check_rows="all", gram_every=7)
+
+
+@pytest.mark.parametrize("d,m,k,steps,lam", [
+    (5, 2, 2, 6, 1e-3), (2049, 4, 100, 9, 1e-3), (100_003, 16, 1000, 40, 1e-4),
+    (1_000_001, 8, 33_333, 12, 1e-6), (3_000_017, 8, 30_000, 11, 1e-4),
+])
+def test_accumulator_rhs_ragged_sizes(d, m, k, steps, lam):
+    rng = np.random.default_rng(d + 1)
+    scale = np.exp(rng.standard_normal(d))
+    grads = ((scale * rng.standard_normal(d)).astype(np.float32) for _ in range(steps))
+    run_parity(d, m, k, lam, grads, flags=ref.RHS_ACCUMULATOR, check_rows="all", gram_every=3)
+
+
+def test_accumulator_rhs_c2_shape_first_steps():
+    w = gradgen.C2
+    run_parity(w.d, w.m, w.k, w.lam, stream_grads(w, 12), flags=ref.RHS_ACCUMULATOR)
+
+
 def test_heavy_ties():
     # values from a small set: most of the selection is decided by the index rule
     d, m, k = 50_000, 4, 777
