@@ -104,6 +104,17 @@ int efcp_get_row(efcp_ctx* ctx, int32_t slot, int32_t* host_idx, float* host_val
 int efcp_get_gram(efcp_ctx* ctx, double* host_S);
 int efcp_get_weights(efcp_ctx* ctx, double* host_w);
 
+/*
+ * efcp_get_window - device pointers to the ring buffer G = (I, V) for read-only
+ * inspection by code running on the same device (tests compute residuals of the defining
+ * linear system at sizes where copying the window to the host is too slow).  Waits for the
+ * device first.  *dev_I and *dev_V point to m rows of k entries each (row = ring slot);
+ * inside a row the entries of each slab of coordinates are contiguous but not sorted
+ * (Section 3.1 leaves the order inside a row open; efcp_get_row returns ascending order).
+ * The pointers stay valid until efcp_destroy; writing through them is undefined.
+ */
+int efcp_get_window(efcp_ctx* ctx, const int32_t** dev_I, const float** dev_V);
+
 /* Number of completed efcp_step calls on this handle (-1 for a NULL handle). */
 int64_t efcp_step_count(efcp_ctx* ctx);
 

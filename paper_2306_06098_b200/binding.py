@@ -35,6 +35,7 @@ EXPORTS = {
     "efcp_get_row": ([_vp, _i32, _vp, _vp], C.c_int),
     "efcp_get_gram": ([_vp, _vp], C.c_int),
     "efcp_get_weights": ([_vp, _vp], C.c_int),
+    "efcp_get_window": ([_vp, _vp, _vp], C.c_int),
     "efcp_step_count": ([_vp], _i64),
     "efcp_status": ([_vp], C.c_int),
     "efcp_last_cuda_error": ([_vp], C.c_int),
@@ -181,6 +182,23 @@ class Efcp:
         out = np.empty((self.m, self.m), np.float64)
         self._check(_lib.efcp_get_gram(self._h, _np_ptr(out)), "efcp_get_gram")
         return out
+
+    def window(self):
+        """(I, V): the ring buffer as read-only (m, k) device tensors that alias the library's
+        memory (efcp_get_window); valid until close()."""
+        pi, pv = _vp(), _vp()
+        self._check(_lib.efcp_get_window(self._h, C.cast(C.byref(pi), _vp),
+                                         C.cast(C.byref(pv), _vp)), "efcp_get_window")
+
+        class _Alias:
+            def __init__(self, ptr, typestr, shape):
+                self.__cuda_array_interface__ = {"shape": shape, "typestr": typestr,
+                                                 "data": (ptr, False), "version": 3}
+
+        shape = (self.m, self.k)
+        dev = torch.device("cuda", torch.cuda.current_device())
+        return (torch.as_tensor(_Alias(pi.value, "<i4", shape), device=dev),
+                torch.as_tensor(_Alias(pv.value, "<f4", shape), device=dev))
 
     def weights(self) -> np.ndarray:
         out = np.empty(self.m, np.float64)

@@ -503,6 +503,15 @@ int efcp_get_weights(efcp_ctx* ctx, double* host_w) {
   return rc;
 }
 
+int efcp_get_window(efcp_ctx* ctx, const int32_t** dev_I, const float** dev_V) {
+  if (!ctx || !dev_I || !dev_V) return EFCP_EINVAL;
+  const int rc = sync_status(ctx);
+  if (rc == EFCP_ECUDA) return rc;
+  *dev_I = ctx->I;
+  *dev_V = ctx->V;
+  return rc;
+}
+
 int64_t efcp_step_count(efcp_ctx* ctx) { return ctx ? ctx->t : -1; }
 
 int efcp_status(efcp_ctx* ctx) {

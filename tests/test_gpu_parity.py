@@ -239,3 +239,79 @@ def test_host_entry_point_matches_device_entry_point():
         b.step_host(gh, uh)
         assert np.array_equal(bits(a.error()), bits(b.error()))
         assert rel_l2(uh.numpy(), ud.cpu().numpy()) <= 1e-5
+
+
+# ---- full size, in the launch configuration the benchmark times
+def _device_stream(w, device="cuda"):
+    return gradgen.GradStream.for_workload(w, device)
+
+
+@pytest.mark.parametrize("w", [gradgen.C3, gradgen.C4], ids=lambda w: w.name)
+def test_full_size_first_steps_match_oracle(w):
+    """Element by element at the full dimension: every coordinate of the error buffer, the
+    inserted rows and the update, for the first steps of the workload's own gradient stream
+    (generated on the device, the same bytes copied to the oracle)."""
+    B = _binding()
+    steps = 3
+    gs = _device_stream(w)
+    gpu = B.Efcp(w.d, w.m, w.k, w.lam)
+    cpu = ref.RefEFCP(w.d, w.m, w.k, w.lam)
+    u_dev = torch.empty(w.d, dtype=torch.float32, device="cuda")
+    for t in range(steps):
+        g_dev = gs.next()
+        gpu.step(g_dev, u_dev)
+        u_ref = cpu.step(g_dev.cpu().numpy())
+        assert gpu.status() == 0
+        assert np.array_equal(bits(gpu.error()), bits(cpu.error())), f"error buffer differs, step {t}"
+        gi, gv = gpu.row(t)
+        ci, cv = cpu.row(t)
+        assert np.array_equal(gi, ci) and np.array_equal(bits(gv), bits(cv)), f"row differs, step {t}"
+        assert rel_l2(u_dev.cpu().numpy(), u_ref) <= U_TOL
+    gpu.close()
+    cpu.close()
+
+
+@pytest.mark.parametrize("w,flags", [(gradgen.C3, 0), (gradgen.C4, 0), (gradgen.C3, 1)],
+                         ids=["c3", "c4", "c3_rhs_accumulator"])
+def test_full_size_steady_state_residual(w, flags):
+    """With the window completely filled (the state the benchmark times) the update must
+    solve the defining system (lambda I + (1/m) G^T G) u = x up to the rounding of u itself:
+    | F u - x | <= 4 * 2^-24 * | lambda |u| + (1/m) |G|^T (|G| |u|) |, evaluated in fp64 on
+    the device from the library's own window.  A wrong coefficient, a dropped row or a
+    misplaced entry breaks this by orders of magnitude."""
+    B = _binding()
+    gs = _device_stream(w)
+    gpu = B.Efcp(w.d, w.m, w.k, w.lam, flags)
+    u = torch.empty(w.d, dtype=torch.float32, device="cuda")
+    for t in range(w.m + 3):
+        g = gs.next()
+        gpu.step(g, u)
+    assert gpu.status() == 0
+    del gs
+    lam = float(np.float32(w.lam))
+    I, V = gpu.window()
+    slot = (gpu.step_count - 1) % w.m
+    ud = u.double()
+    x = torch.zeros(w.d, dtype=torch.float64, device="cuda")
+    if flags:
+        x += torch.from_numpy(gpu.error()).cuda().double()
+    x.index_add_(0, I[slot].long(), V[slot].double())
+    Gu = torch.empty(w.m, dtype=torch.float64, device="cuda")
+    Gau = torch.empty(w.m, dtype=torch.float64, device="cuda")
+    for r in range(w.m):
+        idx, val = I[r].long(), V[r].double()
+        ur = ud[idx]
+        Gu[r] = (val * ur).sum()
+        Gau[r] = (val.abs() * ur.abs()).sum()
+    Fu = lam * ud
+    bound = lam * ud.abs()
+    for r in range(w.m):
+        idx, val = I[r].long(), V[r].double()
+        Fu.index_add_(0, idx, val * (Gu[r] / w.m))
+        bound.index_add_(0, idx, val.abs() * (Gau[r] / w.m))
+    res = float((Fu - x).norm())
+    lim = 4 * 2.0 ** -24 * float(bound.norm())
+    print(f"{w.name}: |Fu - x| = {res:.3e}, rounding bound {lim:.3e}, |x| = {float(x.norm()):.3e}")
+    assert res <= lim
+    assert gpu.last_residual() < 1e-9
+    gpu.close()
