@@ -178,6 +178,41 @@ __device__ __forceinline__ void prefetch_segment(const int32_t* Ir, const float*
   if (half * 128 < bytes) asm volatile("prefetch.global.L2 [%0];" ::"l"(p + half * 128));
 }
 
+// The last pass over a segment: N groups of 32 entries (1 <= N <= kDepth), only the last of
+// which can be incomplete.  `use(q, index, value)` consumes entry q of this lane; a lane
+// without an entry in the last group gets (pad, 0).
+template <int N, typename F>
+__device__ __forceinline__ void tail_pass(const int32_t* pi, const float* pv, bool last_on, int pad,
+                                          F&& use) {
+  int ii[N];
+  float vv[N];
+#pragma unroll
+  for (int q = 0; q < N - 1; ++q) {
+    ii[q] = __ldcs(pi + 32 * q);
+    vv[q] = __ldcs(pv + 32 * q);
+  }
+  ii[N - 1] = last_on ? __ldcs(pi + 32 * (N - 1)) : pad;
+  vv[N - 1] = last_on ? __ldcs(pv + 32 * (N - 1)) : 0.f;
+#pragma unroll
+  for (int q = 0; q < N; ++q) use(q, ii[q], vv[q]);
+}
+
+template <typename F>
+__device__ __forceinline__ void tail_dispatch(int groups, const int32_t* pi, const float* pv,
+                                              bool last_on, int pad, F&& use) {
+  static_assert(kDepth <= 16, "tail_dispatch covers up to 16 groups");
+  switch (groups) {
+#define EFCP_TAIL_CASE(N) \
+    case N: if (N <= kDepth) tail_pass<(N <= kDepth ? N : 1)>(pi, pv, last_on, pad, use); break;
+    EFCP_TAIL_CASE(1) EFCP_TAIL_CASE(2) EFCP_TAIL_CASE(3) EFCP_TAIL_CASE(4)
+    EFCP_TAIL_CASE(5) EFCP_TAIL_CASE(6) EFCP_TAIL_CASE(7) EFCP_TAIL_CASE(8)
+    EFCP_TAIL_CASE(9) EFCP_TAIL_CASE(10) EFCP_TAIL_CASE(11) EFCP_TAIL_CASE(12)
+    EFCP_TAIL_CASE(13) EFCP_TAIL_CASE(14) EFCP_TAIL_CASE(15) EFCP_TAIL_CASE(16)
+#undef EFCP_TAIL_CASE
+    default: break;
+  }
+}
+
 // Slab scheduling of the two slab kernels.  Slabs differ in weight (the kept entries
 // cluster where the gradient is large), so blocks do not take a fixed share: block b starts
 // with slab b and then draws the next unprocessed slab from a counter in global memory
@@ -281,18 +316,11 @@ __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_sp_rows(
 #pragma unroll
         for (int q = 0; q < kDepth; ++q) use(q, ii[q] - base, vv[q]);
       }
-      if (j0 - lane < e2) {  // the last, partial pass (warp-uniform condition)
-        int ii[kDepth];
-        float vv[kDepth];
-#pragma unroll
-        for (int q = 0; q < kDepth; ++q) {
-          const int j = j0 + 32 * q;
-          const bool on = j < e2;
-          ii[q] = on ? __ldcs(Ir + j) : base;
-          vv[q] = on ? __ldcs(Vr + j) : 0.f;
-        }
-#pragma unroll
-        for (int q = 0; q < kDepth; ++q) use(q, ii[q] - base, vv[q]);
+      const int rem = e2 - (j0 - lane);  // entries left for the last pass (warp-uniform)
+      if (rem > 0) {
+        const int groups = (rem + 31) >> 5;
+        tail_dispatch(groups, Ir + j0, Vr + j0, j0 + 32 * (groups - 1) < e2, base,
+                      [&](int q, int i, float v) { use(q, i - base, v); });
       }
       if (ACC) {
         acc = warp_sum(acc);
@@ -414,19 +442,13 @@ __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_lcg(
 #pragma unroll
         for (int q = 0; q < kDepth; ++q) atomicAdd(&acc[ii[q]], c * vv[q]);
       }
-      if (j0 - lane < e) {  // the last, partial pass
-        int ii[kDepth];
-        float vv[kDepth];
-#pragma unroll
-        for (int q = 0; q < kDepth; ++q) {
-          const int j = j0 + 32 * q;
-          const bool on = j < e;
-          ii[q] = on ? __ldcs(Ir + j) - base : -1;
-          vv[q] = on ? __ldcs(Vr + j) : 0.f;
-        }
-#pragma unroll
-        for (int q = 0; q < kDepth; ++q)
-          if (ii[q] >= 0) atomicAdd(&acc[ii[q]], c * vv[q]);
+      const int rem = e - (j0 - lane);  // entries left for the last pass (warp-uniform)
+      if (rem > 0) {
+        const int groups = (rem + 31) >> 5;
+        tail_dispatch(groups, Ir + j0, Vr + j0, j0 + 32 * (groups - 1) < e, -1,
+                      [&](int, int i, float v) {
+                        if (i >= 0) atomicAdd(&acc[i - base], c * v);
+                      });
       }
     }
     __syncthreads();
