@@ -84,8 +84,10 @@ int pick_slab_width(int64_t d, int m, int num_sms) {
   }
   // shared memory: W*4 + 16*m must stay under the 227 KB per-block limit
   while (slab_smem_bytes(W, m) * kSlabBlocksPerSM > 200 * 1024 && W > 1024) W >>= 1;
-  // enough slabs to give every SM several
-  while (W > 1024 && (d + W - 1) / W < int64_t(4) * num_sms) W >>= 1;
+  // at least one slab per SM (the slab kernels run one block per SM and rebalance by
+  // drawing slabs from a counter), but no slab narrower than 2048 coordinates: below that
+  // a row's segment is a handful of entries and the per-row bookkeeping dominates
+  while (W > 2048 && (d + W - 1) / W < int64_t(num_sms)) W >>= 1;
   return W;
 }
 
