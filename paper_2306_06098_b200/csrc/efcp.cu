@@ -77,13 +77,13 @@ struct Sizes {
 };
 
 int pick_slab_width(int64_t d, int m, int num_sms) {
-  int W = (32768 / kSlabBlocksPerSM) & ~31;
+  int W = (40960 / kSlabBlocksPerSM) & ~31;  // 160 KB of the 227 KB a block may use
   if (const char* env = getenv("EFCP_SLAB_W")) {
     const int v = atoi(env);
     if (v >= 256 && v <= 49152 && (v & 31) == 0) return v;
   }
   // shared memory: W*4 + 16*m must stay under the 227 KB per-block limit
-  while (slab_smem_bytes(W, m) * kSlabBlocksPerSM > 200 * 1024 && W > 1024) W >>= 1;
+  while (slab_smem_bytes(W, m) * kSlabBlocksPerSM > 220 * 1024 && W > 1024) W >>= 1;
   // at least one slab per SM (the slab kernels run one block per SM and rebalance by
   // drawing slabs from a counter), but no slab narrower than 2048 coordinates: below that
   // a row's segment is a handful of entries and the per-row bookkeeping dominates
@@ -369,7 +369,7 @@ int efcp_step(efcp_ctx* ctx, const float* grad, float* update, void* stream_) {
   EFCP_LAUNCHED();
   k_slab_order<<<1, 1024, 0, st>>>(ctx->colsum, ctx->n_slabs, ctx->order);
   EFCP_LAUNCHED();
-  k_layout_row<<<(ctx->n_slabs + kLayoutWarps - 1) / kLayoutWarps, kLayoutWarps * 32, 0, st>>>(
+  k_layout_row<<<ctx->n_slabs, kLayoutWarps * 32, 0, st>>>(
       ctx->sel_idx, ctx->sel_val, k, ctx->W, ctx->n_slabs, m, slot, ctx->offs, row_idx, row_val,
       ctx->slab_ctr);
   EFCP_LAUNCHED();

@@ -214,11 +214,12 @@ __global__ void __launch_bounds__(kChunkThreads, 8) k_compact_cand(
   __syncthreads();
   const uint32_t b1 = sc->b1;
   for (int ch = blockIdx.x; ch < n_chunks; ch += gridDim.x) {
-    if (off[ch + 1] == off[ch]) continue;  // no candidate in this chunk (block-uniform)
     const int64_t base = int64_t(ch) * kChunk + threadIdx.x * kPerThread;
     float v[kPerThread];
     bool ok[kPerThread];
+    const int off0 = off[ch], off1 = off[ch + 1];  // in flight together with the chunk
     load_chunk8(a, base, d, v, ok);
+    if (off1 == off0) continue;  // no candidate in this chunk (block-uniform)
     int c = 0;
 #pragma unroll
     for (int q = 0; q < kPerThread; ++q) {
@@ -226,7 +227,7 @@ __global__ void __launch_bounds__(kChunkThreads, 8) k_compact_cand(
       c += ok[q] ? 1 : 0;
     }
     int total;
-    int pos = off[ch] + block_excl_scan<int>(c, &total, sm);
+    int pos = off0 + block_excl_scan<int>(c, &total, sm);
 #pragma unroll
     for (int q = 0; q < kPerThread; ++q) {
       if (ok[q]) {
@@ -340,6 +341,11 @@ __global__ void __launch_bounds__(kChunkThreads) k_write_sel(
     float v[kPerThread];
     bool ok[kPerThread];
     load_chunk8(cand_val, base, n, v, ok);
+    int32_t ci[kPerThread];  // fetched now, with the values, not after the scans
+#pragma unroll
+    for (int q = 0; q < kPerThread; ++q) ci[q] = ok[q] ? cand_idx[base + q] : 0;
+    const int eq_before_chunk = pre_eq[c];
+    const int gt_before_chunk = off_gt[c];
     bool is_eq[kPerThread];
     int my_eq = 0;
 #pragma unroll
@@ -350,7 +356,6 @@ __global__ void __launch_bounds__(kChunkThreads) k_write_sel(
       my_eq += is_eq[q] ? 1 : 0;
     }
     int tot;
-    const int eq_before_chunk = pre_eq[c];
     int eq_rank = eq_before_chunk + block_excl_scan<int>(my_eq, &tot, sm);
     int my_sel = 0;
 #pragma unroll
@@ -361,12 +366,12 @@ __global__ void __launch_bounds__(kChunkThreads) k_write_sel(
       }
       my_sel += ok[q] ? 1 : 0;
     }
-    int64_t pos = int64_t(off_gt[c]) + min(eq_before_chunk, n_eq) +
+    int64_t pos = int64_t(gt_before_chunk) + min(eq_before_chunk, n_eq) +
                   block_excl_scan<int>(my_sel, &tot, sm);
 #pragma unroll
     for (int q = 0; q < kPerThread; ++q) {
       if (ok[q] && pos < k_total) {
-        const int32_t j = cand_idx[base + q];
+        const int32_t j = ci[q];
         row_idx[pos] = j;
         row_val[pos] = v[q];
         e[j] = 0.0f;

@@ -30,7 +30,7 @@
 namespace efcp {
 
 constexpr int kLayoutChunk = 512;   // entries permuted together (a multiple of 32)
-constexpr int kLayoutWarps = 8;     // warps (= slabs) per block of k_layout_row
+constexpr int kLayoutWarps = 4;     // warps per block of k_layout_row (one block per slab)
 
 // offs[s][slot] for the new row from its ascending index list: entry `pos` starts every
 // slab between its predecessor's slab (exclusive) and its own (inclusive); the last entry
@@ -84,7 +84,7 @@ __global__ void __launch_bounds__(1024) k_slab_order(const int64_t* __restrict__
 
 // Insert of the new row: from the ascending (index, value) list of the selection,
 //   ring slot <- the row, every segment [offs[s][slot], offs[s+1][slot]) in the
-//   bank-interleaved order described above.  One warp per slab.
+//   bank-interleaved order described above.  One block per slab, one warp per chunk.
 __global__ void __launch_bounds__(kLayoutWarps * 32) k_layout_row(
     const int32_t* __restrict__ src_idx, const float* __restrict__ src_val, int64_t k, int W,
     int n_slabs, int m, int slot, const int32_t* __restrict__ offs,
@@ -95,15 +95,14 @@ __global__ void __launch_bounds__(kLayoutWarps * 32) k_layout_row(
   __shared__ int s_cnt[kLayoutWarps][32];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   if (blockIdx.x == 0 && threadIdx.x < 2) slab_ctr[threadIdx.x] = 0;  // SP and LCG work counters
-  const int s = blockIdx.x * kLayoutWarps + warp;
-  if (s >= n_slabs) return;
+  const int s = blockIdx.x;  // one block per slab, its warps share the chunks of the segment
   const int seg_b = offs[int64_t(s) * m + slot];
   const int seg_e = offs[int64_t(s + 1) * m + slot];
   int32_t* ci = s_idx[warp];
   float* cv = s_val[warp];
   uint16_t* cq = s_q[warp];
   int* cnt = s_cnt[warp];
-  for (int c0 = seg_b; c0 < seg_e; c0 += kLayoutChunk) {
+  for (int c0 = seg_b + warp * kLayoutChunk; c0 < seg_e; c0 += kLayoutWarps * kLayoutChunk) {
     const int n = min(kLayoutChunk, seg_e - c0);
     cnt[lane] = 0;
     __syncwarp();
