@@ -34,14 +34,8 @@ UNIT = "steps/s"
 # DRAM traffic per launch of the dominant kernels from the ncu captures summarised under
 # profiles/ (dram__bytes_read.sum + dram__bytes_write.sum), keyed by workload; None until
 # a capture of that workload exists.  Scaled from a smaller capture where noted there.
-# Captured on c3_resnet18 (same kernels, window 0.96 GB); DRAM traffic is proportional to
-# the bytes streamed, so the C4 figures are the C3 traffic / C3 algorithmic bytes ratio
-# (k_sp_rows 1.009, k_lcg 0.981) times the C4 algorithmic bytes per launch.
-NCU_TRAFFIC_BYTES = {
-    "c3_resnet18": {"sp": 966_382_848, "lcg": 984_982_528},
-    "c4_bert_base": {"sp": int(1.0092 * 8 * 1024 * 1_094_822),
-                     "lcg": int(0.9807 * (8 * 1024 * 1_094_822 + 4 * 109_482_240))},
-}
+# None until captured again: the kernels have changed since the last capture.
+NCU_TRAFFIC_BYTES = {}
 
 
 def load_peak():
@@ -292,11 +286,16 @@ def main():
                "h2d_bytes_per_step": 4 * w.d, "d2h_bytes_per_step": 4 * w.d,
                "steps": args.e2e_steps}
 
-    # roofline of the dominant kernel (HBM bound): algorithmic bytes per launch / time
+    # roofline of the dominant kernel (HBM bound): bytes the kernel has to move per launch /
+    # its time.  The kernels stream a window entry as a 16-bit slab-relative index and an
+    # fp32 value: 6 bytes.  (Counted with the 32-bit indices of the (I, V) format, 8 bytes
+    # per entry, the same times give the `as_int32_indices` figures.)
+    # x = a_t adds one read of xi to SP and one to LCG.
     peak, peak_src = load_peak()
-    # x = a_t adds one read of xi to SP and one to LCG
-    alg = {"sp": 8 * w.m * w.k + (4 * w.d if acc else 0),
-           "lcg": 8 * w.m * w.k + 4 * w.d + (4 * w.d if acc else 0)}
+    mk = w.m * w.k
+    xi_read = 4 * w.d if acc else 0
+    alg = {"sp": 6 * mk + xi_read, "lcg": 6 * mk + 4 * w.d + xi_read}
+    alg8 = {"sp": 8 * mk + xi_read, "lcg": 8 * mk + 4 * w.d + xi_read}
     kern = max(("sp", "lcg"), key=lambda s: stages[s])
     avg_ms = stages[kern] / max(n_rec, 1)
     achieved = alg[kern] / (avg_ms * 1e-3) / 1e9
@@ -304,9 +303,14 @@ def main():
                 "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": None if acc else NCU_TRAFFIC_BYTES.get(w.name, {}).get(kern),
                 "peak_source": peak_src, "algorithmic_bytes_per_launch": alg[kern],
-                "avg_launch_ms": avg_ms}
-    step_bytes = 16 * w.m * w.k + 16 * w.d + 8 * w.k + (8 * w.d if acc else 0)
+                "avg_launch_ms": avg_ms,
+                "as_int32_indices": {"algorithmic_bytes_per_launch": alg8[kern],
+                                     "achieved": alg8[kern] / (avg_ms * 1e-3) / 1e9,
+                                     "frac": alg8[kern] / (avg_ms * 1e-3) / 1e9 / peak}}
+    step_bytes = 12 * mk + 16 * w.d + 10 * w.k + 2 * xi_read
     step_gbs = step_bytes / (ms_per_step * 1e-3) / 1e9
+    step_bytes8 = 16 * mk + 16 * w.d + 8 * w.k + 2 * xi_read
+    step_gbs8 = step_bytes8 / (ms_per_step * 1e-3) / 1e9
     stage_ms = {s: stages[s] / max(n_rec, 1) for s in stages}
 
     cpu_baseline = None
@@ -331,7 +335,11 @@ def main():
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
             "roofline": roofline,
             "step_hbm": {"algorithmic_bytes_per_step": step_bytes, "achieved_gbs": step_gbs,
-                         "frac_of_peak": step_gbs / peak, "frac_of_8tbs": step_gbs / 8000.0},
+                         "frac_of_peak": step_gbs / peak, "frac_of_8tbs": step_gbs / 8000.0,
+                         "as_int32_indices": {"algorithmic_bytes_per_step": step_bytes8,
+                                              "achieved_gbs": step_gbs8,
+                                              "frac_of_peak": step_gbs8 / peak,
+                                              "frac_of_8tbs": step_gbs8 / 8000.0}},
             "stage_ms": stage_ms,
             "cpu_baseline": cpu_baseline,
         }

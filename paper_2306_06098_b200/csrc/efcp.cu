@@ -35,6 +35,7 @@ struct efcp_ctx {
   // state
   float* e = nullptr;
   int32_t* I = nullptr;
+  uint16_t* R = nullptr;  // slab-relative copy of I, the index stream SP and LCG read
   float* V = nullptr;
   int32_t* offs = nullptr;
   double* S = nullptr;
@@ -102,7 +103,7 @@ Sizes compute_sizes(int64_t d, int32_t m, int64_t k, int num_sms) {
   z.grid_slab = z.n_slabs < num_sms * kSlabBlocksPerSM ? z.n_slabs : num_sms * kSlabBlocksPerSM;
   int64_t b = 0;
   b += align256(d * 4);                                   // e
-  b += 2 * align256(int64_t(m) * k * 4);                  // I, V
+  b += 2 * align256(int64_t(m) * k * 4) + align256(int64_t(m) * k * 2);  // I, V, R
   b += align256(int64_t(z.n_slabs + 1) * m * 4);          // offs
   b += 2 * align256(int64_t(m) * m * 8);                  // S, B
   b += align256((kBins1 + kBins2 + kBins3) * 4);          // hist
@@ -243,6 +244,7 @@ int efcp_create_ex(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float lambda
   const int64_t mk = int64_t(m) * k;
   if ((rc = dev_alloc(ctx, &ctx->e, d * 4))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->I, mk * 4))) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->R, mk * 2))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->V, mk * 4))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->offs, int64_t(z.n_slabs + 1) * m * 4))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->S, int64_t(m) * m * 8))) return fail(rc);
@@ -269,6 +271,7 @@ int efcp_create_ex(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float lambda
   bool ok = true;
   ok &= cudaMemset(ctx->e, 0, size_t(d) * 4) == cudaSuccess;
   ok &= cudaMemset(ctx->V, 0, size_t(mk) * 4) == cudaSuccess;
+  ok &= cudaMemset(ctx->R, 0, size_t(mk) * 2) == cudaSuccess;
   ok &= cudaMemset(ctx->offs, 0, size_t(z.n_slabs + 1) * m * 4) == cudaSuccess;
   ok &= cudaMemset(ctx->S, 0, size_t(m) * m * 8) == cudaSuccess;
   ok &= cudaMemset(ctx->colsum, 0, size_t(z.n_slabs + 1) * 8) == cudaSuccess;
@@ -370,7 +373,8 @@ int efcp_step(efcp_ctx* ctx, const float* grad, float* update, void* stream_) {
   k_slab_order<<<1, 1024, 0, st>>>(ctx->colsum, ctx->n_slabs, ctx->order);
   EFCP_LAUNCHED();
   k_layout_row<<<ctx->n_slabs, kLayoutWarps * 32, 0, st>>>(
-      ctx->sel_idx, ctx->sel_val, k, ctx->W, ctx->n_slabs, m, slot, ctx->offs, row_idx, row_val,
+      ctx->sel_idx, ctx->sel_val, k, ctx->W, ctx->n_slabs, m, slot, ctx->offs, row_idx,
+      ctx->R + int64_t(slot) * k, row_val,
       ctx->slab_ctr);
   EFCP_LAUNCHED();
   // scalar products with the new row, Gram row/column
@@ -381,11 +385,11 @@ int efcp_step(efcp_ctx* ctx, const float* grad, float* update, void* stream_) {
   prof_mark(ctx, 1, st);
   if (acc_mode)
     k_sp_rows<true><<<ctx->grid_slab, kSlabThreads, smem, st>>>(
-        ctx->I, ctx->V, ctx->offs, k, m, ctx->W, ctx->n_slabs, slot, ctx->slab_part, ctx->slab_ctr,
+        ctx->R, ctx->V, ctx->offs, k, m, ctx->W, ctx->n_slabs, slot, ctx->slab_part, ctx->slab_ctr,
         ctx->order, ctx->e, d);
   else
     k_sp_rows<false><<<ctx->grid_slab, kSlabThreads, smem, st>>>(
-        ctx->I, ctx->V, ctx->offs, k, m, ctx->W, ctx->n_slabs, slot, ctx->slab_part, ctx->slab_ctr,
+        ctx->R, ctx->V, ctx->offs, k, m, ctx->W, ctx->n_slabs, slot, ctx->slab_part, ctx->slab_ctr,
         ctx->order, ctx->e, d);
   EFCP_LAUNCHED();
   prof_mark(ctx, 2, st);
@@ -423,7 +427,7 @@ int efcp_step(efcp_ctx* ctx, const float* grad, float* update, void* stream_) {
   const float inv_lambda = 1.0f / ctx->lambda;
 #define EFCP_LCG_LAUNCH(VEC, ACC)                                                              \
   k_lcg<VEC, ACC><<<ctx->grid_slab, kSlabThreads, smem, st>>>(                                 \
-      ctx->I, ctx->V, ctx->offs, k, m, ctx->W, ctx->n_slabs, ctx->wf, update, d,               \
+      ctx->R, ctx->V, ctx->offs, k, m, ctx->W, ctx->n_slabs, ctx->wf, update, d,               \
       ctx->slab_ctr + 1, ctx->order, ctx->e, inv_lambda)
   if (acc_mode) {
     if (uvec) EFCP_LCG_LAUNCH(true, true); else EFCP_LCG_LAUNCH(false, true);

@@ -15,6 +15,12 @@
 // construction) with a small table written when a row is inserted, so Top-k can stay
 // global.
 //
+// Indices as the kernels read them.  Inside slab s an index is s * W plus an offset below
+// W <= 65536, and a segment lies in one slab, so next to I the window keeps R (uint16,
+// m x k, same positions): the slab-relative offsets.  SP and LCG stream R and V, 6 bytes per
+// entry instead of 8, and use the offset directly as the shared-memory address; I is only
+// written (at insert) and read back by efcp_get_row / efcp_get_window.
+//
 // Order inside a segment.  A warp takes 32 consecutive entries of a segment at a time and
 // uses their indices as shared-memory addresses, so what matters for speed is how many
 // of the 32 fall into the same bank (index mod 32).  Neither primitive depends on the
@@ -88,7 +94,8 @@ __global__ void __launch_bounds__(1024) k_slab_order(const int64_t* __restrict__
 __global__ void __launch_bounds__(kLayoutWarps * 32) k_layout_row(
     const int32_t* __restrict__ src_idx, const float* __restrict__ src_val, int64_t k, int W,
     int n_slabs, int m, int slot, const int32_t* __restrict__ offs,
-    int32_t* __restrict__ dst_idx, float* __restrict__ dst_val, int* __restrict__ slab_ctr) {
+    int32_t* __restrict__ dst_idx, uint16_t* __restrict__ dst_rel, float* __restrict__ dst_val,
+    int* __restrict__ slab_ctr) {
   __shared__ int32_t s_idx[kLayoutWarps][kLayoutChunk];
   __shared__ float s_val[kLayoutWarps][kLayoutChunk];
   __shared__ uint16_t s_q[kLayoutWarps][kLayoutChunk];
@@ -138,6 +145,7 @@ __global__ void __launch_bounds__(kLayoutWarps * 32) k_layout_row(
           pos += min(c, q) + ((bb < bank && c > q) ? 1 : 0);
         }
         dst_idx[c0 + pos] = idx;
+        dst_rel[c0 + pos] = uint16_t(idx - s * W);
         dst_val[c0 + pos] = cv[a];
       }
     }
@@ -168,12 +176,12 @@ constexpr int kDepth = EFCP_DEPTH;               // groups of 32 entries a warp 
 // lines of each; longer segments are covered at their start only).  Issued one row ahead
 // of use, so that the loads of the next row find their data in L2 instead of waiting for
 // HBM.
-__device__ __forceinline__ void prefetch_segment(const int32_t* Ir, const float* Vr, int b, int e,
+__device__ __forceinline__ void prefetch_segment(const uint16_t* Rr, const float* Vr, int b, int e,
                                                  int lane) {
   const int half = lane & 15;
-  const char* p = (lane < 16) ? reinterpret_cast<const char*>(Ir + b)
+  const char* p = (lane < 16) ? reinterpret_cast<const char*>(Rr + b)
                               : reinterpret_cast<const char*>(Vr + b);
-  const int bytes = (e - b) * 4;
+  const int bytes = (e - b) * (lane < 16 ? 2 : 4);
   if (half * 128 < bytes) asm volatile("prefetch.global.L2 [%0];" ::"l"(p + half * 128));
 }
 
@@ -181,7 +189,7 @@ __device__ __forceinline__ void prefetch_segment(const int32_t* Ir, const float*
 // which can be incomplete.  `use(q, index, value)` consumes entry q of this lane; a lane
 // without an entry in the last group gets (pad, 0).
 template <int N, typename F>
-__device__ __forceinline__ void tail_pass(const int32_t* pi, const float* pv, bool last_on, int pad,
+__device__ __forceinline__ void tail_pass(const uint16_t* pi, const float* pv, bool last_on, int pad,
                                           F&& use) {
   int ii[N];
   float vv[N];
@@ -190,14 +198,14 @@ __device__ __forceinline__ void tail_pass(const int32_t* pi, const float* pv, bo
     ii[q] = __ldcs(pi + 32 * q);
     vv[q] = __ldcs(pv + 32 * q);
   }
-  ii[N - 1] = last_on ? __ldcs(pi + 32 * (N - 1)) : pad;
+  ii[N - 1] = last_on ? int(__ldcs(pi + 32 * (N - 1))) : pad;
   vv[N - 1] = last_on ? __ldcs(pv + 32 * (N - 1)) : 0.f;
 #pragma unroll
   for (int q = 0; q < N; ++q) use(q, ii[q], vv[q]);
 }
 
 template <typename F>
-__device__ __forceinline__ void tail_dispatch(int groups, const int32_t* pi, const float* pv,
+__device__ __forceinline__ void tail_dispatch(int groups, const uint16_t* pi, const float* pv,
                                               bool last_on, int pad, F&& use) {
   static_assert(kDepth <= 16, "tail_dispatch covers up to 16 groups");
   switch (groups) {
@@ -230,7 +238,7 @@ __device__ __forceinline__ void tail_dispatch(int groups, const int32_t* pi, con
 // serves both sums.  `stride` is the row length of slab_part (m or 2 m).
 template <bool ACC>
 __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_sp_rows(
-    const int32_t* __restrict__ I, const float* __restrict__ V, const int32_t* __restrict__ offs,
+    const uint16_t* __restrict__ R, const float* __restrict__ V, const int32_t* __restrict__ offs,
     int64_t k, int m, int W, int n_slabs, int slot, double* __restrict__ slab_part, int* ctr,
     const int32_t* __restrict__ order, const float* __restrict__ e, int64_t d) {
   extern __shared__ __align__(16) unsigned char smraw[];
@@ -238,7 +246,7 @@ __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_sp_rows(
   int32_t* seg = reinterpret_cast<int32_t*>(smraw + size_t(W) * 4 + size_t(m) * 8);
   uint32_t* mask = reinterpret_cast<uint32_t*>(smraw + size_t(W) * 4 + size_t(m) * 16);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
-  const int32_t* Inew = I + int64_t(slot) * k;
+  const uint16_t* Rnew = R + int64_t(slot) * k;
   const float* Vnew = V + int64_t(slot) * k;
   const int stride = ACC ? 2 * m : m;
   __shared__ int s_next;
@@ -263,7 +271,7 @@ __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_sp_rows(
     {
       const int b = seg[slot], e2 = seg[m + slot];
       for (int j = b + tid; j < e2; j += blockDim.x) {
-        const int i = Inew[j] - base;
+        const int i = Rnew[j];
         xs[i] = Vnew[j];
         if (ACC) atomicOr(&mask[i >> 5], 1u << (i & 31));
       }
@@ -279,11 +287,11 @@ __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_sp_rows(
         }
         continue;
       }
-      const int32_t* Ir = I + int64_t(r) * k;
+      const uint16_t* Rr = R + int64_t(r) * k;
       const float* Vr = V + int64_t(r) * k;
       if (r + nwarps < m) {
         const int rn = r + nwarps;
-        prefetch_segment(I + int64_t(rn) * k, V + int64_t(rn) * k, seg[rn], seg[m + rn], lane);
+        prefetch_segment(R + int64_t(rn) * k, V + int64_t(rn) * k, seg[rn], seg[m + rn], lane);
       }
       double acc = 0.0, acc2 = 0.0;  // COMPRESSED: two chains of <row, c>; ACC: <row, c>, <row, xi>
       auto use = [&](int q, int i, float v) {
@@ -303,7 +311,7 @@ __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_sp_rows(
       // constant offset from one pointer pair.
       int j0 = b + lane;
       for (; j0 + 32 * (kDepth - 1) < e2 - 31 + lane; j0 += 32 * kDepth) {
-        const int32_t* pi = Ir + j0;
+        const uint16_t* pi = Rr + j0;
         const float* pv = Vr + j0;
         int ii[kDepth];
         float vv[kDepth];
@@ -313,13 +321,13 @@ __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_sp_rows(
           vv[q] = __ldcs(pv + 32 * q);
         }
 #pragma unroll
-        for (int q = 0; q < kDepth; ++q) use(q, ii[q] - base, vv[q]);
+        for (int q = 0; q < kDepth; ++q) use(q, ii[q], vv[q]);
       }
       const int rem = e2 - (j0 - lane);  // entries left for the last pass (warp-uniform)
       if (rem > 0) {
         const int groups = (rem + 31) >> 5;
-        tail_dispatch(groups, Ir + j0, Vr + j0, j0 + 32 * (groups - 1) < e2, base,
-                      [&](int q, int i, float v) { use(q, i - base, v); });
+        tail_dispatch(groups, Rr + j0, Vr + j0, j0 + 32 * (groups - 1) < e2, 0,
+                      [&](int q, int i, float v) { use(q, i, v); });
       }
       if (ACC) {
         acc = warp_sum(acc);
@@ -388,7 +396,7 @@ __global__ void __launch_bounds__(128) k_sp_finish(const double* __restrict__ pa
 // With ACC (x = a_t) the accumulator of a slab starts from xi_t / lambda instead of zero.
 template <bool VEC, bool ACC>
 __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_lcg(
-    const int32_t* __restrict__ I, const float* __restrict__ V, const int32_t* __restrict__ offs,
+    const uint16_t* __restrict__ R, const float* __restrict__ V, const int32_t* __restrict__ offs,
     int64_t k, int m, int W, int n_slabs, const float* __restrict__ wf, float* __restrict__ u,
     int64_t d, int* ctr, const int32_t* __restrict__ order, const float* __restrict__ xi,
     float inv_lambda) {
@@ -419,15 +427,15 @@ __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_lcg(
       const int b = seg[r], e = seg[m + r];
       const float c = wc[r];
       if (b >= e || c == 0.f) continue;
-      const int32_t* Ir = I + int64_t(r) * k;
+      const uint16_t* Rr = R + int64_t(r) * k;
       const float* Vr = V + int64_t(r) * k;
       if (r + nwarps < m) {
         const int rn = r + nwarps;
-        prefetch_segment(I + int64_t(rn) * k, V + int64_t(rn) * k, seg[rn], seg[m + rn], lane);
+        prefetch_segment(R + int64_t(rn) * k, V + int64_t(rn) * k, seg[rn], seg[m + rn], lane);
       }
       int j0 = b + lane;
       for (; j0 + 32 * (kDepth - 1) < e - 31 + lane; j0 += 32 * kDepth) {  // full passes
-        const int32_t* pi = Ir + j0;
+        const uint16_t* pi = Rr + j0;
         const float* pv = Vr + j0;
         int ii[kDepth];
         float vv[kDepth];
@@ -437,16 +445,14 @@ __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_lcg(
           vv[q] = __ldcs(pv + 32 * q);
         }
 #pragma unroll
-        for (int q = 0; q < kDepth; ++q) ii[q] -= base;
-#pragma unroll
         for (int q = 0; q < kDepth; ++q) atomicAdd(&acc[ii[q]], c * vv[q]);
       }
       const int rem = e - (j0 - lane);  // entries left for the last pass (warp-uniform)
       if (rem > 0) {
         const int groups = (rem + 31) >> 5;
-        tail_dispatch(groups, Ir + j0, Vr + j0, j0 + 32 * (groups - 1) < e, -1,
+        tail_dispatch(groups, Rr + j0, Vr + j0, j0 + 32 * (groups - 1) < e, -1,
                       [&](int, int i, float v) {
-                        if (i >= 0) atomicAdd(&acc[i - base], c * v);
+                        if (i >= 0) atomicAdd(&acc[i], c * v);
                       });
       }
     }
