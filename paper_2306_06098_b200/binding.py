@@ -107,9 +107,9 @@ class Efcp:
         self._h = h
 
     def close(self):
-        if self._h:
+        if self._h and _lib is not None:  # (_lib is gone while the interpreter shuts down)
             _lib.efcp_destroy(self._h)
-            self._h = None
+        self._h = None
 
     def __del__(self):
         self.close()

@@ -45,6 +45,9 @@ struct efcp_ctx {
   int32_t* chunk_off = nullptr;
   int32_t* cand_idx = nullptr;
   float* cand_val = nullptr;
+  uint16_t* bk_off = nullptr;  // speculative candidate buckets, one of kChunk entries per chunk
+  float* bk_val = nullptr;
+  bool spec = true;            // EFCP_NO_SPEC=1 forces the two-pass candidate path
   int32_t* sel_idx = nullptr;  // the selection of the current step, ascending (k entries)
   float* sel_val = nullptr;
   int32_t* sel_gt = nullptr;
@@ -109,6 +112,7 @@ Sizes compute_sizes(int64_t d, int32_t m, int64_t k, int num_sms) {
   b += align256((kBins1 + kBins2 + kBins3) * 4);          // hist
   b += 3 * align256(int64_t(z.n_chunks + 1) * 4);         // chunk_off, sel_gt, sel_eq
   b += 2 * align256(d * 4);                               // cand_idx, cand_val
+  b += align256(int64_t(z.n_chunks) * kChunk * 2) + align256(int64_t(z.n_chunks) * kChunk * 4);  // buckets
   b += 2 * align256(k * 4);                               // sel_idx, sel_val
   b += align256(sizeof(Scalars));
   b += align256(int64_t(z.n_slabs) * m * 8);              // slab_part
@@ -255,6 +259,9 @@ int efcp_create_ex(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float lambda
   if ((rc = dev_alloc(ctx, &ctx->sel_eq, int64_t(z.n_chunks + 1) * 4))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->cand_idx, d * 4))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->cand_val, d * 4))) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->bk_off, int64_t(z.n_chunks) * kChunk * 2))) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->bk_val, int64_t(z.n_chunks) * kChunk * 4))) return fail(rc);
+  if (const char* env = getenv("EFCP_NO_SPEC")) ctx->spec = atoi(env) == 0;
   if ((rc = dev_alloc(ctx, &ctx->sel_idx, k * 4))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->sel_val, k * 4))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->sc, sizeof(Scalars)))) return fail(rc);
@@ -330,17 +337,23 @@ int efcp_step(efcp_ctx* ctx, const float* grad, float* update, void* stream_) {
   const double mlambda = double(m) * double(ctx->lambda);
 
   prof_mark(ctx, 0, st);
-  // a = xi + g, digit-1 histogram
-  const int ef_grid = ctx->num_sms * 2;
-  if ((reinterpret_cast<uintptr_t>(grad) & 15) == 0)
-    k_ef_hist1<true><<<ef_grid, 512, 0, st>>>(ctx->e, grad, d, hist1, ctx->sc);
-  else
-    k_ef_hist1<false><<<ef_grid, 512, 0, st>>>(ctx->e, grad, d, hist1, ctx->sc);
-  EFCP_LAUNCHED();
-  k_pick<kBins1, 1><<<1, 1024, 0, st>>>(hist1, ctx->sc, uint32_t(k));
-  EFCP_LAUNCHED();
-  // candidates: everything at or above the threshold bin, in index order
+  // a = xi + g, digit-1 histogram, speculative candidate buckets
   const int chunk_grid = ctx->n_chunks < ctx->num_sms * 8 ? ctx->n_chunks : ctx->num_sms * 8;
+  const int spec = ctx->spec ? 1 : 0;
+  if ((reinterpret_cast<uintptr_t>(grad) & 15) == 0)
+    k_ef_spec<true><<<chunk_grid, kChunkThreads, 0, st>>>(ctx->e, grad, d, hist1, ctx->sc,
+                                                          ctx->chunk_off, ctx->bk_off,
+                                                          ctx->bk_val, ctx->n_chunks, spec);
+  else
+    k_ef_spec<false><<<chunk_grid, kChunkThreads, 0, st>>>(ctx->e, grad, d, hist1, ctx->sc,
+                                                           ctx->chunk_off, ctx->bk_off,
+                                                           ctx->bk_val, ctx->n_chunks, spec);
+  EFCP_LAUNCHED();
+  const uint32_t spec_limit = uint32_t(std::min<int64_t>(d, 3 * k + 65536));
+  k_pick<kBins1, 1><<<1, 1024, 0, st>>>(hist1, ctx->sc, uint32_t(k), spec, spec_limit);
+  EFCP_LAUNCHED();
+  // candidates: everything at or above the threshold bin, in index order.  The two-pass
+  // kernels return at once when the buckets are good, k_compact_buckets when they are not.
   k_count_chunks<<<chunk_grid, kChunkThreads, 0, st>>>(ctx->e, d, ctx->sc, ctx->chunk_off,
                                                        ctx->n_chunks);
   EFCP_LAUNCHED();
@@ -349,6 +362,10 @@ int efcp_step(efcp_ctx* ctx, const float* grad, float* update, void* stream_) {
   k_compact_cand<<<chunk_grid, kChunkThreads, 0, st>>>(ctx->e, d, ctx->sc, ctx->chunk_off,
                                                        ctx->cand_idx, ctx->cand_val, hist2,
                                                        ctx->n_chunks);
+  EFCP_LAUNCHED();
+  k_compact_buckets<<<ctx->num_sms * 4, 256, 0, st>>>(ctx->bk_off, ctx->bk_val, ctx->sc,
+                                                      ctx->chunk_off, ctx->cand_idx,
+                                                      ctx->cand_val, hist2, ctx->n_chunks);
   EFCP_LAUNCHED();
   k_pick<kBins2, 2><<<1, 1024, 0, st>>>(hist2, ctx->sc, uint32_t(k));
   EFCP_LAUNCHED();

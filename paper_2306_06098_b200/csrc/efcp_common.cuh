@@ -33,6 +33,8 @@ struct Scalars {
   int32_t n_cand;   // candidates: entries whose digit 1 is >= b1
   int32_t n_sel;    // entries selected (must equal k)
   uint32_t status;  // sticky status bits
+  uint32_t have_prev;  // b1 holds the previous step's threshold bin
+  uint32_t spec_ok;    // this step's speculative candidate buckets cover the threshold bin
   uint32_t pad;
   double schur;     // Schur complement of the bordered inverse (1 / B_ii)
   double beta;      // B_ii before the row was replaced

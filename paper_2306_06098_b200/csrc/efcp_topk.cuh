@@ -14,7 +14,133 @@
 
 namespace efcp {
 
-// a = xi + g in place over xi, histogram of digit 1, non-finite detection.
+// Speculation.  The threshold of the selection moves little from one step to the next, so
+// the kernel that forms a = xi + g already sets aside, chunk by chunk, every entry at or
+// above a guessed bin of digit 1 (the previous step's threshold bin minus kSpecMargin).
+// k_pick<.., 1> then knows the true threshold bin: if the guess was not above it and did
+// not let in too many entries, the candidate list is compacted from these buckets and the
+// accumulator is not read again; otherwise (first step, threshold fell by more than the
+// margin) the two-pass path below, k_count_chunks + k_compact_cand, runs as before.  Both
+// routes give the same exact selection.
+constexpr int kSpecMargin = 1;
+
+__device__ __forceinline__ uint32_t spec_guess(const Scalars* sc, int enable) {
+  if (!enable || !sc->have_prev) return uint32_t(kBins1);  // nothing is set aside
+  return sc->b1 > uint32_t(kSpecMargin) ? sc->b1 - kSpecMargin : 0u;
+}
+
+// a = xi + g in place over xi, histogram of digit 1, non-finite detection, and the
+// speculative buckets: chunk ch gets its entries with digit 1 >= guess, in index order, at
+// bk_off / bk_val [ch * kChunk ...) (offset inside the chunk, value); cnt[ch] = how many.
+template <bool VEC>
+__global__ void __launch_bounds__(kChunkThreads, 8) k_ef_spec(
+    float* __restrict__ e, const float* __restrict__ g, int64_t d, uint32_t* __restrict__ hist1,
+    Scalars* sc, int32_t* __restrict__ cnt, uint16_t* __restrict__ bk_off,
+    float* __restrict__ bk_val, int n_chunks, int enable) {
+  __shared__ uint32_t h[kBins1];
+  __shared__ int sm[33];
+  for (int i = threadIdx.x; i < kBins1; i += blockDim.x) h[i] = 0u;
+  const uint32_t guess = spec_guess(sc, enable);
+  __syncthreads();
+  bool bad = false;
+  for (int ch = blockIdx.x; ch < n_chunks; ch += gridDim.x) {
+    const int local = threadIdx.x * kPerThread;
+    const int64_t base = int64_t(ch) * kChunk + local;
+    float a[kPerThread];
+    bool ok[kPerThread];
+    if (VEC && base + kPerThread <= d) {
+      float4* e4 = reinterpret_cast<float4*>(e + base);
+      const float4* g4 = reinterpret_cast<const float4*>(g + base);
+      float4 e0 = e4[0], e1 = e4[1];
+      const float4 g0 = __ldcs(g4), g1 = __ldcs(g4 + 1);
+      e0.x = __fadd_rn(e0.x, g0.x); e0.y = __fadd_rn(e0.y, g0.y);
+      e0.z = __fadd_rn(e0.z, g0.z); e0.w = __fadd_rn(e0.w, g0.w);
+      e1.x = __fadd_rn(e1.x, g1.x); e1.y = __fadd_rn(e1.y, g1.y);
+      e1.z = __fadd_rn(e1.z, g1.z); e1.w = __fadd_rn(e1.w, g1.w);
+      e4[0] = e0; e4[1] = e1;
+      a[0] = e0.x; a[1] = e0.y; a[2] = e0.z; a[3] = e0.w;
+      a[4] = e1.x; a[5] = e1.y; a[6] = e1.z; a[7] = e1.w;
+#pragma unroll
+      for (int q = 0; q < kPerThread; ++q) ok[q] = true;
+    } else {
+#pragma unroll
+      for (int q = 0; q < kPerThread; ++q) {
+        ok[q] = base + q < d;
+        a[q] = 0.f;
+        if (ok[q]) {
+          a[q] = __fadd_rn(e[base + q], g[base + q]);
+          e[base + q] = a[q];
+        }
+      }
+    }
+    int c = 0;
+#pragma unroll
+    for (int q = 0; q < kPerThread; ++q) {
+      const uint32_t key = mag_key(a[q]);
+      if (ok[q]) {
+        atomicAdd(&h[key >> kShift1], 1u);
+        bad |= key >= 0x7F800000u;
+      }
+      ok[q] = ok[q] && (key >> kShift1) >= guess;
+      c += ok[q] ? 1 : 0;
+    }
+    int total;
+    int pos = block_excl_scan<int>(c, &total, sm);
+    if (total) {
+      uint16_t* bo = bk_off + int64_t(ch) * kChunk;
+      float* bv = bk_val + int64_t(ch) * kChunk;
+#pragma unroll
+      for (int q = 0; q < kPerThread; ++q) {
+        if (ok[q]) {
+          bo[pos] = uint16_t(local + q);
+          bv[pos] = a[q];
+          ++pos;
+        }
+      }
+    }
+    if (threadIdx.x == 0) cnt[ch] = total;
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < kBins1; i += blockDim.x) {
+    const uint32_t c = h[i];
+    if (c) atomicAdd(&hist1[i], c);
+  }
+  if (bad) atomicOr(&sc->status, kStNonFinite);
+}
+
+// The candidate list from the speculative buckets (runs only when sc->spec_ok): chunk ch's
+// entries go to cand[off[ch] ...), digit 2 of the entries inside the true threshold bin is
+// histogrammed.  One warp per chunk.
+__global__ void __launch_bounds__(256) k_compact_buckets(
+    const uint16_t* __restrict__ bk_off, const float* __restrict__ bk_val, const Scalars* sc,
+    const int32_t* __restrict__ off, int32_t* __restrict__ cand_idx, float* __restrict__ cand_val,
+    uint32_t* __restrict__ hist2, int n_chunks) {
+  if (!sc->spec_ok) return;
+  __shared__ uint32_t h[kBins2];
+  for (int i = threadIdx.x; i < kBins2; i += blockDim.x) h[i] = 0u;
+  __syncthreads();
+  const uint32_t b1 = sc->b1;
+  const int lane = threadIdx.x & 31, wpb = blockDim.x >> 5;
+  for (int ch = blockIdx.x * wpb + (threadIdx.x >> 5); ch < n_chunks; ch += gridDim.x * wpb) {
+    const int o0 = off[ch], n = off[ch + 1] - o0;
+    const uint16_t* bo = bk_off + int64_t(ch) * kChunk;
+    const float* bv = bk_val + int64_t(ch) * kChunk;
+    for (int i = lane; i < n; i += 32) {
+      const float v = bv[i];
+      cand_idx[o0 + i] = int32_t(int64_t(ch) * kChunk + bo[i]);
+      cand_val[o0 + i] = v;
+      const uint32_t key = mag_key(v);
+      if ((key >> kShift1) == b1) atomicAdd(&h[(key >> kShift2) & (kBins2 - 1)], 1u);
+    }
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < kBins2; i += blockDim.x) {
+    const uint32_t cc = h[i];
+    if (cc) atomicAdd(&hist2[i], cc);
+  }
+}
+
+// The same first pass without the buckets (kept for callers of the two-pass path only).
 template <bool VEC>
 __global__ void __launch_bounds__(512) k_ef_hist1(float* __restrict__ e,
                                                    const float* __restrict__ g, int64_t d,
@@ -72,15 +198,21 @@ __global__ void __launch_bounds__(512) k_ef_hist1(float* __restrict__ e,
 
 // Finds the threshold bin of one digit: the bin b with count(bins > b) < k_rem <=
 // count(bins >= b).  Clears the histogram for the next step.  One block of 1024.
+// At level 1, `spec` >= 0 also judges the speculation of k_ef_spec (spec = its `enable`):
+// sc->spec_ok = the guessed bin is not above the threshold bin and lets in at most
+// `spec_limit` entries.
 template <int NB, int LEVEL>
 __global__ void __launch_bounds__(1024) k_pick(uint32_t* __restrict__ hist, Scalars* sc,
-                                                uint32_t k_total) {
+                                                uint32_t k_total, int spec = -1,
+                                                uint32_t spec_limit = 0) {
   __shared__ uint32_t h[NB];
   __shared__ uint32_t sm[33];
   for (int i = threadIdx.x; i < NB; i += blockDim.x) {
     h[i] = hist[i];
     hist[i] = 0u;
   }
+  uint32_t guess = NB;
+  if (LEVEL == 1 && spec >= 0) guess = spec_guess(sc, spec);  // before b1 is overwritten
   __syncthreads();
   const uint32_t k_rem = LEVEL == 1 ? k_total : (LEVEL == 2 ? sc->k1 : sc->k2);
   constexpr int P = (NB + 1023) / 1024;
@@ -110,6 +242,20 @@ __global__ void __launch_bounds__(1024) k_pick(uint32_t* __restrict__ hist, Scal
     }
   }
   if (threadIdx.x == 0 && total < k_rem) atomicOr(&sc->status, kStCount);
+  if (LEVEL == 1 && spec >= 0) {
+    uint32_t let_in = 0;
+#pragma unroll
+    for (int p = 0; p < P; ++p) {
+      const int pos = threadIdx.x * P + p;
+      if (pos < NB && uint32_t(NB - 1 - pos) >= guess) let_in += h[NB - 1 - pos];
+    }
+    uint32_t n_spec;
+    (void)block_excl_scan<uint32_t>(let_in, &n_spec, sm);
+    if (threadIdx.x == 0) {  // after the scan's barriers every thread has written b1
+      sc->spec_ok = (guess < uint32_t(NB) && guess <= sc->b1 && n_spec <= spec_limit) ? 1u : 0u;
+      sc->have_prev = 1u;
+    }
+  }
 }
 
 __device__ __forceinline__ void load_chunk8(const float* __restrict__ a, int64_t base, int64_t n,
@@ -137,6 +283,7 @@ __global__ void __launch_bounds__(kChunkThreads) k_count_chunks(const float* __r
                                                                  int32_t* __restrict__ cnt,
                                                                  int n_chunks) {
   __shared__ int sm[33];
+  if (sc->spec_ok) return;  // the speculative buckets already hold the counts
   const uint32_t b1 = sc->b1;
   for (int ch = blockIdx.x; ch < n_chunks; ch += gridDim.x) {
     const int64_t base = int64_t(ch) * kChunk + threadIdx.x * kPerThread;
@@ -210,6 +357,7 @@ __global__ void __launch_bounds__(kChunkThreads, 8) k_compact_cand(
     int n_chunks) {
   __shared__ uint32_t h[kBins2];
   __shared__ int sm[33];
+  if (sc->spec_ok) return;  // k_compact_buckets builds the list instead
   for (int i = threadIdx.x; i < kBins2; i += blockDim.x) h[i] = 0u;
   __syncthreads();
   const uint32_t b1 = sc->b1;

@@ -315,3 +315,24 @@ def test_full_size_steady_state_residual(w, flags):
     assert res <= lim
     assert gpu.last_residual() < 1e-9
     gpu.close()
+
+
+def test_threshold_jumps_between_steps():
+    """The selection threshold of one step is the starting guess of the next; gradients whose
+    scale jumps by factors of 30 to 1000 in both directions make that guess useless, and the
+    result must not change (the exact two-pass route takes over)."""
+    d, m, k = 400_003, 8, 4000
+    rng = np.random.default_rng(21)
+    scales = [1.0, 1.0, 0.03, 0.03, 30.0, 1.0, 0.01, 10.0, 10.0, 1.0, 1.0, 1.0]
+    grads = ((s * rng.standard_normal(d)).astype(np.float32) for s in scales)
+    run_parity(d, m, k, 1e-3, grads, check_rows="all")
+
+
+def test_two_pass_route_alone(monkeypatch):
+    """EFCP_NO_SPEC=1 switches the speculative candidate buckets off: same results."""
+    monkeypatch.setenv("EFCP_NO_SPEC", "1")
+    d, m, k = 300_007, 8, 3000
+    rng = np.random.default_rng(22)
+    scale = np.exp(rng.standard_normal(d))
+    grads = ((scale * rng.standard_normal(d)).astype(np.float32) for _ in range(10))
+    run_parity(d, m, k, 1e-4, grads, check_rows="all")
