@@ -34,8 +34,14 @@ UNIT = "steps/s"
 # DRAM traffic per launch of the dominant kernels from the ncu captures summarised under
 # profiles/ (dram__bytes_read.sum + dram__bytes_write.sum), keyed by workload; None until
 # a capture of that workload exists.  Scaled from a smaller capture where noted there.
-# None until captured again: the kernels have changed since the last capture.
-NCU_TRAFFIC_BYTES = {}
+# Captured on a quarter-size copy of c4_bert_base (same slab width and segment lengths, see
+# profiles/): DRAM traffic / bytes to move was 1.106 for k_sp_rows and 1.084 for k_lcg, and it
+# is proportional to the bytes streamed, so the C4 figures are those ratios times the C4 bytes
+# per launch.
+NCU_TRAFFIC_BYTES = {
+    "c4_bert_base": {"sp": int(1.106 * 6 * 1024 * 1_094_822),
+                     "lcg": int(1.084 * (6 * 1024 * 1_094_822 + 4 * 109_482_240))},
+}
 
 
 def load_peak():
