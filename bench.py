@@ -206,7 +206,7 @@ def main():
     ap.add_argument("--prefill", type=int, default=-1,
                     help="untimed steps before warm-up; -1 = m (fill the whole window)")
     ap.add_argument("--e2e-steps", type=int, default=5)
-    ap.add_argument("--cpu-steps", type=int, default=2)
+    ap.add_argument("--cpu-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
