@@ -27,6 +27,10 @@
 //     Woodbury-Sherman-Morrison rank-one recursion of Section 2.1 as a second,
 //     independent route to the same coefficients.
 //   * linear combination of gradients: Section 2.1 "LCG" and Eq. (2).
+//   * optional bfloat16 window values: Section 3.1 "Format for V".  Reading taken (the paper
+//     only says the optimizer still converges with bfloat16 values): Compress returns the
+//     selected values rounded to bfloat16, and line 7 of Algorithm 1 is applied to that c,
+//     so the rounding residue is fed back like any other compression error.
 //
 // Precision: the state (error buffer, window) is fp32 exactly as the method
 // defines it (one IEEE round-to-nearest add per coordinate, no fused multiply
@@ -37,7 +41,8 @@
 // problems, the invariant a == e_new + dens(c) bit for bit, Top-k against a
 // full stable sort, the closed forms for m = 1 and for rows with disjoint
 // supports, the large-lambda limit, the WSM recursion against the Cholesky
-// route, k == d (dense M-FAC).  No numeric example is printed in the paper, so
+// route, k == d (dense M-FAC); the bfloat16 rounding against a library conversion
+// and hand-made tie cases.  No numeric example is printed in the paper, so
 // beyond those pins the values are "parity unpinned".
 //
 // Threads: OpenMP is used only on loops whose every output element is produced
@@ -58,6 +63,25 @@
 namespace {
 
 constexpr uint32_t kFlagRhsAccumulator = 1u;  // x = a_t instead of x = dens(c_t)
+constexpr uint32_t kFlagValuesBf16 = 2u;      // kept values are rounded to bfloat16
+
+// fp32 -> bfloat16 -> fp32, round to nearest, ties to even (the bfloat16 format of Section
+// 3.1 "Format for V": the upper 16 bits of an IEEE fp32).  NaN stays NaN.
+inline float round_to_bf16(float v) {
+  uint32_t b;
+  std::memcpy(&b, &v, 4);
+  if ((b & 0x7FFFFFFFu) > 0x7F800000u) {
+    b |= 0x00400000u;  // quiet NaN, payload truncated
+    b &= 0xFFFF0000u;
+  } else {
+    const uint32_t lsb = (b >> 16) & 1u;
+    b += 0x7FFFu + lsb;
+    b &= 0xFFFF0000u;
+  }
+  float r;
+  std::memcpy(&r, &b, 4);
+  return r;
+}
 
 inline uint32_t magnitude_key(float v) {
   uint32_t b;
@@ -153,6 +177,11 @@ void cholesky_solve(const double* L, int n, const double* b, double* y) {
 extern "C" {
 
 struct efcp_ref;  // opaque for callers
+
+// Element-wise fp32 -> bfloat16 -> fp32 (round to nearest even), for the pins.
+void efcp_ref_round_bf16(const float* in, float* out, int64_t n) {
+  for (int64_t j = 0; j < n; ++j) out[j] = round_to_bf16(in[j]);
+}
 
 // Exact Top-k of |a| (ties to the lower index), pairs in ascending index order.
 int efcp_ref_topk(const float* a, int64_t d, int64_t k, int32_t* idx, float* val) {
@@ -290,9 +319,16 @@ int efcp_ref_step(efcp_ref* h, const float* grad, float* update) {
   float* val = &o->V[size_t(i) * size_t(k)];
   topk_select(o->a.data(), d, k, o->order, idx, val);
 
-  // Algorithm 1 line 7: xi = a - c.  At a kept coordinate a - a is +0.
+  // Section 3.1 "Format for V" (optional): the window holds bfloat16 values, so c is the
+  // selection with every value rounded to bfloat16.
+  if (o->flags & kFlagValuesBf16)
+    for (int64_t r = 0; r < k; ++r) val[r] = round_to_bf16(val[r]);
+
+  // Algorithm 1 line 7: xi = a - c.  At a kept coordinate a - a is +0; with rounded values
+  // the rounding residue a - bf16(a) (exact in fp32) stays in the error buffer.
   o->e = o->a;
-  for (int64_t r = 0; r < k; ++r) o->e[size_t(idx[r])] = 0.0f;
+  for (int64_t r = 0; r < k; ++r)
+    o->e[size_t(idx[r])] = o->a[size_t(idx[r])] - val[r];
   o->t += 1;
 
   // Right-hand side x of the inverse-Fisher-vector product.

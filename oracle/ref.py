@@ -11,6 +11,7 @@ from . import build as _build
 
 RHS_COMPRESSED = 0
 RHS_ACCUMULATOR = 1
+VALUES_BF16 = 2
 
 _lib = None
 
@@ -36,6 +37,8 @@ def lib():
         L.efcp_ref_topk_fullsort.argtypes = [vp, i64, i64, vp, vp]
         L.efcp_ref_woodbury_coef.argtypes = [vp, vp, i32, f64, vp]
         L.efcp_ref_wsm_coef.argtypes = [vp, vp, i32, f64, vp]
+        L.efcp_ref_round_bf16.argtypes = [vp, vp, i64]
+        L.efcp_ref_round_bf16.restype = None
         L.efcp_ref_num_threads.argtypes = []
         _lib = L
     return _lib
@@ -58,6 +61,13 @@ def topk(a: np.ndarray, k: int, fullsort: bool = False):
     if rc != 0:
         raise ValueError(f"efcp_ref_topk rc={rc}")
     return idx, val
+
+
+def round_bf16(a: np.ndarray) -> np.ndarray:
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    out = np.empty_like(a)
+    lib().efcp_ref_round_bf16(_ptr(a), _ptr(out), a.size)
+    return out
 
 
 def woodbury_coef(S, p, lam):

@@ -22,7 +22,8 @@ def topk_by_sort(a: np.ndarray, k: int):
 class DenseSim:
     """EFCP with a dense m x d window and a brute-force d x d solve (tiny sizes only)."""
 
-    def __init__(self, d, m, k, lam, rhs_accumulator=False):
+    def __init__(self, d, m, k, lam, rhs_accumulator=False, values_bf16=False):
+        self.bf16 = values_bf16
         self.d, self.m, self.k = d, m, k
         self.lam = float(np.float32(lam))
         self.acc_mode = rhs_accumulator
@@ -34,10 +35,13 @@ class DenseSim:
         g = g.astype(np.float32)
         a = (self.e + g).astype(np.float32)
         idx, val = topk_by_sort(a, self.k)
+        if self.bf16:  # library conversion, not the oracle's bit manipulation
+            import torch
+            val = torch.from_numpy(val).to(torch.bfloat16).to(torch.float32).numpy()
         c = np.zeros(self.d, np.float32)
         c[idx] = val
         e_new = a.copy()
-        e_new[idx] = 0.0
+        e_new[idx] = a[idx] - val
         self.e = e_new
         self.G[self.t % self.m] = c.astype(np.float64)
         self.t += 1

@@ -132,6 +132,63 @@ def test_update_matches_dense_solve(d, m, k, steps, lam, acc_mode):
     assert np.allclose(o.gram(), sim.G @ sim.G.T, rtol=1e-12, atol=1e-12)
 
 
+# ------------------------------------------- bfloat16 window values (Section 3.1, "Format for V")
+def test_bf16_rounding_matches_library_conversion_and_ties_to_even():
+    import torch
+    rng = np.random.default_rng(30)
+    x = np.concatenate([
+        (rng.standard_normal(200_000) * np.exp(8 * rng.standard_normal(200_000))).astype(np.float32),
+        rng.integers(0, 2 ** 32, 200_000, dtype=np.uint64).astype(np.uint32).view(np.float32),
+        np.array([0.0, -0.0, 1.0, np.inf, -np.inf, 3.3895314e38, 1e-45, 1.17549435e-38], np.float32)])
+    x = x[~np.isnan(x)]
+    want = torch.from_numpy(x).to(torch.bfloat16).to(torch.float32).numpy()
+    got = ref.round_bf16(x)
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+    # exact ties: 1 + 2^-8 lies halfway between 1 and 1 + 2^-7 -> even mantissa (1.0);
+    # 1 + 3 * 2^-8 lies halfway between 1 + 2^-7 and 1 + 2^-6 -> 1 + 2^-6
+    ties = np.array([1 + 2.0 ** -8, 1 + 3 * 2.0 ** -8, -(1 + 2.0 ** -8)], np.float32)
+    assert ref.round_bf16(ties).tolist() == [1.0, 1 + 2.0 ** -6, -1.0]
+    assert np.isnan(ref.round_bf16(np.array([np.nan], np.float32))[0])
+    # near the largest finite value rounding goes to infinity, as the format demands
+    assert np.isinf(ref.round_bf16(np.array([3.4e38], np.float32))[0])
+
+
+def test_bf16_values_feed_the_rounding_residue_back():
+    rng = np.random.default_rng(31)
+    d, m, k = 2001, 4, 55
+    o = ref.RefEFCP(d, m, k, 1e-3, ref.VALUES_BF16)
+    e_prev = np.zeros(d, np.float32)
+    for t in range(7):
+        g = (rng.standard_normal(d) * np.exp(rng.standard_normal(d))).astype(np.float32)
+        o.step(g)
+        a = (e_prev + g).astype(np.float32)
+        idx, val = o.row(t % m)
+        want_i, want_v = topk_by_sort(a, k)       # selection is by the unrounded magnitude
+        assert np.array_equal(idx, want_i)
+        assert np.all((val.view(np.uint32) & 0xFFFF) == 0)          # representable in bfloat16
+        assert np.all(np.abs(val - want_v) <= np.abs(want_v) * 2.0 ** -8)
+        e = o.error()
+        dens = np.zeros(d, np.float32)
+        dens[idx] = val
+        assert np.array_equal((e + dens).view(np.uint32), a.view(np.uint32))  # a = xi + c, exactly
+        e_prev = e
+
+
+@pytest.mark.parametrize("d,m,k,steps,lam", [(96, 2, 17, 5, 1e-3), (200, 8, 21, 20, 1e-2)])
+def test_bf16_update_matches_dense_solve(d, m, k, steps, lam):
+    rng = np.random.default_rng(d)
+    o = ref.RefEFCP(d, m, k, lam, ref.VALUES_BF16)
+    sim = DenseSim(d, m, k, lam, values_bf16=True)
+    scale = np.exp(rng.standard_normal(d))
+    for t in range(steps):
+        g = (scale * rng.standard_normal(d)).astype(np.float32)
+        u = o.step(g)
+        want = sim.step(g)
+        assert np.array_equal(o.error().view(np.uint32), sim.e.view(np.uint32))
+        assert rel(u, want) < 2e-6, (t, rel(u, want))
+        assert rel(o.update_rowform(), want) < 2e-6
+
+
 def test_m1_closed_form():
     # m = 1: F^-1 x = x/lam - g (g.x) / (lam (m lam + g.g))
     rng = np.random.default_rng(5)
