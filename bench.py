@@ -203,6 +203,8 @@ def main():
                     % ", ".join(sorted(gradgen.WORKLOADS)))
     ap.add_argument("--rhs", default="compressed", choices=["compressed", "accumulator"],
                     help="precondition c_t (Algorithm 1, default) or the whole accumulator a_t")
+    ap.add_argument("--values", default="fp32", choices=["fp32", "bf16"],
+                    help="window value format (bf16: Section 3.1 'Format for V', not the default)")
     ap.add_argument("--prefill", type=int, default=-1,
                     help="untimed steps before warm-up; -1 = m (fill the whole window)")
     ap.add_argument("--e2e-steps", type=int, default=5)
@@ -227,8 +229,10 @@ def main():
     K, W = args.steps, args.warmup
     gs = gradgen.GradStream(w.d, w.rank, w.seed + rank, w.scale_block, w.noise, str(device))
     acc = args.rhs == "accumulator"
+    bf16 = args.values == "bf16"
     opt = binding.Efcp(w.d, w.m, w.k, w.lam,
-                       binding.RHS_ACCUMULATOR if acc else binding.RHS_COMPRESSED)
+                       (binding.RHS_ACCUMULATOR if acc else binding.RHS_COMPRESSED) |
+                       (binding.VALUES_BF16 if bf16 else 0))
     gbuf = torch.empty(w.d, dtype=torch.float32, device=device)
     ubuf = torch.empty(w.d, dtype=torch.float32, device=device)
 
@@ -300,20 +304,21 @@ def main():
     peak, peak_src = load_peak()
     mk = w.m * w.k
     xi_read = 4 * w.d if acc else 0
-    alg = {"sp": 6 * mk + xi_read, "lcg": 6 * mk + 4 * w.d + xi_read}
+    entry = 4 if bf16 else 6  # bytes streamed per window entry
+    alg = {"sp": entry * mk + xi_read, "lcg": entry * mk + 4 * w.d + xi_read}
     alg8 = {"sp": 8 * mk + xi_read, "lcg": 8 * mk + 4 * w.d + xi_read}
     kern = max(("sp", "lcg"), key=lambda s: stages[s])
     avg_ms = stages[kern] / max(n_rec, 1)
     achieved = alg[kern] / (avg_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": {"sp": "k_sp_rows", "lcg": "k_lcg"}[kern],
                 "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": None if acc else NCU_TRAFFIC_BYTES.get(w.name, {}).get(kern),
+                "traffic": None if (acc or bf16) else NCU_TRAFFIC_BYTES.get(w.name, {}).get(kern),
                 "peak_source": peak_src, "algorithmic_bytes_per_launch": alg[kern],
                 "avg_launch_ms": avg_ms,
                 "as_int32_indices": {"algorithmic_bytes_per_launch": alg8[kern],
                                      "achieved": alg8[kern] / (avg_ms * 1e-3) / 1e9,
                                      "frac": alg8[kern] / (avg_ms * 1e-3) / 1e9 / peak}}
-    step_bytes = 12 * mk + 16 * w.d + 10 * w.k + 2 * xi_read
+    step_bytes = 2 * entry * mk + 16 * w.d + 10 * w.k + 2 * xi_read
     step_gbs = step_bytes / (ms_per_step * 1e-3) / 1e9
     step_bytes8 = 16 * mk + 16 * w.d + 8 * w.k + 2 * xi_read
     step_gbs8 = step_bytes8 / (ms_per_step * 1e-3) / 1e9
@@ -334,7 +339,7 @@ def main():
             "warmup": W, "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": w.name, "d": w.d, "m": w.m, "k": w.k, "lambda": w.lam,
-                       "rhs": args.rhs, "prefill_steps": prefill,
+                       "rhs": args.rhs, "window_values": args.values, "prefill_steps": prefill,
                        "parallelism": f"replicas x{world}",
                        "l2": "inputs larger than L2 (window %.2f GB, gradient %.2f GB)" % (
                            8 * w.m * w.k / 1e9, 4 * w.d / 1e9)},

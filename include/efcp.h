@@ -44,6 +44,13 @@ typedef struct efcp_ctx efcp_ctx;
 #define EFCP_RHS_ACCUMULATOR 1u /* precondition the full accumulator a_t = xi_t + c_t
                                    (u = F^-1 a_t; costs one more read of xi in SP and LCG)  */
 
+#define EFCP_VALUES_BF16     2u /* window values in bfloat16 (Section 3.1, "Format for V"):
+                                   the kept values are rounded to bfloat16 (nearest even),
+                                   c holds the rounded values and xi = a - c keeps the
+                                   rounding residue, so a = xi + c stays exact.  SP and LCG
+                                   then read 4 bytes per window entry instead of 6.  Cannot
+                                   be combined with EFCP_RHS_ACCUMULATOR.                   */
+
 /*
  * efcp_create / efcp_create_ex - Algorithm 1 lines 1-2: set up an empty window and
  * xi_0 = 0 for dimension d, window length m, k kept entries per step (Top-k of

@@ -15,7 +15,7 @@ LIB_PATH = os.path.join(_HERE, "csrc", "libefcp.so")
 
 OK, EINVAL, ENOMEM, ECUDA, ENUMERIC, ETIMEOUT, EINTERNAL, ETOOBIG = 0, -1, -2, -3, -4, -5, -6, -7
 TOPK_STATIC_MAX_D = 1 << 20
-RHS_COMPRESSED, RHS_ACCUMULATOR = 0, 1
+RHS_COMPRESSED, RHS_ACCUMULATOR, VALUES_BF16 = 0, 1, 2
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(

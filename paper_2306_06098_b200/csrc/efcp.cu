@@ -36,6 +36,7 @@ struct efcp_ctx {
   float* e = nullptr;
   int32_t* I = nullptr;
   uint16_t* R = nullptr;  // slab-relative copy of I, the index stream SP and LCG read
+  bf16raw* V16 = nullptr; // EFCP_VALUES_BF16: the value stream SP and LCG read (V holds the same values)
   float* V = nullptr;
   int32_t* offs = nullptr;
   double* S = nullptr;
@@ -226,7 +227,8 @@ int efcp_create_ex(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float lambda
   if (!out) return EFCP_EINVAL;
   *out = nullptr;
   if (!valid_args(d, m, k) || !(lambda > 0.f) || !std::isfinite(lambda)) return EFCP_EINVAL;
-  if (flags & ~EFCP_RHS_ACCUMULATOR) return EFCP_EINVAL;
+  if (flags & ~(EFCP_RHS_ACCUMULATOR | EFCP_VALUES_BF16)) return EFCP_EINVAL;
+  if ((flags & EFCP_RHS_ACCUMULATOR) && (flags & EFCP_VALUES_BF16)) return EFCP_EINVAL;
   efcp_ctx* ctx = new (std::nothrow) efcp_ctx();
   if (!ctx) return EFCP_ENOMEM;
   int rc = EFCP_OK;
@@ -249,6 +251,10 @@ int efcp_create_ex(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float lambda
   if ((rc = dev_alloc(ctx, &ctx->e, d * 4))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->I, mk * 4))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->R, mk * 2))) return fail(rc);
+  if (flags & EFCP_VALUES_BF16) {
+    if ((rc = dev_alloc(ctx, &ctx->V16, mk * 2))) return fail(rc);
+    if (cudaMemset(ctx->V16, 0, size_t(mk) * 2) != cudaSuccess) return fail(EFCP_ECUDA);
+  }
   if ((rc = dev_alloc(ctx, &ctx->V, mk * 4))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->offs, int64_t(z.n_slabs + 1) * m * 4))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->S, int64_t(m) * m * 8))) return fail(rc);
@@ -290,12 +296,15 @@ int efcp_create_ex(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float lambda
   k_init_identity<<<ctx->num_sms * 2, 256>>>(ctx->B, m, 1.0 / (double(m) * double(lambda)));
   const size_t smem = slab_smem_bytes(z.W, m);
   const auto attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
-  ok &= cudaFuncSetAttribute(k_sp_rows<false>, attr, int(smem)) == cudaSuccess;
-  ok &= cudaFuncSetAttribute(k_sp_rows<true>, attr, int(smem)) == cudaSuccess;
-  ok &= cudaFuncSetAttribute(k_lcg<true, false>, attr, int(smem)) == cudaSuccess;
-  ok &= cudaFuncSetAttribute(k_lcg<false, false>, attr, int(smem)) == cudaSuccess;
-  ok &= cudaFuncSetAttribute(k_lcg<true, true>, attr, int(smem)) == cudaSuccess;
-  ok &= cudaFuncSetAttribute(k_lcg<false, true>, attr, int(smem)) == cudaSuccess;
+  ok &= cudaFuncSetAttribute(k_sp_rows<false, float>, attr, int(smem)) == cudaSuccess;
+  ok &= cudaFuncSetAttribute(k_sp_rows<true, float>, attr, int(smem)) == cudaSuccess;
+  ok &= cudaFuncSetAttribute(k_sp_rows<false, bf16raw>, attr, int(smem)) == cudaSuccess;
+  ok &= cudaFuncSetAttribute(k_lcg<true, false, float>, attr, int(smem)) == cudaSuccess;
+  ok &= cudaFuncSetAttribute(k_lcg<false, false, float>, attr, int(smem)) == cudaSuccess;
+  ok &= cudaFuncSetAttribute(k_lcg<true, true, float>, attr, int(smem)) == cudaSuccess;
+  ok &= cudaFuncSetAttribute(k_lcg<false, true, float>, attr, int(smem)) == cudaSuccess;
+  ok &= cudaFuncSetAttribute(k_lcg<true, false, bf16raw>, attr, int(smem)) == cudaSuccess;
+  ok &= cudaFuncSetAttribute(k_lcg<false, false, bf16raw>, attr, int(smem)) == cudaSuccess;
   ok &= cudaDeviceSynchronize() == cudaSuccess;
   if (!ok) {
     ctx->last_cuda = int(cudaGetLastError());
@@ -382,7 +391,7 @@ int efcp_step(efcp_ctx* ctx, const float* grad, float* update, void* stream_) {
   EFCP_LAUNCHED();
   k_write_sel<<<cand_grid, kChunkThreads, 0, st>>>(ctx->cand_idx, ctx->cand_val, ctx->sc,
                                                    ctx->sel_gt, ctx->sel_eq, ctx->sel_idx,
-                                                   ctx->sel_val, ctx->e, k);
+                                                   ctx->sel_val, ctx->e, k, ctx->V16 ? 1 : 0);
   EFCP_LAUNCHED();
   k_row_offsets<<<ctx->num_sms * 4, 256, 0, st>>>(ctx->sel_idx, k, ctx->W, ctx->n_slabs, m, slot,
                                                   ctx->offs, ctx->colsum);
@@ -391,7 +400,7 @@ int efcp_step(efcp_ctx* ctx, const float* grad, float* update, void* stream_) {
   EFCP_LAUNCHED();
   k_layout_row<<<ctx->n_slabs, kLayoutWarps * 32, 0, st>>>(
       ctx->sel_idx, ctx->sel_val, k, ctx->W, ctx->n_slabs, m, slot, ctx->offs, row_idx,
-      ctx->R + int64_t(slot) * k, row_val,
+      ctx->R + int64_t(slot) * k, row_val, ctx->V16 ? ctx->V16 + int64_t(slot) * k : nullptr,
       ctx->slab_ctr);
   EFCP_LAUNCHED();
   // scalar products with the new row, Gram row/column
@@ -400,14 +409,14 @@ int efcp_step(efcp_ctx* ctx, const float* grad, float* update, void* stream_) {
   double* rhs = dw + m;
   const size_t smem = slab_smem_bytes(ctx->W, m);
   prof_mark(ctx, 1, st);
-  if (acc_mode)
-    k_sp_rows<true><<<ctx->grid_slab, kSlabThreads, smem, st>>>(
-        ctx->R, ctx->V, ctx->offs, k, m, ctx->W, ctx->n_slabs, slot, ctx->slab_part, ctx->slab_ctr,
-        ctx->order, ctx->e, d);
-  else
-    k_sp_rows<false><<<ctx->grid_slab, kSlabThreads, smem, st>>>(
-        ctx->R, ctx->V, ctx->offs, k, m, ctx->W, ctx->n_slabs, slot, ctx->slab_part, ctx->slab_ctr,
-        ctx->order, ctx->e, d);
+#define EFCP_SP_LAUNCH(ACC, VT, VPTR)                                                          \
+  k_sp_rows<ACC, VT><<<ctx->grid_slab, kSlabThreads, smem, st>>>(                              \
+      ctx->R, VPTR, ctx->V, ctx->offs, k, m, ctx->W, ctx->n_slabs, slot, ctx->slab_part,       \
+      ctx->slab_ctr, ctx->order, ctx->e, d)
+  if (ctx->V16) EFCP_SP_LAUNCH(false, bf16raw, ctx->V16);
+  else if (acc_mode) EFCP_SP_LAUNCH(true, float, ctx->V);
+  else EFCP_SP_LAUNCH(false, float, ctx->V);
+#undef EFCP_SP_LAUNCH
   EFCP_LAUNCHED();
   prof_mark(ctx, 2, st);
   const int sp_parts = ctx->n_slabs < kSpParts ? ctx->n_slabs : kSpParts;
@@ -442,14 +451,19 @@ int efcp_step(efcp_ctx* ctx, const float* grad, float* update, void* stream_) {
   prof_mark(ctx, 3, st);
   const bool uvec = (reinterpret_cast<uintptr_t>(update) & 15) == 0;
   const float inv_lambda = 1.0f / ctx->lambda;
-#define EFCP_LCG_LAUNCH(VEC, ACC)                                                              \
-  k_lcg<VEC, ACC><<<ctx->grid_slab, kSlabThreads, smem, st>>>(                                 \
-      ctx->R, ctx->V, ctx->offs, k, m, ctx->W, ctx->n_slabs, ctx->wf, update, d,               \
+#define EFCP_LCG_LAUNCH(VEC, ACC, VT, VPTR)                                                    \
+  k_lcg<VEC, ACC, VT><<<ctx->grid_slab, kSlabThreads, smem, st>>>(                             \
+      ctx->R, VPTR, ctx->offs, k, m, ctx->W, ctx->n_slabs, ctx->wf, update, d,                 \
       ctx->slab_ctr + 1, ctx->order, ctx->e, inv_lambda)
-  if (acc_mode) {
-    if (uvec) EFCP_LCG_LAUNCH(true, true); else EFCP_LCG_LAUNCH(false, true);
+  if (ctx->V16) {
+    if (uvec) EFCP_LCG_LAUNCH(true, false, bf16raw, ctx->V16);
+    else EFCP_LCG_LAUNCH(false, false, bf16raw, ctx->V16);
+  } else if (acc_mode) {
+    if (uvec) EFCP_LCG_LAUNCH(true, true, float, ctx->V);
+    else EFCP_LCG_LAUNCH(false, true, float, ctx->V);
   } else {
-    if (uvec) EFCP_LCG_LAUNCH(true, false); else EFCP_LCG_LAUNCH(false, false);
+    if (uvec) EFCP_LCG_LAUNCH(true, false, float, ctx->V);
+    else EFCP_LCG_LAUNCH(false, false, float, ctx->V);
   }
 #undef EFCP_LCG_LAUNCH
   EFCP_LAUNCHED();

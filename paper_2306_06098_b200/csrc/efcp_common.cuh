@@ -43,6 +43,27 @@ struct Scalars {
 
 __device__ __forceinline__ uint32_t mag_key(float v) { return __float_as_uint(v) & 0x7FFFFFFFu; }
 
+// bfloat16 (the upper half of an IEEE fp32) as raw bits: the optional value format of the
+// window (Section 3.1, "Format for V").
+struct bf16raw {
+  uint16_t bits;
+};
+// fp32 -> bfloat16, round to nearest, ties to even; NaN stays a (quiet) NaN.
+__device__ __forceinline__ uint16_t bf16_bits_rn(float v) {
+  uint32_t b = __float_as_uint(v);
+  if ((b & 0x7FFFFFFFu) > 0x7F800000u) return uint16_t((b | 0x00400000u) >> 16);
+  b += 0x7FFFu + ((b >> 16) & 1u);
+  return uint16_t(b >> 16);
+}
+__device__ __forceinline__ float bf16_to_float(uint16_t bits) {
+  return __uint_as_float(uint32_t(bits) << 16);
+}
+// streaming load of one window value of either format
+__device__ __forceinline__ float load_value(const float* p) { return __ldcs(p); }
+__device__ __forceinline__ float load_value(const bf16raw* p) {
+  return bf16_to_float(__ldcs(reinterpret_cast<const uint16_t*>(p)));
+}
+
 // Exclusive prefix sum over the threads of a block (blockDim.x a multiple of 32,
 // at most 1024).  sm needs 33 entries.  *total receives the block sum.
 template <typename T>

@@ -472,13 +472,14 @@ __global__ void __launch_bounds__(1024) k_scan_sel(int32_t* __restrict__ cnt_gt,
   }
 }
 
-// Final ordered compaction: writes the kept (index, value) pairs into the ring slot in
-// ascending index order and sets the kept coordinates of xi to +0 (xi = a - c).
+// Final ordered compaction: writes the kept (index, value) pairs in ascending index order
+// and sets the kept coordinates of xi to a - c: +0, or with bfloat16 window values
+// (values_bf16) the rounding residue a - bf16(a).
 __global__ void __launch_bounds__(kChunkThreads) k_write_sel(
     const int32_t* __restrict__ cand_idx, const float* __restrict__ cand_val, const Scalars* sc,
     const int32_t* __restrict__ off_gt, const int32_t* __restrict__ pre_eq,
     int32_t* __restrict__ row_idx, float* __restrict__ row_val, float* __restrict__ e,
-    int64_t k_total) {
+    int64_t k_total, int values_bf16) {
   __shared__ int sm[33];
   const int n = sc->n_cand;
   const uint32_t T = sc->T;
@@ -521,8 +522,14 @@ __global__ void __launch_bounds__(kChunkThreads) k_write_sel(
       if (ok[q] && pos < k_total) {
         const int32_t j = ci[q];
         row_idx[pos] = j;
-        row_val[pos] = v[q];
-        e[j] = 0.0f;
+        if (values_bf16) {  // c holds the rounded value, the residue stays in xi (exact)
+          const float r = bf16_to_float(bf16_bits_rn(v[q]));
+          row_val[pos] = r;
+          e[j] = __fsub_rn(v[q], r);
+        } else {
+          row_val[pos] = v[q];
+          e[j] = 0.0f;
+        }
         ++pos;
       }
     }

@@ -95,7 +95,7 @@ __global__ void __launch_bounds__(kLayoutWarps * 32) k_layout_row(
     const int32_t* __restrict__ src_idx, const float* __restrict__ src_val, int64_t k, int W,
     int n_slabs, int m, int slot, const int32_t* __restrict__ offs,
     int32_t* __restrict__ dst_idx, uint16_t* __restrict__ dst_rel, float* __restrict__ dst_val,
-    int* __restrict__ slab_ctr) {
+    bf16raw* __restrict__ dst_v16, int* __restrict__ slab_ctr) {
   __shared__ int32_t s_idx[kLayoutWarps][kLayoutChunk];
   __shared__ float s_val[kLayoutWarps][kLayoutChunk];
   __shared__ uint16_t s_q[kLayoutWarps][kLayoutChunk];
@@ -147,6 +147,7 @@ __global__ void __launch_bounds__(kLayoutWarps * 32) k_layout_row(
         dst_idx[c0 + pos] = idx;
         dst_rel[c0 + pos] = uint16_t(idx - s * W);
         dst_val[c0 + pos] = cv[a];
+        if (dst_v16) dst_v16[c0 + pos].bits = bf16_bits_rn(cv[a]);  // exact: already rounded
       }
     }
     __syncwarp();
@@ -176,36 +177,37 @@ constexpr int kDepth = EFCP_DEPTH;               // groups of 32 entries a warp 
 // lines of each; longer segments are covered at their start only).  Issued one row ahead
 // of use, so that the loads of the next row find their data in L2 instead of waiting for
 // HBM.
-__device__ __forceinline__ void prefetch_segment(const uint16_t* Rr, const float* Vr, int b, int e,
+template <typename VT>
+__device__ __forceinline__ void prefetch_segment(const uint16_t* Rr, const VT* Vr, int b, int e,
                                                  int lane) {
   const int half = lane & 15;
   const char* p = (lane < 16) ? reinterpret_cast<const char*>(Rr + b)
                               : reinterpret_cast<const char*>(Vr + b);
-  const int bytes = (e - b) * (lane < 16 ? 2 : 4);
+  const int bytes = (e - b) * (lane < 16 ? 2 : int(sizeof(VT)));
   if (half * 128 < bytes) asm volatile("prefetch.global.L2 [%0];" ::"l"(p + half * 128));
 }
 
 // The last pass over a segment: N groups of 32 entries (1 <= N <= kDepth), only the last of
 // which can be incomplete.  `use(q, index, value)` consumes entry q of this lane; a lane
 // without an entry in the last group gets (pad, 0).
-template <int N, typename F>
-__device__ __forceinline__ void tail_pass(const uint16_t* pi, const float* pv, bool last_on, int pad,
+template <int N, typename VT, typename F>
+__device__ __forceinline__ void tail_pass(const uint16_t* pi, const VT* pv, bool last_on, int pad,
                                           F&& use) {
   int ii[N];
   float vv[N];
 #pragma unroll
   for (int q = 0; q < N - 1; ++q) {
     ii[q] = __ldcs(pi + 32 * q);
-    vv[q] = __ldcs(pv + 32 * q);
+    vv[q] = load_value(pv + 32 * q);
   }
   ii[N - 1] = last_on ? int(__ldcs(pi + 32 * (N - 1))) : pad;
-  vv[N - 1] = last_on ? __ldcs(pv + 32 * (N - 1)) : 0.f;
+  vv[N - 1] = last_on ? load_value(pv + 32 * (N - 1)) : 0.f;
 #pragma unroll
   for (int q = 0; q < N; ++q) use(q, ii[q], vv[q]);
 }
 
-template <typename F>
-__device__ __forceinline__ void tail_dispatch(int groups, const uint16_t* pi, const float* pv,
+template <typename VT, typename F>
+__device__ __forceinline__ void tail_dispatch(int groups, const uint16_t* pi, const VT* pv,
                                               bool last_on, int pad, F&& use) {
   static_assert(kDepth <= 16, "tail_dispatch covers up to 16 groups");
   switch (groups) {
@@ -236,9 +238,12 @@ __device__ __forceinline__ void tail_dispatch(int groups, const uint16_t* pi, co
 // shared memory holds a_t (xi_t with the kept coordinates, which are zero in xi_t, filled
 // in from c_t) and a bit mask says which coordinates belong to c_t, so that one gather
 // serves both sums.  `stride` is the row length of slab_part (m or 2 m).
-template <bool ACC>
+// VT is the format of the streamed values: float, or bf16raw (same values, half the bytes);
+// Vf is the fp32 copy, used for the new row only.
+template <bool ACC, typename VT>
 __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_sp_rows(
-    const uint16_t* __restrict__ R, const float* __restrict__ V, const int32_t* __restrict__ offs,
+    const uint16_t* __restrict__ R, const VT* __restrict__ V, const float* __restrict__ Vf,
+    const int32_t* __restrict__ offs,
     int64_t k, int m, int W, int n_slabs, int slot, double* __restrict__ slab_part, int* ctr,
     const int32_t* __restrict__ order, const float* __restrict__ e, int64_t d) {
   extern __shared__ __align__(16) unsigned char smraw[];
@@ -247,7 +252,7 @@ __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_sp_rows(
   uint32_t* mask = reinterpret_cast<uint32_t*>(smraw + size_t(W) * 4 + size_t(m) * 16);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
   const uint16_t* Rnew = R + int64_t(slot) * k;
-  const float* Vnew = V + int64_t(slot) * k;
+  const float* Vnew = Vf + int64_t(slot) * k;
   const int stride = ACC ? 2 * m : m;
   __shared__ int s_next;
   for (int t = blockIdx.x; t < n_slabs;) {  // t: position in the hand-out order
@@ -288,7 +293,7 @@ __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_sp_rows(
         continue;
       }
       const uint16_t* Rr = R + int64_t(r) * k;
-      const float* Vr = V + int64_t(r) * k;
+      const VT* Vr = V + int64_t(r) * k;
       if (r + nwarps < m) {
         const int rn = r + nwarps;
         prefetch_segment(R + int64_t(rn) * k, V + int64_t(rn) * k, seg[rn], seg[m + rn], lane);
@@ -312,13 +317,13 @@ __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_sp_rows(
       int j0 = b + lane;
       for (; j0 + 32 * (kDepth - 1) < e2 - 31 + lane; j0 += 32 * kDepth) {
         const uint16_t* pi = Rr + j0;
-        const float* pv = Vr + j0;
+        const VT* pv = Vr + j0;
         int ii[kDepth];
         float vv[kDepth];
 #pragma unroll
         for (int q = 0; q < kDepth; ++q) {
           ii[q] = __ldcs(pi + 32 * q);
-          vv[q] = __ldcs(pv + 32 * q);
+          vv[q] = load_value(pv + 32 * q);
         }
 #pragma unroll
         for (int q = 0; q < kDepth; ++q) use(q, ii[q], vv[q]);
@@ -394,9 +399,9 @@ __global__ void __launch_bounds__(128) k_sp_finish(const double* __restrict__ pa
 // shared-memory accumulator (Eq. (2) in the form that has no x/lambda term, see
 // efcp_mxm.cuh).  Every element of u is written exactly once.
 // With ACC (x = a_t) the accumulator of a slab starts from xi_t / lambda instead of zero.
-template <bool VEC, bool ACC>
+template <bool VEC, bool ACC, typename VT>
 __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_lcg(
-    const uint16_t* __restrict__ R, const float* __restrict__ V, const int32_t* __restrict__ offs,
+    const uint16_t* __restrict__ R, const VT* __restrict__ V, const int32_t* __restrict__ offs,
     int64_t k, int m, int W, int n_slabs, const float* __restrict__ wf, float* __restrict__ u,
     int64_t d, int* ctr, const int32_t* __restrict__ order, const float* __restrict__ xi,
     float inv_lambda) {
@@ -428,7 +433,7 @@ __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_lcg(
       const float c = wc[r];
       if (b >= e || c == 0.f) continue;
       const uint16_t* Rr = R + int64_t(r) * k;
-      const float* Vr = V + int64_t(r) * k;
+      const VT* Vr = V + int64_t(r) * k;
       if (r + nwarps < m) {
         const int rn = r + nwarps;
         prefetch_segment(R + int64_t(rn) * k, V + int64_t(rn) * k, seg[rn], seg[m + rn], lane);
@@ -436,13 +441,13 @@ __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_lcg(
       int j0 = b + lane;
       for (; j0 + 32 * (kDepth - 1) < e - 31 + lane; j0 += 32 * kDepth) {  // full passes
         const uint16_t* pi = Rr + j0;
-        const float* pv = Vr + j0;
+        const VT* pv = Vr + j0;
         int ii[kDepth];
         float vv[kDepth];
 #pragma unroll
         for (int q = 0; q < kDepth; ++q) {
           ii[q] = __ldcs(pi + 32 * q);
-          vv[q] = __ldcs(pv + 32 * q);
+          vv[q] = load_value(pv + 32 * q);
         }
 #pragma unroll
         for (int q = 0; q < kDepth; ++q) atomicAdd(&acc[ii[q]], c * vv[q]);

@@ -51,8 +51,9 @@ def test_strerror_and_state_bytes_need_no_device(lib):
         assert lib.efcp_state_bytes(*bad) == -1
     d, m, k = 109_482_240, 1024, 1_094_822
     b = lib.efcp_state_bytes(d, m, k)
-    # window (8mk) + error buffer (4d) are the floor; scratch stays within a few d-vectors
-    assert 8 * m * k + 4 * d <= b <= 8 * m * k + 4 * d + 16 * d + (64 << 20)
+    # window (8mk) + error buffer (4d) are the floor; on top come the 16-bit index stream
+    # (2mk) and scratch of a few d-vectors
+    assert 8 * m * k + 4 * d <= b <= 10 * m * k + 4 * d + 20 * d + (128 << 20)
 
 
 def test_null_handles_are_rejected_without_a_device(lib):

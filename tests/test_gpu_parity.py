@@ -35,7 +35,7 @@ def lincomb_amplification(cpu, u_ref):
     combination (the precision the paper's LCG kernel uses) loses this factor times the
     fp32 unit roundoff; it is ~1 for the benchmark workloads and large only when window
     rows are nearly parallel (e.g. k = 1 with a repeated coordinate)."""
-    assert cpu.flags == ref.RHS_COMPRESSED
+    assert not cpu.flags & ref.RHS_ACCUMULATOR
     w = -cpu.coef()
     w[(cpu.step_count - 1) % cpu.m] += 1.0 / np.float64(np.float32(cpu.lam))
     acc = np.zeros(cpu.d)
@@ -142,6 +142,31 @@ def test_accumulator_rhs_ragged_sizes(d, m, k, steps, lam):
 def test_accumulator_rhs_c2_shape_first_steps():
     w = gradgen.C2
     run_parity(w.d, w.m, w.k, w.lam, stream_grads(w, 12), flags=ref.RHS_ACCUMULATOR)
+
+
+# ---- bfloat16 window values (EFCP_VALUES_BF16)
+def test_bf16_values_c1_full_run():
+    w = gradgen.C1
+    run_parity(w.d, w.m, w.k, w.lam, stream_grads(w, w.steps), flags=ref.VALUES_BF16,
+               check_rows="all", gram_every=7)
+
+
+@pytest.mark.parametrize("d,m,k,steps,lam", [
+    (5, 2, 2, 6, 1e-3), (2049, 4, 100, 9, 1e-3), (100_003, 16, 1000, 40, 1e-4),
+    (1_000_001, 8, 33_333, 12, 1e-4), (3_000_017, 8, 30_000, 11, 1e-4),
+])
+def test_bf16_values_ragged_sizes(d, m, k, steps, lam):
+    rng = np.random.default_rng(d + 2)
+    scale = np.exp(rng.standard_normal(d))
+    grads = ((scale * rng.standard_normal(d)).astype(np.float32) for _ in range(steps))
+    run_parity(d, m, k, lam, grads, flags=ref.VALUES_BF16, check_rows="all", gram_every=3)
+
+
+def test_bf16_values_cannot_be_combined_with_accumulator_rhs():
+    B = _binding()
+    with pytest.raises(B.EfcpError) as ei:
+        B.Efcp(100, 2, 10, 1e-3, B.VALUES_BF16 | B.RHS_ACCUMULATOR)
+    assert ei.value.code == B.EINVAL
 
 
 def test_heavy_ties():
