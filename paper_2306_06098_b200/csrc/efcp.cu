@@ -629,7 +629,7 @@ std::mutex g_static_mu;
 unsigned char* g_static_ptr[kMaxDevices] = {};  // device address of the array, per device
 int g_static_sms[kMaxDevices] = {};
 
-// Digit-1 histogram of the magnitude keys of a (the part of k_ef_hist1 that does not
+// Digit-1 histogram of the magnitude keys of a (the part of k_ef_spec that does not
 // touch an error buffer).
 __global__ void __launch_bounds__(512) k_hist1_only(const float* __restrict__ a, int64_t d,
                                                     uint32_t* __restrict__ hist1) {

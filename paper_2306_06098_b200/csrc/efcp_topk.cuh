@@ -140,62 +140,6 @@ __global__ void __launch_bounds__(256) k_compact_buckets(
   }
 }
 
-// The same first pass without the buckets (kept for callers of the two-pass path only).
-template <bool VEC>
-__global__ void __launch_bounds__(512) k_ef_hist1(float* __restrict__ e,
-                                                   const float* __restrict__ g, int64_t d,
-                                                   uint32_t* __restrict__ hist1, Scalars* sc) {
-  __shared__ uint32_t h[kBins1];
-  for (int i = threadIdx.x; i < kBins1; i += blockDim.x) h[i] = 0u;
-  __syncthreads();
-  bool bad = false;
-  const int64_t tid = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
-  const int64_t nth = int64_t(gridDim.x) * blockDim.x;
-  auto tally = [&](float a) {
-    const uint32_t key = mag_key(a);
-    atomicAdd(&h[key >> kShift1], 1u);
-    bad |= key >= 0x7F800000u;
-  };
-  int64_t scalar_from = 0;
-  if (VEC) {
-    const int64_t nv = d >> 2;
-    float4* e4 = reinterpret_cast<float4*>(e);
-    const float4* g4 = reinterpret_cast<const float4*>(g);
-    int64_t v = tid;
-    for (; v + nth < nv; v += 2 * nth) {
-      float4 e0 = e4[v], e1 = e4[v + nth];
-      const float4 g0 = __ldcs(g4 + v), g1 = __ldcs(g4 + v + nth);
-      e0.x = __fadd_rn(e0.x, g0.x); e0.y = __fadd_rn(e0.y, g0.y);
-      e0.z = __fadd_rn(e0.z, g0.z); e0.w = __fadd_rn(e0.w, g0.w);
-      e1.x = __fadd_rn(e1.x, g1.x); e1.y = __fadd_rn(e1.y, g1.y);
-      e1.z = __fadd_rn(e1.z, g1.z); e1.w = __fadd_rn(e1.w, g1.w);
-      e4[v] = e0; e4[v + nth] = e1;
-      tally(e0.x); tally(e0.y); tally(e0.z); tally(e0.w);
-      tally(e1.x); tally(e1.y); tally(e1.z); tally(e1.w);
-    }
-    for (; v < nv; v += nth) {
-      float4 e0 = e4[v];
-      const float4 g0 = __ldcs(g4 + v);
-      e0.x = __fadd_rn(e0.x, g0.x); e0.y = __fadd_rn(e0.y, g0.y);
-      e0.z = __fadd_rn(e0.z, g0.z); e0.w = __fadd_rn(e0.w, g0.w);
-      e4[v] = e0;
-      tally(e0.x); tally(e0.y); tally(e0.z); tally(e0.w);
-    }
-    scalar_from = nv << 2;
-  }
-  for (int64_t j = scalar_from + tid; j < d; j += nth) {
-    const float a = __fadd_rn(e[j], g[j]);
-    e[j] = a;
-    tally(a);
-  }
-  __syncthreads();
-  for (int i = threadIdx.x; i < kBins1; i += blockDim.x) {
-    const uint32_t c = h[i];
-    if (c) atomicAdd(&hist1[i], c);
-  }
-  if (bad) atomicOr(&sc->status, kStNonFinite);
-}
-
 // Finds the threshold bin of one digit: the bin b with count(bins > b) < k_rem <=
 // count(bins >= b).  Clears the histogram for the next step.  One block of 1024.
 // At level 1, `spec` >= 0 also judges the speculation of k_ef_spec (spec = its `enable`):

@@ -168,7 +168,7 @@ __host__ __device__ inline size_t slab_smem_bytes(int W, int m) {
 #endif
 constexpr int kSlabBlocksPerSM = EFCP_SLAB_BLOCKS;  // resident blocks of a slab kernel per SM
 #ifndef EFCP_DEPTH
-#define EFCP_DEPTH 8
+#define EFCP_DEPTH 12
 #endif
 constexpr int kSlabThreads = EFCP_SLAB_THREADS;  // threads of a slab-kernel block (one block per SM)
 constexpr int kDepth = EFCP_DEPTH;               // groups of 32 entries a warp loads per pass
