@@ -122,6 +122,31 @@ int efcp_get_weights(efcp_ctx* ctx, double* host_w);
  */
 int efcp_get_window(efcp_ctx* ctx, const int32_t** dev_I, const float** dev_V);
 
+/*
+ * Checkpoint / resume.  The optimizer state of Algorithm 1 is xi and the window G (plus what
+ * the library derives from them: S, the inverse, the offset table, the index and value
+ * streams); efcp_state_export copies all of it into host memory, efcp_state_import puts it
+ * back into a handle created with the same d, m, k, lambda and flags on the same kind of
+ * GPU (the slab width, which depends on d, m and the SM count, must agree).  A run resumed
+ * from an imported state continues like the run that exported it: the state bit for bit,
+ * the updates up to the fp32 rounding of their accumulation order.
+ *   efcp_state_size   : bytes efcp_state_export writes (-1 for a NULL handle).
+ *   efcp_state_export : waits for the device; host_buf needs efcp_state_size bytes.
+ *   efcp_state_import : waits for the device; EFCP_EINVAL when the header does not match
+ *                       the handle or `bytes` is too small.
+ */
+int64_t efcp_state_size(efcp_ctx* ctx);
+int efcp_state_export(efcp_ctx* ctx, void* host_buf, int64_t bytes);
+int efcp_state_import(efcp_ctx* ctx, const void* host_buf, int64_t bytes);
+
+/*
+ * efcp_error_norm - the Euclidean norm of the error buffer xi (fp64 accumulation), the
+ * numerator of the error-feedback evolution metric |xi_t| / (|g_1| + ... + |g_t|) of
+ * Section 4 ("Error Feedback Evolution During Training"); the gradient norms are the
+ * caller's.  Waits for the device.  *out (host) receives the norm.
+ */
+int efcp_error_norm(efcp_ctx* ctx, double* out);
+
 /* Number of completed efcp_step calls on this handle (-1 for a NULL handle). */
 int64_t efcp_step_count(efcp_ctx* ctx);
 

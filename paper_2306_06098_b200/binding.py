@@ -36,6 +36,10 @@ EXPORTS = {
     "efcp_get_gram": ([_vp, _vp], C.c_int),
     "efcp_get_weights": ([_vp, _vp], C.c_int),
     "efcp_get_window": ([_vp, _vp, _vp], C.c_int),
+    "efcp_state_size": ([_vp], _i64),
+    "efcp_state_export": ([_vp, _vp, _i64], C.c_int),
+    "efcp_state_import": ([_vp, _vp, _i64], C.c_int),
+    "efcp_error_norm": ([_vp, _vp], C.c_int),
     "efcp_step_count": ([_vp], _i64),
     "efcp_status": ([_vp], C.c_int),
     "efcp_last_cuda_error": ([_vp], C.c_int),
@@ -199,6 +203,23 @@ class Efcp:
         dev = torch.device("cuda", torch.cuda.current_device())
         return (torch.as_tensor(_Alias(pi.value, "<i4", shape), device=dev),
                 torch.as_tensor(_Alias(pv.value, "<f4", shape), device=dev))
+
+    def state_export(self) -> np.ndarray:
+        """The whole optimizer state as one host byte array (efcp_state_export)."""
+        n = int(_lib.efcp_state_size(self._h))
+        buf = np.empty(n, np.uint8)
+        self._check(_lib.efcp_state_export(self._h, _np_ptr(buf), n), "efcp_state_export")
+        return buf
+
+    def state_import(self, buf: np.ndarray):
+        buf = np.ascontiguousarray(buf, np.uint8)
+        self._check(_lib.efcp_state_import(self._h, _np_ptr(buf), buf.size), "efcp_state_import")
+
+    def error_norm(self) -> float:
+        out = C.c_double()
+        self._check(_lib.efcp_error_norm(self._h, C.cast(C.byref(out), C.c_void_p)),
+                    "efcp_error_norm")
+        return float(out.value)
 
     def weights(self) -> np.ndarray:
         out = np.empty(self.m, np.float64)

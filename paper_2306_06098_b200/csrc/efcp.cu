@@ -549,6 +549,134 @@ int efcp_get_window(efcp_ctx* ctx, const int32_t** dev_I, const float** dev_V) {
   return rc;
 }
 
+namespace {
+
+struct StateHeader {
+  uint64_t magic;
+  int64_t d, k, t;
+  int32_t m, W, n_slabs;
+  uint32_t flags;
+  float lambda;
+  uint32_t pad;
+};
+constexpr uint64_t kStateMagic = 0x3130505443464645ull;  // "EFCPTP01"
+
+struct StatePart {
+  void* dev;
+  int64_t bytes;
+};
+
+// the device arrays a checkpoint holds, in file order
+std::vector<StatePart> state_parts(efcp_ctx* ctx) {
+  const int64_t mk = int64_t(ctx->m) * ctx->k, mm = int64_t(ctx->m) * ctx->m;
+  std::vector<StatePart> p = {
+      {ctx->e, ctx->d * 4},
+      {ctx->I, mk * 4},
+      {ctx->V, mk * 4},
+      {ctx->R, mk * 2},
+      {ctx->offs, int64_t(ctx->n_slabs + 1) * ctx->m * 4},
+      {ctx->colsum, int64_t(ctx->n_slabs + 1) * 8},
+      {ctx->S, mm * 8},
+      {ctx->B, mm * 8},
+  };
+  if (ctx->V16) p.push_back({ctx->V16, mk * 2});
+  return p;
+}
+
+// sum of squares of e in fp64: per-block partials, then one block
+__global__ void __launch_bounds__(256) k_sumsq(const float* __restrict__ e, int64_t d,
+                                                double* __restrict__ part) {
+  __shared__ double sm[32];
+  double acc = 0.0;
+  for (int64_t j = int64_t(blockIdx.x) * blockDim.x + threadIdx.x; j < d;
+       j += int64_t(gridDim.x) * blockDim.x) {
+    const double v = double(e[j]);
+    acc += v * v;
+  }
+  acc = block_sum(acc, sm);
+  if (threadIdx.x == 0) part[blockIdx.x] = acc;
+}
+__global__ void __launch_bounds__(256) k_sum_parts(const double* __restrict__ part, int n,
+                                                    double* __restrict__ out) {
+  __shared__ double sm[32];
+  double acc = 0.0;
+  for (int i = threadIdx.x; i < n; i += blockDim.x) acc += part[i];
+  acc = block_sum(acc, sm);
+  if (threadIdx.x == 0) *out = acc;
+}
+
+}  // namespace
+
+int64_t efcp_state_size(efcp_ctx* ctx) {
+  if (!ctx) return -1;
+  int64_t b = int64_t(sizeof(StateHeader));
+  for (const StatePart& p : state_parts(ctx)) b += p.bytes;
+  return b;
+}
+
+int efcp_state_export(efcp_ctx* ctx, void* host_buf, int64_t bytes) {
+  if (!ctx || !host_buf || bytes < efcp_state_size(ctx)) return EFCP_EINVAL;
+  const int rc = sync_status(ctx);
+  if (rc == EFCP_ECUDA) return rc;
+  StateHeader h{};
+  h.magic = kStateMagic; h.d = ctx->d; h.k = ctx->k; h.t = ctx->t; h.m = ctx->m; h.W = ctx->W;
+  h.n_slabs = ctx->n_slabs; h.flags = ctx->flags; h.lambda = ctx->lambda;
+  unsigned char* out = static_cast<unsigned char*>(host_buf);
+  std::memcpy(out, &h, sizeof(h));
+  out += sizeof(h);
+  for (const StatePart& p : state_parts(ctx)) {
+    EFCP_CUDA(cudaMemcpy(out, p.dev, size_t(p.bytes), cudaMemcpyDeviceToHost));
+    out += p.bytes;
+  }
+  return rc;
+}
+
+int efcp_state_import(efcp_ctx* ctx, const void* host_buf, int64_t bytes) {
+  if (!ctx || !host_buf || bytes < efcp_state_size(ctx)) return EFCP_EINVAL;
+  StateHeader h;
+  std::memcpy(&h, host_buf, sizeof(h));
+  if (h.magic != kStateMagic || h.d != ctx->d || h.k != ctx->k || h.m != ctx->m ||
+      h.W != ctx->W || h.n_slabs != ctx->n_slabs || h.flags != ctx->flags ||
+      std::memcmp(&h.lambda, &ctx->lambda, 4) != 0 || h.t < 0)
+    return EFCP_EINVAL;
+  EFCP_CUDA(cudaSetDevice(ctx->device));
+  EFCP_CUDA(cudaDeviceSynchronize());
+  const unsigned char* in = static_cast<const unsigned char*>(host_buf) + sizeof(h);
+  for (const StatePart& p : state_parts(ctx)) {
+    EFCP_CUDA(cudaMemcpy(p.dev, in, size_t(p.bytes), cudaMemcpyHostToDevice));
+    in += p.bytes;
+  }
+  // scalars: clear the sticky status and the previous threshold (the next step takes the
+  // two-pass route once; the selection does not depend on the route)
+  EFCP_CUDA(cudaMemset(ctx->sc, 0, sizeof(Scalars)));
+  EFCP_CUDA(cudaMemset(ctx->hist, 0, (kBins1 + kBins2 + kBins3) * 4));
+  ctx->t = h.t;
+  return EFCP_OK;
+}
+
+int efcp_error_norm(efcp_ctx* ctx, double* out) {
+  if (!ctx || !out) return EFCP_EINVAL;
+  const int rc = sync_status(ctx);
+  if (rc == EFCP_ECUDA) return rc;
+  // scratch: the SP partial buffers are idle between steps (m >= 1 doubles each; use slab_part)
+  const int blocks = int(std::min<int64_t>(ctx->num_sms * 4, int64_t(ctx->n_slabs) * ctx->m - 1));
+  const int nb = blocks < 1 ? 1 : blocks;
+  if (int64_t(ctx->n_slabs) * ctx->m < 2) {  // degenerate sizes: do it on the host
+    std::vector<float> h(static_cast<size_t>(ctx->d));
+    EFCP_CUDA(cudaMemcpy(h.data(), ctx->e, size_t(ctx->d) * 4, cudaMemcpyDeviceToHost));
+    double s = 0.0;
+    for (float v : h) s += double(v) * double(v);
+    *out = std::sqrt(s);
+    return rc;
+  }
+  k_sumsq<<<nb, 256>>>(ctx->e, ctx->d, ctx->slab_part + 1);
+  k_sum_parts<<<1, 256>>>(ctx->slab_part + 1, nb, ctx->slab_part);
+  double s = 0.0;
+  EFCP_CUDA(cudaMemcpy(&s, ctx->slab_part, 8, cudaMemcpyDeviceToHost));
+  *out = std::sqrt(s);
+  return rc;
+}
+
 int64_t efcp_step_count(efcp_ctx* ctx) { return ctx ? ctx->t : -1; }
 
 int efcp_status(efcp_ctx* ctx) {

@@ -361,3 +361,55 @@ def test_two_pass_route_alone(monkeypatch):
     scale = np.exp(rng.standard_normal(d))
     grads = ((scale * rng.standard_normal(d)).astype(np.float32) for _ in range(10))
     run_parity(d, m, k, 1e-4, grads, check_rows="all")
+
+
+@pytest.mark.parametrize("flags", [0, 1, 2], ids=["fp32", "rhs_accumulator", "values_bf16"])
+def test_checkpoint_resume_continues_bit_for_bit(flags):
+    B = _binding()
+    d, m, k = 250_003, 6, 2500
+    rng = np.random.default_rng(40 + flags)
+    scale = np.exp(rng.standard_normal(d))
+    grads = [(scale * rng.standard_normal(d)).astype(np.float32) for _ in range(16)]
+    a = B.Efcp(d, m, k, 1e-4, flags)
+    g_dev = torch.empty(d, dtype=torch.float32, device="cuda")
+    ua = torch.empty(d, dtype=torch.float32, device="cuda")
+    ub = torch.empty(d, dtype=torch.float32, device="cuda")
+    for g in grads[:9]:  # past one turn of the ring
+        g_dev.copy_(torch.from_numpy(g))
+        a.step(g_dev, ua)
+    blob = a.state_export()
+    b = B.Efcp(d, m, k, 1e-4, flags)
+    b.state_import(blob)
+    assert b.step_count == a.step_count == 9
+    for g in grads[9:]:
+        g_dev.copy_(torch.from_numpy(g))
+        a.step(g_dev, ua)
+        b.step(g_dev, ub)
+        # the update is a sum of fp32 shared-memory atomics whose order is not fixed: equal up
+        # to fp32 rounding of the accumulation; the state below is bit for bit
+        assert rel_l2(ub.cpu().numpy(), ua.cpu().numpy()) <= 1e-6
+        assert np.array_equal(bits(a.error()), bits(b.error()))
+    for s in range(m):
+        ai, av = a.row(s)
+        bi, bv = b.row(s)
+        assert np.array_equal(ai, bi) and np.array_equal(bits(av), bits(bv))
+    # a blob of another shape is refused
+    c = B.Efcp(d, m + 1, k, 1e-4, flags)
+    with pytest.raises(B.EfcpError) as ei:
+        c.state_import(blob)
+    assert ei.value.code == B.EINVAL
+
+
+def test_error_norm_is_the_norm_of_the_error_buffer():
+    B = _binding()
+    d, m, k = 123_457, 4, 1000
+    rng = np.random.default_rng(50)
+    opt = B.Efcp(d, m, k, 1e-3)
+    g_dev = torch.empty(d, dtype=torch.float32, device="cuda")
+    u = torch.empty(d, dtype=torch.float32, device="cuda")
+    assert opt.error_norm() == 0.0
+    for _ in range(5):
+        g_dev.copy_(torch.from_numpy(rng.standard_normal(d).astype(np.float32)))
+        opt.step(g_dev, u)
+        want = np.linalg.norm(opt.error().astype(np.float64))
+        assert abs(opt.error_norm() - want) <= 1e-12 * want
