@@ -413,3 +413,32 @@ def test_error_norm_is_the_norm_of_the_error_buffer():
         opt.step(g_dev, u)
         want = np.linalg.norm(opt.error().astype(np.float64))
         assert abs(opt.error_norm() - want) <= 1e-12 * want
+
+
+def test_large_window_m2048():
+    # a window longer than the benchmark's: the shared-memory budget forces a narrower slab
+    d, m, k = 600_011, 2048, 600
+    rng = np.random.default_rng(60)
+    scale = np.exp(rng.standard_normal(d))
+    grads = ((scale * rng.standard_normal(d)).astype(np.float32) for _ in range(4))
+    run_parity(d, m, k, 1e-3, grads, gram_every=2)
+
+
+def test_steps_on_a_side_stream():
+    B = _binding()
+    d, m, k = 200_003, 4, 2000
+    rng = np.random.default_rng(61)
+    gpu = B.Efcp(d, m, k, 1e-3)
+    cpu = ref.RefEFCP(d, m, k, 1e-3)
+    side = torch.cuda.Stream()
+    g_dev = torch.empty(d, dtype=torch.float32, device="cuda")
+    u_dev = torch.empty(d, dtype=torch.float32, device="cuda")
+    for t in range(6):
+        g = rng.standard_normal(d).astype(np.float32)
+        g_dev.copy_(torch.from_numpy(g))
+        side.wait_stream(torch.cuda.current_stream())
+        gpu.step(g_dev, u_dev, stream=side)
+        side.synchronize()
+        u_ref = cpu.step(g)
+        assert np.array_equal(bits(gpu.error()), bits(cpu.error()))
+        assert rel_l2(u_dev.cpu().numpy(), u_ref) <= U_TOL
