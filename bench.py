@@ -296,32 +296,33 @@ def main():
                "h2d_bytes_per_step": 4 * w.d, "d2h_bytes_per_step": 4 * w.d,
                "steps": args.e2e_steps}
 
-    # roofline of the dominant kernel (HBM bound): bytes the kernel has to move per launch /
-    # its time.  The kernels stream a window entry as a 16-bit slab-relative index and an
-    # fp32 value: 6 bytes.  (Counted with the 32-bit indices of the (I, V) format, 8 bytes
-    # per entry, the same times give the `as_int32_indices` figures.)
+    # roofline of the dominant kernel (HBM bound): algorithmic bytes per launch / its time.
+    # Algorithmic bytes are those of the method's (I, V) window format, int32 index + fp32
+    # value = 8 bytes per entry (4 + 2 with bf16 values), as the scope table counts them.  The
+    # kernels themselves stream a 16-bit slab-relative index instead of the int32 one, i.e.
+    # 6 (4) bytes per entry: `moved` repeats the figures with the bytes actually read, which
+    # is what the DRAM counters (`traffic`) have to be compared with.
     # x = a_t adds one read of xi to SP and one to LCG.
     peak, peak_src = load_peak()
     mk = w.m * w.k
     xi_read = 4 * w.d if acc else 0
-    entry = 4 if bf16 else 6  # bytes streamed per window entry
-    alg = {"sp": entry * mk + xi_read, "lcg": entry * mk + 4 * w.d + xi_read}
-    alg8 = {"sp": 8 * mk + xi_read, "lcg": 8 * mk + 4 * w.d + xi_read}
+    val_b = 2 if bf16 else 4
+    alg = {"sp": (4 + val_b) * mk + xi_read, "lcg": (4 + val_b) * mk + 4 * w.d + xi_read}
+    mov = {"sp": (2 + val_b) * mk + xi_read, "lcg": (2 + val_b) * mk + 4 * w.d + xi_read}
     kern = max(("sp", "lcg"), key=lambda s: stages[s])
     avg_ms = stages[kern] / max(n_rec, 1)
     achieved = alg[kern] / (avg_ms * 1e-3) / 1e9
+    moved = mov[kern] / (avg_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": {"sp": "k_sp_rows", "lcg": "k_lcg"}[kern],
                 "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": None if (acc or bf16) else NCU_TRAFFIC_BYTES.get(w.name, {}).get(kern),
                 "peak_source": peak_src, "algorithmic_bytes_per_launch": alg[kern],
                 "avg_launch_ms": avg_ms,
-                "as_int32_indices": {"algorithmic_bytes_per_launch": alg8[kern],
-                                     "achieved": alg8[kern] / (avg_ms * 1e-3) / 1e9,
-                                     "frac": alg8[kern] / (avg_ms * 1e-3) / 1e9 / peak}}
-    step_bytes = 2 * entry * mk + 16 * w.d + 10 * w.k + 2 * xi_read
+                "moved": {"bytes_per_launch": mov[kern], "achieved": moved, "frac": moved / peak}}
+    step_bytes = 2 * (4 + val_b) * mk + 16 * w.d + 8 * w.k + 2 * xi_read
     step_gbs = step_bytes / (ms_per_step * 1e-3) / 1e9
-    step_bytes8 = 16 * mk + 16 * w.d + 8 * w.k + 2 * xi_read
-    step_gbs8 = step_bytes8 / (ms_per_step * 1e-3) / 1e9
+    step_moved = 2 * (2 + val_b) * mk + 16 * w.d + 10 * w.k + 2 * xi_read
+    step_moved_gbs = step_moved / (ms_per_step * 1e-3) / 1e9
     stage_ms = {s: stages[s] / max(n_rec, 1) for s in stages}
 
     cpu_baseline = None
@@ -347,10 +348,9 @@ def main():
             "roofline": roofline,
             "step_hbm": {"algorithmic_bytes_per_step": step_bytes, "achieved_gbs": step_gbs,
                          "frac_of_peak": step_gbs / peak, "frac_of_8tbs": step_gbs / 8000.0,
-                         "as_int32_indices": {"algorithmic_bytes_per_step": step_bytes8,
-                                              "achieved_gbs": step_gbs8,
-                                              "frac_of_peak": step_gbs8 / peak,
-                                              "frac_of_8tbs": step_gbs8 / 8000.0}},
+                         "moved": {"bytes_per_step": step_moved, "achieved_gbs": step_moved_gbs,
+                                   "frac_of_peak": step_moved_gbs / peak,
+                                   "frac_of_8tbs": step_moved_gbs / 8000.0}},
             "stage_ms": stage_ms,
             "cpu_baseline": cpu_baseline,
         }

@@ -92,7 +92,7 @@ int pick_slab_width(int64_t d, int m, int num_sms) {
   // at least one slab per SM (the slab kernels run one block per SM and rebalance by
   // drawing slabs from a counter), but no slab narrower than 2048 coordinates: below that
   // a row's segment is a handful of entries and the per-row bookkeeping dominates
-  while (W > 2048 && (d + W - 1) / W < int64_t(num_sms)) W >>= 1;
+  while (W / 2 >= 2048 && (d + W - 1) / W < int64_t(num_sms)) W = (W / 2) & ~31;
   return W;
 }
 
