@@ -95,6 +95,8 @@ struct Oracle {
   int64_t k = 0;
   float lambda = 0.f;
   uint32_t flags = 0;
+  int64_t block = 0;  // > 0: Top-k is applied per block of this many coordinates
+  int64_t k_req = 0;  // the k the caller asked for (k is the row length actually kept)
   int64_t t = 0;  // number of completed steps
   std::vector<float> e;      // error feedback buffer (xi), d
   std::vector<float> a;      // accumulator of the last step, d
@@ -265,15 +267,30 @@ int efcp_ref_wsm_coef(const double* S, const double* p, int32_t m, double lambda
   return 0;
 }
 
-int efcp_ref_create(efcp_ref** out, int64_t d, int32_t m, int64_t k, float lambda,
-                    uint32_t flags) {
+// Entries block-wise Top-k keeps in a block of `len` coordinates at density k/d:
+// ceil(len * k / d) (Section 3.1 "Sparsity Pattern": ceil(B / 100) at 1 %).
+int64_t efcp_ref_block_count(int64_t len, int64_t k, int64_t d) { return (len * k + d - 1) / d; }
+
+// block > 0: Top-k applied in blocks of `block` coordinates (Section 3.1, "Sparsity
+// Pattern"); every row then holds the sum of the per-block counts, see
+// efcp_ref_row_length.  block == 0: one global Top-k of k entries.
+int efcp_ref_create_blockwise(efcp_ref** out, int64_t d, int32_t m, int64_t k, float lambda,
+                              uint32_t flags, int64_t block) {
   if (!out) return -1;
   *out = nullptr;
-  if (d < 1 || m < 1 || k < 1 || k > d || d >= (int64_t(1) << 31)) return -1;
+  if (d < 1 || m < 1 || k < 1 || k > d || d >= (int64_t(1) << 31) || block < 0) return -1;
   if (!(lambda > 0.f) || !std::isfinite(lambda)) return -1;
   Oracle* o = new (std::nothrow) Oracle();
   if (!o) return -2;
   try {
+    o->k_req = k;
+    o->block = block;
+    if (block > 0) {
+      int64_t total = 0;
+      for (int64_t b0 = 0; b0 < d; b0 += block)
+        total += efcp_ref_block_count(std::min(block, d - b0), k, d);
+      k = total;
+    }
     o->d = d; o->m = m; o->k = k; o->lambda = lambda; o->flags = flags;
     o->e.assign(size_t(d), 0.f);
     o->a.assign(size_t(d), 0.f);
@@ -297,6 +314,17 @@ int efcp_ref_create(efcp_ref** out, int64_t d, int32_t m, int64_t k, float lambd
   return 0;
 }
 
+int efcp_ref_create(efcp_ref** out, int64_t d, int32_t m, int64_t k, float lambda,
+                    uint32_t flags) {
+  return efcp_ref_create_blockwise(out, d, m, k, lambda, flags, 0);
+}
+
+// Entries per row: k for global Top-k, the sum of the per-block counts otherwise.
+int64_t efcp_ref_row_length(efcp_ref* h) {
+  Oracle* o = reinterpret_cast<Oracle*>(h);
+  return o ? o->k : -1;
+}
+
 void efcp_ref_destroy(efcp_ref* h) { delete reinterpret_cast<Oracle*>(h); }
 
 // One optimizer step.  grad and update are host arrays of d floats.
@@ -317,7 +345,20 @@ int efcp_ref_step(efcp_ref* h, const float* grad, float* update) {
   const int32_t i = int32_t(o->t % m);
   int32_t* idx = &o->I[size_t(i) * size_t(k)];
   float* val = &o->V[size_t(i) * size_t(k)];
-  topk_select(o->a.data(), d, k, o->order, idx, val);
+  if (o->block > 0) {
+    // Section 3.1 "Sparsity Pattern": an exact Top-k inside every block of `block`
+    // coordinates; the blocks follow one another, so the row stays in ascending order.
+    int64_t pos = 0;
+    for (int64_t b0 = 0; b0 < d; b0 += o->block) {
+      const int64_t len = std::min(o->block, d - b0);
+      const int64_t c = efcp_ref_block_count(len, o->k_req, d);
+      topk_select(o->a.data() + b0, len, c, o->order, idx + pos, val + pos);
+      for (int64_t r = 0; r < c; ++r) idx[pos + r] += int32_t(b0);
+      pos += c;
+    }
+  } else {
+    topk_select(o->a.data(), d, k, o->order, idx, val);
+  }
 
   // Section 3.1 "Format for V" (optional): the window holds bfloat16 values, so c is the
   // selection with every value rounded to bfloat16.

@@ -23,6 +23,9 @@ def lib():
         vp, i32, i64, f32, u32, f64 = (C.c_void_p, C.c_int32, C.c_int64, C.c_float,
                                        C.c_uint32, C.c_double)
         L.efcp_ref_create.argtypes = [C.POINTER(vp), i64, i32, i64, f32, u32]
+        L.efcp_ref_create_blockwise.argtypes = [C.POINTER(vp), i64, i32, i64, f32, u32, i64]
+        L.efcp_ref_row_length.argtypes = [vp]
+        L.efcp_ref_row_length.restype = i64
         L.efcp_ref_destroy.argtypes = [vp]
         L.efcp_ref_destroy.restype = None
         L.efcp_ref_step.argtypes = [vp, vp, vp]
@@ -91,14 +94,19 @@ def wsm_coef(S, p, lam):
 
 
 class RefEFCP:
-    def __init__(self, d, m, k, lam, flags=RHS_COMPRESSED):
+    def __init__(self, d, m, k, lam, flags=RHS_COMPRESSED, block=0):
+        """block > 0: Top-k in blocks of `block` coordinates; self.k then becomes the row
+        length (the sum of the per-block counts), self.k_req keeps the requested k."""
         self._h = None
         self.d, self.m, self.k, self.lam, self.flags = int(d), int(m), int(k), float(lam), flags
+        self.k_req, self.block = int(k), int(block)
         h = C.c_void_p()
-        rc = lib().efcp_ref_create(C.byref(h), self.d, self.m, self.k, self.lam, flags)
+        rc = lib().efcp_ref_create_blockwise(C.byref(h), self.d, self.m, self.k, self.lam, flags,
+                                             self.block)
         if rc != 0:
             raise ValueError(f"efcp_ref_create rc={rc}")
         self._h = h
+        self.k = int(lib().efcp_ref_row_length(h))
 
     def close(self):
         if self._h:

@@ -189,6 +189,45 @@ def test_bf16_update_matches_dense_solve(d, m, k, steps, lam):
         assert rel(o.update_rowform(), want) < 2e-6
 
 
+# ------------------------------------------- block-wise Top-k (Section 3.1, "Sparsity Pattern")
+def test_blockwise_topk_keeps_the_stated_count_in_every_block():
+    rng = np.random.default_rng(33)
+    d, m, k, block = 10_007, 3, 100, 1000      # 1 % -> ceil(1000/100) = 10 per full block
+    o = ref.RefEFCP(d, m, k, 1e-3, block=block)
+    assert o.k == 10 * 10 + 1                   # ten full blocks, ceil(7 * 100 / 10007) = 1
+    e_prev = np.zeros(d, np.float32)
+    for t in range(5):
+        g = (rng.standard_normal(d) * np.exp(rng.standard_normal(d))).astype(np.float32)
+        o.step(g)
+        a = (e_prev + g).astype(np.float32)
+        idx, val = o.row(t % m)
+        assert np.all(np.diff(idx) > 0)
+        want_i, want_v = [], []
+        for b0 in range(0, d, block):
+            blk = a[b0:b0 + block]
+            c = -(-blk.size * k // d)
+            bi, bv = topk_by_sort(blk, c)       # the definition, block by block
+            want_i.append(bi + b0)
+            want_v.append(bv)
+        assert np.array_equal(idx, np.concatenate(want_i))
+        assert np.array_equal(val.view(np.uint32), np.concatenate(want_v).view(np.uint32))
+        e = o.error()
+        assert not e[idx].any()
+        e_prev = e
+
+
+def test_blockwise_with_one_block_is_global_topk():
+    rng = np.random.default_rng(34)
+    d, m, k = 3000, 2, 77
+    a = ref.RefEFCP(d, m, k, 1e-2)
+    b = ref.RefEFCP(d, m, k, 1e-2, block=d)
+    assert b.k == k
+    for _ in range(4):
+        g = rng.standard_normal(d).astype(np.float32)
+        ua, ub = a.step(g), b.step(g)
+        assert np.array_equal(ua.view(np.uint32), ub.view(np.uint32))
+
+
 def test_m1_closed_form():
     # m = 1: F^-1 x = x/lam - g (g.x) / (lam (m lam + g.g))
     rng = np.random.default_rng(5)
