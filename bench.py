@@ -205,6 +205,9 @@ def main():
                     help="precondition c_t (Algorithm 1, default) or the whole accumulator a_t")
     ap.add_argument("--values", default="fp32", choices=["fp32", "bf16"],
                     help="window value format (bf16: Section 3.1 'Format for V', not the default)")
+    ap.add_argument("--block", type=int, default=0,
+                    help="block-wise Top-k with blocks of this many coordinates (Section 3.1 "
+                         "'Sparsity Pattern'); 0 = global Top-k, the default")
     ap.add_argument("--prefill", type=int, default=-1,
                     help="untimed steps before warm-up; -1 = m (fill the whole window)")
     ap.add_argument("--e2e-steps", type=int, default=5)
@@ -232,7 +235,10 @@ def main():
     bf16 = args.values == "bf16"
     opt = binding.Efcp(w.d, w.m, w.k, w.lam,
                        (binding.RHS_ACCUMULATOR if acc else binding.RHS_COMPRESSED) |
-                       (binding.VALUES_BF16 if bf16 else 0))
+                       (binding.VALUES_BF16 if bf16 else 0), args.block)
+    if args.block:  # rows are a little longer than k: count the bytes of what is really kept
+        w = gradgen.Workload(w.name, w.d, w.m, opt.k, w.lam, w.steps, w.rank, w.scale_block,
+                             w.seed, w.noise)
     gbuf = torch.empty(w.d, dtype=torch.float32, device=device)
     ubuf = torch.empty(w.d, dtype=torch.float32, device=device)
 
@@ -340,7 +346,9 @@ def main():
             "warmup": W, "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": w.name, "d": w.d, "m": w.m, "k": w.k, "lambda": w.lam,
-                       "rhs": args.rhs, "window_values": args.values, "prefill_steps": prefill,
+                       "rhs": args.rhs, "window_values": args.values,
+                       "topk": f"blockwise({args.block})" if args.block else "global",
+                       "prefill_steps": prefill,
                        "parallelism": f"replicas x{world}",
                        "l2": "inputs larger than L2 (window %.2f GB, gradient %.2f GB)" % (
                            8 * w.m * w.k / 1e9, 4 * w.d / 1e9)},

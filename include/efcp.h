@@ -64,6 +64,22 @@ int efcp_create_ex(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float lambda
                    uint32_t flags);
 
 /*
+ * efcp_create_blockwise - the same optimizer with Top-k applied in blocks (Section 3.1,
+ * "Sparsity Pattern"): the coordinates are cut into blocks of `block` coordinates and every
+ * block keeps exactly ceil(len * k / d) entries of largest magnitude, len being the block's
+ * length (the last block may be shorter), ties to the lower index; at 1 % density that is
+ * the paper's ceil(B / 100) per block.  A row of the window then holds efcp_row_length(ctx)
+ * entries (the sum over the blocks, a little above k), and every efcp_get_* call that speaks
+ * of k entries means that many.  Everything after the selection is as in efcp_create_ex.
+ *   block: a multiple of 32 in [32, 16384].
+ */
+int efcp_create_blockwise(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float lambda,
+                          uint32_t flags, int32_t block);
+
+/* Entries per window row: k, or the block-wise total (-1 for a NULL handle). */
+int64_t efcp_row_length(efcp_ctx* ctx);
+
+/*
  * efcp_step - Algorithm 1 lines 5-8 for one gradient:
  *     a = xi + g                      (fp32, one rounding per coordinate)
  *     c = TopK_k(a)                   (global over d, exact, ties to the lower index)

@@ -28,6 +28,8 @@ _vp, _i32, _i64, _f32, _u32 = C.c_void_p, C.c_int32, C.c_int64, C.c_float, C.c_u
 EXPORTS = {
     "efcp_create": ([C.POINTER(_vp), _i64, _i32, _i64, _f32], C.c_int),
     "efcp_create_ex": ([C.POINTER(_vp), _i64, _i32, _i64, _f32, _u32], C.c_int),
+    "efcp_create_blockwise": ([C.POINTER(_vp), _i64, _i32, _i64, _f32, _u32, _i32], C.c_int),
+    "efcp_row_length": ([_vp], _i64),
     "efcp_step": ([_vp, _vp, _vp, _vp], C.c_int),
     "efcp_step_host": ([_vp, _vp, _vp, _vp], C.c_int),
     "efcp_destroy": ([_vp], C.c_int),
@@ -101,14 +103,20 @@ def _np_ptr(a: np.ndarray):
 class Efcp:
     """One optimizer state (efcp_ctx) on the current CUDA device."""
 
-    def __init__(self, d: int, m: int, k: int, lam: float, flags: int = RHS_COMPRESSED):
+    def __init__(self, d: int, m: int, k: int, lam: float, flags: int = RHS_COMPRESSED,
+                 block: int = 0):
+        """block > 0: Top-k in blocks of `block` coordinates (efcp_create_blockwise); self.k is
+        then the row length efcp_row_length reports, self.k_req the requested k."""
         self._h = None
         self.d, self.m, self.k, self.lam, self.flags = int(d), int(m), int(k), float(lam), flags
+        self.k_req, self.block = int(k), int(block)
         h = _vp()
-        rc = _lib.efcp_create_ex(C.byref(h), self.d, self.m, self.k, self.lam, flags)
+        rc = _lib.efcp_create_blockwise(C.byref(h), self.d, self.m, self.k, self.lam, flags,
+                                        self.block)
         if rc != OK:
-            raise EfcpError(rc, "efcp_create_ex")
+            raise EfcpError(rc, "efcp_create_blockwise")
         self._h = h
+        self.k = int(_lib.efcp_row_length(h))
 
     def close(self):
         if self._h and _lib is not None:  # (_lib is gone while the interpreter shuts down)

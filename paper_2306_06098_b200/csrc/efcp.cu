@@ -16,6 +16,7 @@
 #include <vector>
 
 #include "efcp_common.cuh"
+#include "efcp_blockwise.cuh"
 #include "efcp_mxm.cuh"
 #include "efcp_topk.cuh"
 #include "efcp_window.cuh"
@@ -23,7 +24,10 @@
 using namespace efcp;
 
 struct efcp_ctx {
-  int64_t d = 0, k = 0;
+  int64_t d = 0, k = 0;  // k: entries per window row
+  int64_t k_req = 0;     // the k of the create call (block-wise Top-k keeps a little more)
+  int block = 0, n_blocks = 0;  // block-wise Top-k: block length in coordinates, number of blocks
+  uint32_t* blk_T = nullptr;    // per block: last step's threshold key
   int32_t m = 0;
   float lambda = 0.f;
   uint32_t flags = 0;
@@ -224,11 +228,26 @@ int efcp_create(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float lambda) {
 
 int efcp_create_ex(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float lambda,
                    uint32_t flags) {
+  return efcp_create_blockwise(out, d, m, k, lambda, flags, 0);
+}
+
+int64_t efcp_row_length(efcp_ctx* ctx) { return ctx ? ctx->k : -1; }
+
+int efcp_create_blockwise(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float lambda,
+                          uint32_t flags, int32_t block) {
   if (!out) return EFCP_EINVAL;
   *out = nullptr;
   if (!valid_args(d, m, k) || !(lambda > 0.f) || !std::isfinite(lambda)) return EFCP_EINVAL;
   if (flags & ~(EFCP_RHS_ACCUMULATOR | EFCP_VALUES_BF16)) return EFCP_EINVAL;
   if ((flags & EFCP_RHS_ACCUMULATOR) && (flags & EFCP_VALUES_BF16)) return EFCP_EINVAL;
+  if (block != 0 && (block < 32 || block > kBlkMax || (block & 31))) return EFCP_EINVAL;
+  const int64_t k_req = k;
+  int n_blocks = 0;
+  if (block) {  // the row length is the sum of the per-block counts
+    n_blocks = int((d + block - 1) / block);
+    const int64_t last = d - int64_t(n_blocks - 1) * block;
+    k = int64_t(n_blocks - 1) * block_count(block, k_req, d) + block_count(last, k_req, d);
+  }
   efcp_ctx* ctx = new (std::nothrow) efcp_ctx();
   if (!ctx) return EFCP_ENOMEM;
   int rc = EFCP_OK;
@@ -244,6 +263,7 @@ int efcp_create_ex(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float lambda
   if (err != cudaSuccess) { (void)cudaGetLastError(); return fail(EFCP_ECUDA); }
   ctx->num_sms = prop.multiProcessorCount;
   ctx->d = d; ctx->m = m; ctx->k = k; ctx->lambda = lambda; ctx->flags = flags;
+  ctx->k_req = k_req; ctx->block = block; ctx->n_blocks = n_blocks;
   const Sizes z = compute_sizes(d, m, k, ctx->num_sms);
   ctx->W = z.W; ctx->n_slabs = z.n_slabs; ctx->n_chunks = z.n_chunks;
   ctx->grid_slab = z.grid_slab;
@@ -277,6 +297,10 @@ int efcp_create_ex(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float lambda
   if ((rc = dev_alloc(ctx, &ctx->vecs, int64_t(9) * m * 8))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->wf, int64_t(m) * 4))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->slab_ctr, 256))) return fail(rc);
+  if (block) {
+    if ((rc = dev_alloc(ctx, &ctx->blk_T, int64_t(n_blocks) * 4))) return fail(rc);
+    if (cudaMemset(ctx->blk_T, 0, size_t(n_blocks) * 4) != cudaSuccess) return fail(EFCP_ECUDA);
+  }
   if ((rc = dev_alloc(ctx, &ctx->colsum, int64_t(z.n_slabs + 1) * 8))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->order, int64_t(z.n_slabs) * 4))) return fail(rc);
 
@@ -296,6 +320,11 @@ int efcp_create_ex(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float lambda
   k_init_identity<<<ctx->num_sms * 2, 256>>>(ctx->B, m, 1.0 / (double(m) * double(lambda)));
   const size_t smem = slab_smem_bytes(z.W, m);
   const auto attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
+  if (block) {
+    const int bs = blk_pad(block) * 4;
+    ok &= cudaFuncSetAttribute(k_ef_block_select<true>, attr, bs) == cudaSuccess;
+    ok &= cudaFuncSetAttribute(k_ef_block_select<false>, attr, bs) == cudaSuccess;
+  }
   ok &= cudaFuncSetAttribute(k_sp_rows<false, float>, attr, int(smem)) == cudaSuccess;
   ok &= cudaFuncSetAttribute(k_sp_rows<true, float>, attr, int(smem)) == cudaSuccess;
   ok &= cudaFuncSetAttribute(k_sp_rows<false, bf16raw>, attr, int(smem)) == cudaSuccess;
@@ -346,53 +375,68 @@ int efcp_step(efcp_ctx* ctx, const float* grad, float* update, void* stream_) {
   const double mlambda = double(m) * double(ctx->lambda);
 
   prof_mark(ctx, 0, st);
-  // a = xi + g, digit-1 histogram, speculative candidate buckets
-  const int chunk_grid = ctx->n_chunks < ctx->num_sms * 8 ? ctx->n_chunks : ctx->num_sms * 8;
-  const int spec = ctx->spec ? 1 : 0;
-  if ((reinterpret_cast<uintptr_t>(grad) & 15) == 0)
-    k_ef_spec<true><<<chunk_grid, kChunkThreads, 0, st>>>(ctx->e, grad, d, hist1, ctx->sc,
-                                                          ctx->chunk_off, ctx->bk_off,
-                                                          ctx->bk_val, ctx->n_chunks, spec);
-  else
-    k_ef_spec<false><<<chunk_grid, kChunkThreads, 0, st>>>(ctx->e, grad, d, hist1, ctx->sc,
-                                                           ctx->chunk_off, ctx->bk_off,
-                                                           ctx->bk_val, ctx->n_chunks, spec);
-  EFCP_LAUNCHED();
-  const uint32_t spec_limit = uint32_t(std::min<int64_t>(d, 3 * k + 65536));
-  k_pick<kBins1, 1><<<1, 1024, 0, st>>>(hist1, ctx->sc, uint32_t(k), spec, spec_limit);
-  EFCP_LAUNCHED();
-  // candidates: everything at or above the threshold bin, in index order.  The two-pass
-  // kernels return at once when the buckets are good, k_compact_buckets when they are not.
-  k_count_chunks<<<chunk_grid, kChunkThreads, 0, st>>>(ctx->e, d, ctx->sc, ctx->chunk_off,
-                                                       ctx->n_chunks);
-  EFCP_LAUNCHED();
-  k_scan_counts<<<1, 1024, 0, st>>>(ctx->chunk_off, ctx->n_chunks, &ctx->sc->n_cand);
-  EFCP_LAUNCHED();
-  k_compact_cand<<<chunk_grid, kChunkThreads, 0, st>>>(ctx->e, d, ctx->sc, ctx->chunk_off,
-                                                       ctx->cand_idx, ctx->cand_val, hist2,
-                                                       ctx->n_chunks);
-  EFCP_LAUNCHED();
-  k_compact_buckets<<<ctx->num_sms * 4, 256, 0, st>>>(ctx->bk_off, ctx->bk_val, ctx->sc,
-                                                      ctx->chunk_off, ctx->cand_idx,
-                                                      ctx->cand_val, hist2, ctx->n_chunks);
-  EFCP_LAUNCHED();
-  k_pick<kBins2, 2><<<1, 1024, 0, st>>>(hist2, ctx->sc, uint32_t(k));
-  EFCP_LAUNCHED();
-  const int cand_grid = ctx->num_sms * 4;
-  k_hist3<<<cand_grid, 256, 0, st>>>(ctx->cand_val, ctx->sc, hist3);
-  EFCP_LAUNCHED();
-  k_pick<kBins3, 3><<<1, 1024, 0, st>>>(hist3, ctx->sc, uint32_t(k));
-  EFCP_LAUNCHED();
-  // exact selection, ring insert, residual
-  k_count_sel<<<cand_grid, kChunkThreads, 0, st>>>(ctx->cand_val, ctx->sc, ctx->sel_gt,
-                                                   ctx->sel_eq);
-  EFCP_LAUNCHED();
-  k_scan_sel<<<1, 1024, 0, st>>>(ctx->sel_gt, ctx->sel_eq, ctx->sc, uint32_t(k));
-  EFCP_LAUNCHED();
-  k_write_sel<<<cand_grid, kChunkThreads, 0, st>>>(ctx->cand_idx, ctx->cand_val, ctx->sc,
-                                                   ctx->sel_gt, ctx->sel_eq, ctx->sel_idx,
-                                                   ctx->sel_val, ctx->e, k, ctx->V16 ? 1 : 0);
-  EFCP_LAUNCHED();
+  if (ctx->block) {
+    // block-wise Top-k: a = xi + g, the selection and xi = a - c in one kernel
+    const int grid = ctx->n_blocks < ctx->num_sms * 3 ? ctx->n_blocks : ctx->num_sms * 3;
+    const size_t bs = size_t(blk_pad(ctx->block)) * 4;
+    if ((reinterpret_cast<uintptr_t>(grad) & 15) == 0)
+      k_ef_block_select<true><<<grid, kBlkThreads, bs, st>>>(
+          ctx->e, grad, d, ctx->k_req, ctx->block, ctx->n_blocks, ctx->blk_T, ctx->sel_idx,
+          ctx->sel_val, ctx->sc, ctx->V16 ? 1 : 0);
+    else
+      k_ef_block_select<false><<<grid, kBlkThreads, bs, st>>>(
+          ctx->e, grad, d, ctx->k_req, ctx->block, ctx->n_blocks, ctx->blk_T, ctx->sel_idx,
+          ctx->sel_val, ctx->sc, ctx->V16 ? 1 : 0);
+    EFCP_LAUNCHED();
+  } else {
+    // a = xi + g, digit-1 histogram, speculative candidate buckets
+    const int chunk_grid = ctx->n_chunks < ctx->num_sms * 8 ? ctx->n_chunks : ctx->num_sms * 8;
+    const int spec = ctx->spec ? 1 : 0;
+    if ((reinterpret_cast<uintptr_t>(grad) & 15) == 0)
+      k_ef_spec<true><<<chunk_grid, kChunkThreads, 0, st>>>(ctx->e, grad, d, hist1, ctx->sc,
+                                                            ctx->chunk_off, ctx->bk_off,
+                                                            ctx->bk_val, ctx->n_chunks, spec);
+    else
+      k_ef_spec<false><<<chunk_grid, kChunkThreads, 0, st>>>(ctx->e, grad, d, hist1, ctx->sc,
+                                                             ctx->chunk_off, ctx->bk_off,
+                                                             ctx->bk_val, ctx->n_chunks, spec);
+    EFCP_LAUNCHED();
+    const uint32_t spec_limit = uint32_t(std::min<int64_t>(d, 3 * k + 65536));
+    k_pick<kBins1, 1><<<1, 1024, 0, st>>>(hist1, ctx->sc, uint32_t(k), spec, spec_limit);
+    EFCP_LAUNCHED();
+    // candidates: everything at or above the threshold bin, in index order.  The two-pass
+    // kernels return at once when the buckets are good, k_compact_buckets when they are not.
+    k_count_chunks<<<chunk_grid, kChunkThreads, 0, st>>>(ctx->e, d, ctx->sc, ctx->chunk_off,
+                                                         ctx->n_chunks);
+    EFCP_LAUNCHED();
+    k_scan_counts<<<1, 1024, 0, st>>>(ctx->chunk_off, ctx->n_chunks, &ctx->sc->n_cand);
+    EFCP_LAUNCHED();
+    k_compact_cand<<<chunk_grid, kChunkThreads, 0, st>>>(ctx->e, d, ctx->sc, ctx->chunk_off,
+                                                         ctx->cand_idx, ctx->cand_val, hist2,
+                                                         ctx->n_chunks);
+    EFCP_LAUNCHED();
+    k_compact_buckets<<<ctx->num_sms * 4, 256, 0, st>>>(ctx->bk_off, ctx->bk_val, ctx->sc,
+                                                        ctx->chunk_off, ctx->cand_idx,
+                                                        ctx->cand_val, hist2, ctx->n_chunks);
+    EFCP_LAUNCHED();
+    k_pick<kBins2, 2><<<1, 1024, 0, st>>>(hist2, ctx->sc, uint32_t(k));
+    EFCP_LAUNCHED();
+    const int cand_grid = ctx->num_sms * 4;
+    k_hist3<<<cand_grid, 256, 0, st>>>(ctx->cand_val, ctx->sc, hist3);
+    EFCP_LAUNCHED();
+    k_pick<kBins3, 3><<<1, 1024, 0, st>>>(hist3, ctx->sc, uint32_t(k));
+    EFCP_LAUNCHED();
+    // exact selection, ring insert, residual
+    k_count_sel<<<cand_grid, kChunkThreads, 0, st>>>(ctx->cand_val, ctx->sc, ctx->sel_gt,
+                                                     ctx->sel_eq);
+    EFCP_LAUNCHED();
+    k_scan_sel<<<1, 1024, 0, st>>>(ctx->sel_gt, ctx->sel_eq, ctx->sc, uint32_t(k));
+    EFCP_LAUNCHED();
+    k_write_sel<<<cand_grid, kChunkThreads, 0, st>>>(ctx->cand_idx, ctx->cand_val, ctx->sc,
+                                                     ctx->sel_gt, ctx->sel_eq, ctx->sel_idx,
+                                                     ctx->sel_val, ctx->e, k, ctx->V16 ? 1 : 0);
+    EFCP_LAUNCHED();
+  }
   k_row_offsets<<<ctx->num_sms * 4, 256, 0, st>>>(ctx->sel_idx, k, ctx->W, ctx->n_slabs, m, slot,
                                                   ctx->offs, ctx->colsum);
   EFCP_LAUNCHED();
@@ -557,7 +601,7 @@ struct StateHeader {
   int32_t m, W, n_slabs;
   uint32_t flags;
   float lambda;
-  uint32_t pad;
+  uint32_t pad;  // block length of block-wise Top-k (0: global)
 };
 constexpr uint64_t kStateMagic = 0x3130505443464645ull;  // "EFCPTP01"
 
@@ -621,6 +665,7 @@ int efcp_state_export(efcp_ctx* ctx, void* host_buf, int64_t bytes) {
   StateHeader h{};
   h.magic = kStateMagic; h.d = ctx->d; h.k = ctx->k; h.t = ctx->t; h.m = ctx->m; h.W = ctx->W;
   h.n_slabs = ctx->n_slabs; h.flags = ctx->flags; h.lambda = ctx->lambda;
+  h.pad = uint32_t(ctx->block);
   unsigned char* out = static_cast<unsigned char*>(host_buf);
   std::memcpy(out, &h, sizeof(h));
   out += sizeof(h);
@@ -637,6 +682,7 @@ int efcp_state_import(efcp_ctx* ctx, const void* host_buf, int64_t bytes) {
   std::memcpy(&h, host_buf, sizeof(h));
   if (h.magic != kStateMagic || h.d != ctx->d || h.k != ctx->k || h.m != ctx->m ||
       h.W != ctx->W || h.n_slabs != ctx->n_slabs || h.flags != ctx->flags ||
+      h.pad != uint32_t(ctx->block) ||
       std::memcmp(&h.lambda, &ctx->lambda, 4) != 0 || h.t < 0)
     return EFCP_EINVAL;
   EFCP_CUDA(cudaSetDevice(ctx->device));

@@ -46,14 +46,15 @@ def lincomb_amplification(cpu, u_ref):
 
 
 def run_parity(d, m, k, lam, grads, flags=0, check_rows="new", gram_every=0,
-               allow_amplified=False):
+               allow_amplified=False, block=0):
     """grads: iterable of fp32 numpy arrays.  Returns the worst update error seen.
 
     allow_amplified: for deliberately degenerate windows only - the bound becomes
     U_TOL + 8 * 2^-24 * amplification (see lincomb_amplification)."""
     B = _binding()
-    gpu = B.Efcp(d, m, k, lam, flags)
-    cpu = ref.RefEFCP(d, m, k, lam, flags)
+    gpu = B.Efcp(d, m, k, lam, flags, block)
+    cpu = ref.RefEFCP(d, m, k, lam, flags, block)
+    assert gpu.k == cpu.k  # same row length (matters for block-wise Top-k)
     g_dev = torch.empty(d, dtype=torch.float32, device="cuda")
     u_dev = torch.empty(d, dtype=torch.float32, device="cuda")
     worst = 0.0
@@ -167,6 +168,40 @@ def test_bf16_values_cannot_be_combined_with_accumulator_rhs():
     with pytest.raises(B.EfcpError) as ei:
         B.Efcp(100, 2, 10, 1e-3, B.VALUES_BF16 | B.RHS_ACCUMULATOR)
     assert ei.value.code == B.EINVAL
+
+
+# ---- block-wise Top-k (efcp_create_blockwise)
+@pytest.mark.parametrize("d,m,k,block,steps,flags", [
+    (65_536, 8, 655, 16_384, 20, 0),          # whole blocks, steady threshold
+    (100_003, 4, 1000, 4096, 12, 0),          # ragged last block
+    (1_000_001, 8, 10_000, 16_384, 10, 0),
+    (50_000, 4, 500, 32, 6, 0),               # smallest block: one entry per block
+    (300_007, 4, 3000, 8192, 8, 2),           # with bfloat16 values
+    (300_007, 4, 3000, 8192, 8, 1),           # with x = a_t
+    (20_000, 3, 20_000, 1024, 5, 0),          # k = d: every entry kept
+])
+def test_blockwise_topk(d, m, k, block, steps, flags):
+    rng = np.random.default_rng(d + block)
+    scale = np.exp(rng.standard_normal(d))
+    grads = ((scale * rng.standard_normal(d)).astype(np.float32) for _ in range(steps))
+    run_parity(d, m, k, 1e-3, grads, flags=flags, check_rows="all", block=block)
+
+
+def test_blockwise_topk_ties_and_threshold_jumps():
+    d, m, k, block = 40_000, 4, 400, 2048
+    rng = np.random.default_rng(70)
+    grads = [rng.integers(-2, 3, d).astype(np.float32) for _ in range(4)]
+    grads += [(s * rng.standard_normal(d)).astype(np.float32) for s in (1.0, 0.01, 0.01, 50.0, 1.0)]
+    grads += [np.zeros(d, np.float32), np.full(d, 2.5, np.float32)]
+    run_parity(d, m, k, 1e-2, grads, check_rows="all", block=block)
+
+
+def test_blockwise_rejects_bad_block_sizes():
+    B = _binding()
+    for block in (16, 48, 20_000, -32):
+        with pytest.raises(B.EfcpError) as ei:
+            B.Efcp(10_000, 2, 100, 1e-3, 0, block)
+        assert ei.value.code == B.EINVAL
 
 
 def test_heavy_ties():

@@ -27,12 +27,18 @@ def torchrun(script_args, nproc=2, timeout=240):
 
 
 def json_lines(text):
-    out = []
-    for line in text.splitlines():
-        line = line.strip()
-        if line.startswith("{"):
-            out.append(json.loads(line))
-    return out
+    """Every JSON object in the output (two ranks may print on one line)."""
+    out, dec, i = [], json.JSONDecoder(), 0
+    while True:
+        i = text.find("{", i)
+        if i < 0:
+            return out
+        try:
+            obj, end = dec.raw_decode(text, i)
+            out.append(obj)
+            i = end
+        except json.JSONDecodeError:
+            i += 1
 
 
 def test_two_gloo_ranks_barrier_and_max_over_ranks():
