@@ -163,6 +163,17 @@ int efcp_state_import(efcp_ctx* ctx, const void* host_buf, int64_t bytes);
  */
 int efcp_error_norm(efcp_ctx* ctx, double* out);
 
+/*
+ * efcp_validate - consistency check of the window's derived structures (a debugging aid; the
+ * memory checker of the CUDA toolkit is not always available).  For every written row it
+ * verifies on the device that the offset table is monotone and ends at the row length, that
+ * every entry lies in the slab its segment belongs to, that the 16-bit stream agrees with
+ * the indices, and that the slab weights equal the column sums of the offset table.  Waits
+ * for the device.  Returns EFCP_OK, EFCP_EINTERNAL when a check fails (*bad, if not NULL,
+ * receives the number of violations), or the sticky status if that is an error.
+ */
+int efcp_validate(efcp_ctx* ctx, int64_t* bad);
+
 /* Number of completed efcp_step calls on this handle (-1 for a NULL handle). */
 int64_t efcp_step_count(efcp_ctx* ctx);
 

@@ -42,6 +42,7 @@ EXPORTS = {
     "efcp_state_export": ([_vp, _vp, _i64], C.c_int),
     "efcp_state_import": ([_vp, _vp, _i64], C.c_int),
     "efcp_error_norm": ([_vp, _vp], C.c_int),
+    "efcp_validate": ([_vp, _vp], C.c_int),
     "efcp_step_count": ([_vp], _i64),
     "efcp_status": ([_vp], C.c_int),
     "efcp_last_cuda_error": ([_vp], C.c_int),
@@ -228,6 +229,13 @@ class Efcp:
         self._check(_lib.efcp_error_norm(self._h, C.cast(C.byref(out), C.c_void_p)),
                     "efcp_error_norm")
         return float(out.value)
+
+    def validate(self) -> int:
+        """efcp_validate: raises EfcpError when the window's derived structures are
+        inconsistent; returns 0 otherwise."""
+        bad = C.c_int64()
+        self._check(_lib.efcp_validate(self._h, C.cast(C.byref(bad), C.c_void_p)), "efcp_validate")
+        return int(bad.value)
 
     def weights(self) -> np.ndarray:
         out = np.empty(self.m, np.float64)

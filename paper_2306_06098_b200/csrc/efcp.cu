@@ -651,6 +651,65 @@ __global__ void __launch_bounds__(256) k_sum_parts(const double* __restrict__ pa
 
 }  // namespace
 
+namespace {
+
+// One block per (slab, written row): offsets monotone, entries inside the slab, R == I - s W.
+__global__ void __launch_bounds__(128) k_validate_rows(
+    const int32_t* __restrict__ I, const uint16_t* __restrict__ R, const int32_t* __restrict__ offs,
+    int64_t k, int64_t d, int m, int W, int n_slabs, int rows_written,
+    unsigned long long* __restrict__ bad) {
+  const int s = blockIdx.x, r = blockIdx.y;
+  if (r >= rows_written) return;
+  const int b = offs[int64_t(s) * m + r], e = offs[int64_t(s + 1) * m + r];
+  unsigned long long v = 0;
+  if (threadIdx.x == 0) {
+    if (b > e || b < 0 || e > k) ++v;
+    if (s == 0 && b != 0) ++v;
+    if (s == n_slabs - 1 && e != k) ++v;
+  }
+  const int64_t lo = int64_t(s) * W, hi = lo + W < d ? lo + W : d;
+  for (int j = b + threadIdx.x; j < e && j < k; j += blockDim.x) {
+    const int64_t idx = I[int64_t(r) * k + j];
+    if (idx < lo || idx >= hi) ++v;
+    else if (int64_t(R[int64_t(r) * k + j]) != idx - lo) ++v;
+  }
+  if (v) atomicAdd(bad, v);
+}
+
+// colsum[s] == sum over rows of offs[s][r]
+__global__ void __launch_bounds__(256) k_validate_colsum(const int32_t* __restrict__ offs,
+                                                          const int64_t* __restrict__ colsum,
+                                                          int m, int n_slabs,
+                                                          unsigned long long* __restrict__ bad) {
+  __shared__ double sm[32];
+  const int s = blockIdx.x;
+  double acc = 0.0;  // exact: sums stay far below 2^53
+  for (int r = threadIdx.x; r < m; r += blockDim.x) acc += double(offs[int64_t(s) * m + r]);
+  acc = block_sum(acc, sm);
+  if (threadIdx.x == 0 && int64_t(acc) != colsum[s]) atomicAdd(bad, 1ull);
+}
+
+}  // namespace
+
+int efcp_validate(efcp_ctx* ctx, int64_t* bad_out) {
+  if (!ctx) return EFCP_EINVAL;
+  const int rc = sync_status(ctx);
+  if (rc != EFCP_OK) return rc;
+  // scratch: the SP partial buffer is idle between steps
+  unsigned long long* bad = reinterpret_cast<unsigned long long*>(ctx->partial);
+  EFCP_CUDA(cudaMemset(bad, 0, 8));
+  const int rows = int(ctx->t < ctx->m ? ctx->t : ctx->m);
+  if (rows > 0) {
+    k_validate_rows<<<dim3(ctx->n_slabs, rows), 128>>>(ctx->I, ctx->R, ctx->offs, ctx->k, ctx->d,
+                                                       ctx->m, ctx->W, ctx->n_slabs, rows, bad);
+  }
+  k_validate_colsum<<<ctx->n_slabs + 1, 256>>>(ctx->offs, ctx->colsum, ctx->m, ctx->n_slabs, bad);
+  unsigned long long h = 0;
+  EFCP_CUDA(cudaMemcpy(&h, bad, 8, cudaMemcpyDeviceToHost));
+  if (bad_out) *bad_out = int64_t(h);
+  return h ? EFCP_EINTERNAL : EFCP_OK;
+}
+
 int64_t efcp_state_size(efcp_ctx* ctx) {
   if (!ctx) return -1;
   int64_t b = int64_t(sizeof(StateHeader));

@@ -89,6 +89,7 @@ def run_parity(d, m, k, lam, grads, flags=0, check_rows="new", gram_every=0,
             ci, cv = cpu.row(s)
             assert np.array_equal(gi, ci) and np.array_equal(bits(gv), bits(cv))
     assert gpu.step_count == cpu.step_count
+    assert gpu.validate() == 0  # offset table, 16-bit stream and slab weights are consistent
     print(f"parity d={d} m={m} k={k}: worst update rel-L2 {worst:.3e}")
     gpu.close()
     cpu.close()
