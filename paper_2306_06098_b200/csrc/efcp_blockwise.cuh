@@ -5,12 +5,12 @@
 // and written once and nothing but the selection leaves the SM.
 //
 // The selection needs the count-th largest magnitude key T of the block.  T moves little from
-// step to step, so the kernel first gathers the keys at or above (last step's T of this
-// block) - kBlkMargin; when between `count` and kBlkThreads keys qualify, T is found by a
-// 31-step bisection in which every thread holds one key and a step is one
-// __syncthreads_count.  Otherwise (first step, a jump of the threshold) the bisection runs
-// over all keys of the block.  Either way T is exact, and the output is written in index
-// order from per-thread counts and block scans.
+// step to step, so while a is formed the kernel sets aside (in any order) the keys at or
+// above (last step's T of this block) - kBlkMargin; when between `count` and kBlkThreads keys
+// qualify, T is found by a 31-step bisection in which every thread holds one key and a step
+// is one __syncthreads_count.  Otherwise (first step, a jump of the threshold) the bisection
+// runs over all keys of the block.  Either way T is exact, and the output is written in
+// index order from per-thread counts and one block scan.
 #pragma once
 
 #include "efcp_common.cuh"
@@ -39,13 +39,25 @@ __global__ void __launch_bounds__(kBlkThreads) k_ef_block_select(
   float* as = reinterpret_cast<float*>(smraw);  // blk_pad(B) floats
   __shared__ uint32_t ckey[kBlkThreads];
   __shared__ int sm[33];
+  __shared__ int s_nc;  // candidate keys set aside for the current block
   const int tid = threadIdx.x;
   const int64_t c_full = block_count(B, k_req, d);
   bool bad = false;
+  if (tid == 0) s_nc = 0;
   for (int b = blockIdx.x; b < n_blocks; b += gridDim.x) {
     const int64_t b0 = int64_t(b) * B;
     const int len = int(min(int64_t(B), d - b0));
     const int count = int(block_count(len, k_req, d));
+    const uint32_t told = blk_T[b];
+    const uint32_t lower = told > kBlkMargin ? told - kBlkMargin : 0u;
+    auto note = [&](float x) {  // non-finite check; candidate keys go to ckey, unordered
+      const uint32_t key = mag_key(x);
+      bad |= key >= 0x7F800000u;
+      if (told != 0u && key >= lower) {
+        const int slot = atomicAdd(&s_nc, 1);
+        if (slot < kBlkThreads) ckey[slot] = key;
+      }
+    };
     __syncthreads();  // the previous block's shared data is no longer in use
     // ---- a = xi + g, kept in shared memory and written back as the new xi
     if (VEC && (len & 3) == 0) {
@@ -59,12 +71,14 @@ __global__ void __launch_bounds__(kBlkThreads) k_ef_block_select(
         e4[v] = x;
         const int p = blk_pad(4 * v);  // 4 v .. 4 v + 3 lie in one group of 32
         as[p] = x.x; as[p + 1] = x.y; as[p + 2] = x.z; as[p + 3] = x.w;
+        note(x.x); note(x.y); note(x.z); note(x.w);
       }
     } else {
       for (int i = tid; i < len; i += kBlkThreads) {
         const float x = __fadd_rn(e[b0 + i], g[b0 + i]);
         e[b0 + i] = x;
         as[blk_pad(i)] = x;
+        note(x);
       }
     }
     __syncthreads();
@@ -72,23 +86,9 @@ __global__ void __launch_bounds__(kBlkThreads) k_ef_block_select(
     const int ept = (len + kBlkThreads - 1) / kBlkThreads;
     const int lo = min(len, tid * ept), hi = min(len, lo + ept);
     // ---- the count-th largest key T
-    const uint32_t told = blk_T[b];
-    const uint32_t lower = told > kBlkMargin ? told - kBlkMargin : 0u;
-    int mine = 0;
-    for (int i = lo; i < hi; ++i) {
-      const uint32_t key = mag_key(as[blk_pad(i)]);
-      bad |= key >= 0x7F800000u;
-      mine += key >= lower ? 1 : 0;
-    }
-    int n_cand;
-    int pos = block_excl_scan<int>(mine, &n_cand, sm);
+    const int n_cand = s_nc;
     uint32_t T = 0u;
     if (told != 0u && n_cand >= count && n_cand <= kBlkThreads) {
-      for (int i = lo; i < hi; ++i) {
-        const uint32_t key = mag_key(as[blk_pad(i)]);
-        if (key >= lower) ckey[pos++] = key;
-      }
-      __syncthreads();
       const bool have = tid < n_cand;
       const uint32_t key = have ? ckey[tid] : 0u;
       for (int bit = 30; bit >= 0; --bit) {
@@ -112,20 +112,23 @@ __global__ void __launch_bounds__(kBlkThreads) k_ef_block_select(
       gt += key > T ? 1 : 0;
       eq += key == T ? 1 : 0;
     }
-    int n_gt, n_eq_all;
-    (void)block_excl_scan<int>(gt, &n_gt, sm);
-    int eq_before = block_excl_scan<int>(eq, &n_eq_all, sm);
+    // one scan for both counts (each at most 16384: 15 bits)
+    int tot;
+    const int before = block_excl_scan<int>((gt << 16) | eq, &tot, sm);
+    const int n_gt = tot >> 16, n_eq_all = tot & 0xFFFF;
+    const int gt_before = before >> 16, eq_before = before & 0xFFFF;
     const int need_eq = count - n_gt;
     const int my_eq = max(0, min(eq, need_eq - eq_before));
-    int n_sel;
-    int out = block_excl_scan<int>(gt + my_eq, &n_sel, sm);
+    int out = gt_before + max(0, min(eq_before, need_eq));
+    const int n_sel = n_gt + max(0, min(n_eq_all, need_eq));
+    if (tid == 0) s_nc = 0;  // every thread has read it (barriers above); next block starts at 0
     if (tid == 0) {
       blk_T[b] = T;
       if (n_sel != count || need_eq < 0 || need_eq > n_eq_all) atomicOr(&sc->status, kStCount);
     }
     const int64_t row_off = int64_t(b) * c_full;
     int eq_left = my_eq;
-    for (int i = lo; i < hi; ++i) {
+    for (int i = lo; i < hi && gt + my_eq > 0; ++i) {  // most chunks keep nothing
       const float v = as[blk_pad(i)];
       const uint32_t key = mag_key(v);
       bool take = key > T;
