@@ -222,6 +222,24 @@ __device__ __forceinline__ void tail_dispatch(int groups, const uint16_t* pi, co
   }
 }
 
+// Shared -> global bulk copy (TMA, untiled form): both addresses 16-byte aligned, size a
+// multiple of 16.  Used where the method leaves a large contiguous piece to move: a
+// finished slab of the update.  The fence makes the accumulator's generic-proxy writes
+// visible to the copy engine; wait_read returns when the engine has read shared memory
+// (the global writes may still be in flight; they complete before the kernel ends).
+__device__ __forceinline__ void bulk_store_fence() {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void bulk_s2g(void* gdst, const void* ssrc, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst),
+               "r"(uint32_t(__cvta_generic_to_shared(ssrc))), "r"(bytes)
+               : "memory");
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+__device__ __forceinline__ void bulk_store_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+}
+
 // Slab scheduling of the two slab kernels.  Slabs differ in weight (the kept entries
 // cluster where the gradient is large), so blocks do not take a fixed share: block b starts
 // with slab b and then draws the next unprocessed slab from a counter in global memory
@@ -465,7 +483,17 @@ __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_lcg(
     // write the slab out and clear it for the next one
     const int64_t gbase = int64_t(s) * W;
     const int n = int(min(int64_t(W), d - gbase));
-    if (VEC) {
+    if (VEC && (n & 3) == 0) {
+      // the slab is one contiguous, 16-byte aligned piece of u: a single bulk copy (the
+      // copy engine reads shared memory itself) instead of a load and a store per thread
+      if (tid == 0) {
+        bulk_store_fence();
+        bulk_s2g(u + gbase, acc, uint32_t(n) * 4u);
+        bulk_store_wait_read();  // the engine has read the accumulator: it can be cleared
+      }
+      __syncthreads();
+      for (int i = tid; i < (n >> 2); i += blockDim.x) acc4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    } else if (VEC) {
       float4* u4 = reinterpret_cast<float4*>(u + gbase);
       const int nv = n >> 2;
       for (int i = tid; i < nv; i += blockDim.x) {
