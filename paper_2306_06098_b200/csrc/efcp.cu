@@ -27,6 +27,8 @@ struct efcp_ctx {
   int64_t d = 0, k = 0;  // k: entries per window row
   int64_t k_req = 0;     // the k of the create call (block-wise Top-k keeps a little more)
   int block = 0, n_blocks = 0;  // block-wise Top-k: block length in coordinates, number of blocks
+  int blk_resident = 1;         // thread blocks of the block-wise kernel one SM holds
+  int blk_threads = kBlkThreads;  // threads per thread block of the block-wise kernel
   uint32_t* blk_T = nullptr;    // per block: last step's threshold key
   int32_t m = 0;
   float lambda = 0.f;
@@ -199,6 +201,19 @@ inline void prof_mark(efcp_ctx* ctx, int which, cudaStream_t st) {
     cudaEventRecord(ctx->prof_ev[size_t(ctx->prof_n) * 5 + which], st);
 }
 
+// calls f with the instantiation of the block-wise kernel for `threads` threads per block
+template <typename F>
+bool for_block_kernel(int threads, bool aligned, F f) {
+  if (aligned) {
+    if (threads == 128) return f(k_ef_block_select<true, 128>);
+    if (threads == 256) return f(k_ef_block_select<true, 256>);
+    return f(k_ef_block_select<true, 512>);
+  }
+  if (threads == 128) return f(k_ef_block_select<false, 128>);
+  if (threads == 256) return f(k_ef_block_select<false, 256>);
+  return f(k_ef_block_select<false, 512>);
+}
+
 }  // namespace
 
 extern "C" {
@@ -298,8 +313,9 @@ int efcp_create_blockwise(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float
   if ((rc = dev_alloc(ctx, &ctx->wf, int64_t(m) * 4))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->slab_ctr, 256))) return fail(rc);
   if (block) {
-    if ((rc = dev_alloc(ctx, &ctx->blk_T, int64_t(n_blocks) * 4))) return fail(rc);
-    if (cudaMemset(ctx->blk_T, 0, size_t(n_blocks) * 4) != cudaSuccess) return fail(EFCP_ECUDA);
+    // per block: last step's threshold key, then log2 of the candidate margin
+    if ((rc = dev_alloc(ctx, &ctx->blk_T, int64_t(n_blocks) * 8))) return fail(rc);
+    if (cudaMemset(ctx->blk_T, 0, size_t(n_blocks) * 8) != cudaSuccess) return fail(EFCP_ECUDA);
   }
   if ((rc = dev_alloc(ctx, &ctx->colsum, int64_t(z.n_slabs + 1) * 8))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->order, int64_t(z.n_slabs) * 4))) return fail(rc);
@@ -321,9 +337,19 @@ int efcp_create_blockwise(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float
   const size_t smem = slab_smem_bytes(z.W, m);
   const auto attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
   if (block) {
-    const int bs = blk_pad(block) * 4;
-    ok &= cudaFuncSetAttribute(k_ef_block_select<true>, attr, bs) == cudaSuccess;
-    ok &= cudaFuncSetAttribute(k_ef_block_select<false>, attr, bs) == cudaSuccess;
+    const int bs = int(block_select_smem(block));
+    ctx->blk_threads = block_select_threads(block, block_count(block, k_req, d));
+    ok &= for_block_kernel(ctx->blk_threads, true, [&](auto kern) {
+      int resident = 0;
+      bool good = cudaFuncSetAttribute(kern, attr, bs) == cudaSuccess;
+      good &= cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, kern, ctx->blk_threads,
+                                                            bs) == cudaSuccess;
+      ctx->blk_resident = resident > 0 ? resident : 1;
+      return good;
+    });
+    ok &= for_block_kernel(ctx->blk_threads, false, [&](auto kern) {
+      return cudaFuncSetAttribute(kern, attr, bs) == cudaSuccess;
+    });
   }
   ok &= cudaFuncSetAttribute(k_sp_rows<false, float>, attr, int(smem)) == cudaSuccess;
   ok &= cudaFuncSetAttribute(k_sp_rows<true, float>, attr, int(smem)) == cudaSuccess;
@@ -377,16 +403,15 @@ int efcp_step(efcp_ctx* ctx, const float* grad, float* update, void* stream_) {
   prof_mark(ctx, 0, st);
   if (ctx->block) {
     // block-wise Top-k: a = xi + g, the selection and xi = a - c in one kernel
-    const int grid = ctx->n_blocks < ctx->num_sms * 3 ? ctx->n_blocks : ctx->num_sms * 3;
-    const size_t bs = size_t(blk_pad(ctx->block)) * 4;
-    if ((reinterpret_cast<uintptr_t>(grad) & 15) == 0)
-      k_ef_block_select<true><<<grid, kBlkThreads, bs, st>>>(
-          ctx->e, grad, d, ctx->k_req, ctx->block, ctx->n_blocks, ctx->blk_T, ctx->sel_idx,
-          ctx->sel_val, ctx->sc, ctx->V16 ? 1 : 0);
-    else
-      k_ef_block_select<false><<<grid, kBlkThreads, bs, st>>>(
-          ctx->e, grad, d, ctx->k_req, ctx->block, ctx->n_blocks, ctx->blk_T, ctx->sel_idx,
-          ctx->sel_val, ctx->sc, ctx->V16 ? 1 : 0);
+    const size_t bs = block_select_smem(ctx->block);
+    const int grid = std::min(ctx->n_blocks, ctx->num_sms * ctx->blk_resident);
+    for_block_kernel(ctx->blk_threads, (reinterpret_cast<uintptr_t>(grad) & 15) == 0,
+                     [&](auto kern) {
+                       kern<<<grid, ctx->blk_threads, bs, st>>>(
+                           ctx->e, grad, d, ctx->k_req, ctx->block, ctx->n_blocks, ctx->blk_T,
+                           ctx->sel_idx, ctx->sel_val, ctx->sc, ctx->V16 ? 1 : 0);
+                       return true;
+                     });
     EFCP_LAUNCHED();
   } else {
     // a = xi + g, digit-1 histogram, speculative candidate buckets

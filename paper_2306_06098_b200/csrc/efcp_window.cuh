@@ -479,6 +479,7 @@ __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_lcg(
                       });
       }
     }
+    if (VEC) bulk_store_fence();  // every thread's adds, before the barrier that orders them
     __syncthreads();
     // write the slab out and clear it for the next one
     const int64_t gbase = int64_t(s) * W;
@@ -487,7 +488,6 @@ __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_lcg(
       // the slab is one contiguous, 16-byte aligned piece of u: a single bulk copy (the
       // copy engine reads shared memory itself) instead of a load and a store per thread
       if (tid == 0) {
-        bulk_store_fence();
         bulk_s2g(u + gbase, acc, uint32_t(n) * 4u);
         bulk_store_wait_read();  // the engine has read the accumulator: it can be cleared
       }

@@ -197,6 +197,64 @@ def test_blockwise_topk_ties_and_threshold_jumps():
     run_parity(d, m, k, 1e-2, grads, check_rows="all", block=block)
 
 
+def test_blockwise_dense_selection_beyond_one_key_per_thread():
+    # 20 % density: a block keeps more entries than the kernel has threads, so every step
+    # takes the bisection over all keys of the block
+    d, m, k = 65_536, 4, 13_108
+    rng = np.random.default_rng(71)
+    grads = [rng.standard_normal(d).astype(np.float32) for _ in range(5)]
+    run_parity(d, m, k, 1e-3, grads, check_rows="all", block=4096)
+    run_parity(d, m, k, 1e-3, grads, check_rows="all", block=1024)
+
+
+def test_blockwise_crowded_ranges_and_drifting_threshold():
+    # every block has a hot segment of 300 coordinates of nearly equal magnitude (all the
+    # candidates fall into one warp's range, more than its list holds), and the overall scale
+    # decays and recovers so that the threshold leaves the margin in both directions
+    d, m, k, block = 8192 * 6 + 1000, 4, 502, 8192
+    rng = np.random.default_rng(72)
+    hot = np.zeros(d, bool)
+    for b0 in range(0, d, block):
+        hot[b0 + 700:b0 + 1000] = True
+    grads = []
+    for s in (1.0, 1.0, 0.93, 0.6, 0.2, 0.2, 0.21, 3.0, 3.0, 2.9, 1e-3, 1e-3):
+        g = rng.standard_normal(d)
+        g[hot] = 5.0 + 0.01 * rng.standard_normal(int(hot.sum()))
+        grads.append((s * g).astype(np.float32))
+    run_parity(d, m, k, 1e-2, grads, check_rows="all", block=block)
+    run_parity(d, m, k, 1e-2, grads, check_rows="all", block=16_384)
+
+
+def test_blockwise_unaligned_gradient_and_side_stream():
+    B = _binding()
+    d, m, k, block = 70_001, 4, 700, 4096
+    rng = np.random.default_rng(73)
+    gpu = B.Efcp(d, m, k, 1e-3, 0, block)
+    cpu = ref.RefEFCP(d, m, k, 1e-3, 0, block)
+    gbuf = torch.empty(d + 3, dtype=torch.float32, device="cuda")
+    ubuf = torch.empty(d + 3, dtype=torch.float32, device="cuda")
+    side = torch.cuda.Stream()
+    for t in range(6):
+        g = rng.standard_normal(d).astype(np.float32)
+        off = 1 if t % 2 == 0 else 0  # plain loads on even steps, bulk copies on odd ones
+        gv, uv = gbuf[off:d + off], ubuf[3:d + 3]
+        gv.copy_(torch.from_numpy(g))
+        torch.cuda.synchronize()
+        with torch.cuda.stream(side):
+            gpu.step(gv, uv)
+        side.synchronize()
+        u_ref = cpu.step(g)
+        assert gpu.status() == 0
+        assert np.array_equal(bits(gpu.error()), bits(cpu.error())), t
+        gi, gvals = gpu.row(t % m)
+        ci, cvals = cpu.row(t % m)
+        assert np.array_equal(gi, ci) and np.array_equal(bits(gvals), bits(cvals)), t
+        assert rel_l2(uv.cpu().numpy(), u_ref) <= U_TOL
+    assert gpu.validate() == 0
+    gpu.close()
+    cpu.close()
+
+
 def test_blockwise_rejects_bad_block_sizes():
     B = _binding()
     for block in (16, 48, 20_000, -32):
