@@ -164,6 +164,36 @@ int efcp_state_import(efcp_ctx* ctx, const void* host_buf, int64_t bytes);
 int efcp_error_norm(efcp_ctx* ctx, double* out);
 
 /*
+ * The parameter update (last line of the loop of Algorithm 1) with the decoupled weight
+ * decay of Section 2 (the paragraph on the interaction with regularisation):
+ *     theta <- (1 - gamma eta) theta - eta s u,
+ * where s = 1, or, with clipping of the preconditioned gradient's norm as in the
+ * hyper-parameter appendix (clip_norm > 0), s = min(1, clip_norm / |u|_2).
+ *
+ *   efcp_update_norm  : |u|_2 over the d entries of `update` (device; fp64 accumulation in a
+ *                       fixed order), kept on the device for the efcp_apply_update calls
+ *                       that follow.  Asynchronous on `stream` when host_out is NULL;
+ *                       otherwise waits for the stream and stores the norm in *host_out.
+ *   efcp_apply_update : the formula above on n coordinates, theta and update (device, n
+ *                       floats each, any alignment) being the same sub-range of the
+ *                       parameter vector and of u; groups of parameters with their own eta
+ *                       and gamma are separate calls.  With clip_norm > 0, s uses the norm of
+ *                       the last efcp_update_norm call, which has to have been made since the
+ *                       last efcp_step (EFCP_EINVAL otherwise).  fp32 arithmetic: (1 - gamma
+ *                       eta) and eta s are formed in fp64 and rounded once, the update is one
+ *                       multiply and one fused multiply-add per coordinate.  Asynchronous.
+ *   efcp_step_apply   : efcp_step, then efcp_update_norm (if clip_norm > 0) and
+ *                       efcp_apply_update over all d coordinates, on the same stream.
+ *                       `update` still receives u.
+ * eta >= 0, gamma >= 0, clip_norm >= 0 and finite, 1 <= n <= d; EFCP_EINVAL otherwise.
+ */
+int efcp_update_norm(efcp_ctx* ctx, const float* update, double* host_out, void* stream);
+int efcp_apply_update(efcp_ctx* ctx, float* theta, const float* update, int64_t n, float eta,
+                      float gamma, float clip_norm, void* stream);
+int efcp_step_apply(efcp_ctx* ctx, const float* grad, float* theta, float* update, float eta,
+                    float gamma, float clip_norm, void* stream);
+
+/*
  * efcp_validate - consistency check of the window's derived structures (a debugging aid; the
  * memory checker of the CUDA toolkit is not always available).  For every written row it
  * verifies on the device that the offset table is monotone and ends at the row length, that

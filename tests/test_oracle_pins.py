@@ -324,3 +324,61 @@ def test_thread_count_does_not_change_results():
         outs.add(subprocess.run([sys.executable, "-c", code], env=env, check=True,
                                 capture_output=True, text=True).stdout.strip())
     assert len(outs) == 1
+
+
+# ------------------------------------------- parameter update (Algorithm 1, Section 2)
+def test_update_plain_step_and_element_loop():
+    from oracle import wrapper
+    rng = np.random.default_rng(40)
+    theta, u = rng.standard_normal(257), rng.standard_normal(257)
+    eta, gamma = 0.125, 0.5  # exactly representable: no rounding in the scalars
+    got = wrapper.apply_update(theta, u, eta, gamma)
+    want = np.array([(1 - 0.0625) * theta[i] - 0.125 * u[i] for i in range(257)])
+    assert np.allclose(got, want, rtol=0, atol=1e-15)
+    # gamma = 0 is the last line of Algorithm 1's loop
+    assert np.array_equal(wrapper.apply_update(theta, u, eta), theta - 0.125 * u)
+    # eta = 0 leaves the parameters alone
+    assert np.array_equal(wrapper.apply_update(theta, u, 0.0, 0.3, 5.0), theta)
+
+
+def test_update_decoupled_decay_is_gradient_descent_on_the_l2_regularised_loss():
+    # with the identity as preconditioner, u = grad L(theta) and the decoupled rule is
+    # theta - eta (grad L + gamma theta): gradient descent on L + gamma/2 |theta|^2.  On the
+    # quadratic L = 1/2 theta^T A theta - b^T theta it converges to (A + gamma I)^-1 b.
+    from oracle import wrapper
+    rng = np.random.default_rng(41)
+    M = rng.standard_normal((6, 6))
+    A = M @ M.T + np.eye(6)
+    b = rng.standard_normal(6)
+    gamma, eta = 0.25, 0.03125
+    theta = np.zeros(6)
+    for _ in range(4000):
+        theta = wrapper.apply_update(theta, A @ theta - b, eta, gamma)
+    assert np.allclose(theta, np.linalg.solve(A + gamma * np.eye(6), b), rtol=1e-9, atol=1e-12)
+
+
+def test_update_clipping():
+    from oracle import wrapper
+    rng = np.random.default_rng(42)
+    theta, u = rng.standard_normal(1000), 7.0 * rng.standard_normal(1000)
+    nrm = np.linalg.norm(u)
+    assert abs(wrapper.update_norm(u) - nrm) <= 1e-12 * nrm
+    # active: the step has length eta * c exactly, in the direction of -u
+    step = wrapper.apply_update(theta, u, 0.5, 0.0, clip_norm=10.0) - theta
+    assert abs(np.linalg.norm(step) - 5.0) < 1e-12
+    assert np.allclose(step / np.linalg.norm(step), -u / nrm, atol=1e-14)
+    # inactive above the norm, off at 0, harmless for u = 0
+    for c in (0.0, 2.0 * nrm):
+        assert np.array_equal(wrapper.apply_update(theta, u, 0.5, 0.0, c), theta - 0.5 * u)
+    assert wrapper.clip_scale(np.zeros(5), 1.0) == 1.0
+    # a sub-range with the scale of the whole vector equals the slice of the whole update
+    s = wrapper.clip_scale(u, 10.0)
+    whole = wrapper.apply_update(theta, u, 0.5, 0.125, 10.0)
+    part = wrapper.apply_update(theta[100:300], u[100:300], 0.5, 0.125, scale=s)
+    assert np.array_equal(part, whole[100:300])
+
+
+def test_ef_evolution_metric():
+    from oracle import wrapper
+    got = wrapper.ef_evolution([1.0, 1.0, 3.0], [2.0, 2.0, 2.0])
+    assert np.allclose(got, [0.5, 0.25, 0.5])
