@@ -208,6 +208,11 @@ def main():
     ap.add_argument("--block", type=int, default=0,
                     help="block-wise Top-k with blocks of this many coordinates (Section 3.1 "
                          "'Sparsity Pattern'); 0 = global Top-k, the default")
+    ap.add_argument("--apply-update", action="store_true",
+                    help="time efcp_step_apply: the step plus theta <- (1 - gamma eta) theta - "
+                         "eta s u on a resident parameter vector (eta 1e-3, gamma 1e-4)")
+    ap.add_argument("--clip", type=float, default=0.0,
+                    help="with --apply-update: clip |u| to this norm (adds the norm kernels)")
     ap.add_argument("--prefill", type=int, default=-1,
                     help="untimed steps before warm-up; -1 = m (fill the whole window)")
     ap.add_argument("--e2e-steps", type=int, default=5)
@@ -242,6 +247,14 @@ def main():
     gbuf = torch.empty(w.d, dtype=torch.float32, device=device)
     ubuf = torch.empty(w.d, dtype=torch.float32, device=device)
 
+    theta = torch.randn(w.d, dtype=torch.float32, device=device) if args.apply_update else None
+
+    def one_step(g, stream=None):
+        if theta is None:
+            opt.step(g, ubuf, stream)
+        else:
+            opt.step_apply(g, theta, ubuf, 1e-3, 1e-4, args.clip, stream)
+
     prefill = w.m if args.prefill < 0 else args.prefill
     for _ in range(prefill):
         gs.next(out=gbuf)
@@ -256,7 +269,7 @@ def main():
     torch.cuda.empty_cache()
 
     for i in range(W):
-        opt.step(pool[i % pool_n], ubuf)
+        one_step(pool[i % pool_n])
     torch.cuda.synchronize()
     barrier(world)
     try:  # nvidia-smi numbering ignores CUDA_VISIBLE_DEVICES: address the GPU by UUID
@@ -272,7 +285,7 @@ def main():
     torch.cuda.synchronize()
     ev0.record(stream)
     for i in range(K):
-        opt.step(pool[(W + i) % pool_n], ubuf, stream)
+        one_step(pool[(W + i) % pool_n], stream)
     ev1.record(stream)
     torch.cuda.synchronize()
     barrier(world)
@@ -326,8 +339,12 @@ def main():
                 "avg_launch_ms": avg_ms,
                 "moved": {"bytes_per_launch": mov[kern], "achieved": moved, "frac": moved / peak}}
     step_bytes = 2 * (4 + val_b) * mk + 16 * w.d + 8 * w.k + 2 * xi_read
-    step_gbs = step_bytes / (ms_per_step * 1e-3) / 1e9
     step_moved = 2 * (2 + val_b) * mk + 16 * w.d + 10 * w.k + 2 * xi_read
+    if args.apply_update:  # theta read and written, u read; the norm reads u once more
+        extra = 12 * w.d + (4 * w.d if args.clip > 0 else 0)
+        step_bytes += extra
+        step_moved += extra
+    step_gbs = step_bytes / (ms_per_step * 1e-3) / 1e9
     step_moved_gbs = step_moved / (ms_per_step * 1e-3) / 1e9
     stage_ms = {s: stages[s] / max(n_rec, 1) for s in stages}
 
@@ -349,6 +366,8 @@ def main():
                        "rhs": args.rhs, "window_values": args.values,
                        "topk": f"blockwise({args.block})" if args.block else "global",
                        "prefill_steps": prefill,
+                       "parameter_update": (f"efcp_step_apply (eta 1e-3, gamma 1e-4, clip "
+                                            f"{args.clip:g})" if args.apply_update else "none"),
                        "parallelism": f"replicas x{world}",
                        "l2": "inputs larger than L2 (window %.2f GB, gradient %.2f GB)" % (
                            8 * w.m * w.k / 1e9, 4 * w.d / 1e9)},

@@ -42,6 +42,9 @@ EXPORTS = {
     "efcp_state_export": ([_vp, _vp, _i64], C.c_int),
     "efcp_state_import": ([_vp, _vp, _i64], C.c_int),
     "efcp_error_norm": ([_vp, _vp], C.c_int),
+    "efcp_update_norm": ([_vp, _vp, _vp, _vp], C.c_int),
+    "efcp_apply_update": ([_vp, _vp, _vp, _i64, _f32, _f32, _f32, _vp], C.c_int),
+    "efcp_step_apply": ([_vp, _vp, _vp, _vp, _f32, _f32, _f32, _vp], C.c_int),
     "efcp_validate": ([_vp, _vp], C.c_int),
     "efcp_step_count": ([_vp], _i64),
     "efcp_status": ([_vp], C.c_int),
@@ -229,6 +232,42 @@ class Efcp:
         self._check(_lib.efcp_error_norm(self._h, C.cast(C.byref(out), C.c_void_p)),
                     "efcp_error_norm")
         return float(out.value)
+
+    def update_norm(self, update: torch.Tensor, sync: bool = True, stream=None):
+        """efcp_update_norm: |u|_2, kept on the device for apply_update; returned when sync."""
+        assert update.is_cuda and update.dtype == torch.float32 and update.is_contiguous()
+        assert update.numel() == self.d
+        s = torch.cuda.current_stream() if stream is None else stream
+        out = C.c_double()
+        self._check(_lib.efcp_update_norm(self._h, update.data_ptr(),
+                                          C.cast(C.byref(out), C.c_void_p) if sync else None,
+                                          s.cuda_stream), "efcp_update_norm")
+        return float(out.value) if sync else None
+
+    def apply_update(self, theta: torch.Tensor, update: torch.Tensor, eta: float,
+                     gamma: float = 0.0, clip_norm: float = 0.0, stream=None):
+        """efcp_apply_update on the same sub-range of the parameters and of u (device, fp32,
+        contiguous, equal lengths <= d); asynchronous."""
+        assert theta.is_cuda and update.is_cuda and theta.dtype == update.dtype == torch.float32
+        assert theta.is_contiguous() and update.is_contiguous()
+        assert theta.numel() == update.numel()
+        s = torch.cuda.current_stream() if stream is None else stream
+        self._check(_lib.efcp_apply_update(self._h, theta.data_ptr(), update.data_ptr(),
+                                           theta.numel(), eta, gamma, clip_norm, s.cuda_stream),
+                    "efcp_apply_update")
+        return theta
+
+    def step_apply(self, grad: torch.Tensor, theta: torch.Tensor, update: torch.Tensor,
+                   eta: float, gamma: float = 0.0, clip_norm: float = 0.0, stream=None):
+        """efcp_step_apply: one optimizer step including the parameter update; asynchronous."""
+        for t in (grad, theta, update):
+            assert t.is_cuda and t.dtype == torch.float32 and t.is_contiguous()
+            assert t.numel() == self.d
+        s = torch.cuda.current_stream() if stream is None else stream
+        self._check(_lib.efcp_step_apply(self._h, grad.data_ptr(), theta.data_ptr(),
+                                         update.data_ptr(), eta, gamma, clip_norm,
+                                         s.cuda_stream), "efcp_step_apply")
+        return theta
 
     def validate(self) -> int:
         """efcp_validate: raises EfcpError when the window's derived structures are

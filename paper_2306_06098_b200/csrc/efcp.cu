@@ -17,6 +17,7 @@
 
 #include "efcp_common.cuh"
 #include "efcp_blockwise.cuh"
+#include "efcp_update.cuh"
 #include "efcp_mxm.cuh"
 #include "efcp_topk.cuh"
 #include "efcp_window.cuh"
@@ -28,6 +29,8 @@ struct efcp_ctx {
   int64_t k_req = 0;     // the k of the create call (block-wise Top-k keeps a little more)
   int block = 0, n_blocks = 0;  // block-wise Top-k: block length in coordinates, number of blocks
   int blk_resident = 1;         // thread blocks of the block-wise kernel one SM holds
+  double* upd_norm = nullptr;   // [0]: |u|^2 of the last efcp_update_norm, then its partial sums
+  int64_t norm_t = -1;          // step count at that call
   int blk_threads = kBlkThreads;  // threads per thread block of the block-wise kernel
   uint32_t* blk_T = nullptr;    // per block: last step's threshold key
   int32_t m = 0;
@@ -308,6 +311,7 @@ int efcp_create_blockwise(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float
   if ((rc = dev_alloc(ctx, &ctx->sc, sizeof(Scalars)))) return fail(rc);
   const int64_t sums = (flags & EFCP_RHS_ACCUMULATOR) ? 2 : 1;
   if ((rc = dev_alloc(ctx, &ctx->slab_part, int64_t(z.n_slabs) * m * 8 * sums))) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->upd_norm, int64_t(kUpdMaxBlocks + 1) * 8))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->partial, int64_t(kSpParts) * m * 8 * sums))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->vecs, int64_t(9) * m * 8))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->wf, int64_t(m) * 4))) return fail(rc);
@@ -542,6 +546,66 @@ int efcp_step(efcp_ctx* ctx, const float* grad, float* update, void* stream_) {
   return EFCP_OK;
 }
 
+int efcp_update_norm(efcp_ctx* ctx, const float* update, double* host_out, void* stream_) {
+  if (!ctx || !update) return EFCP_EINVAL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream_);
+  EFCP_CUDA(cudaSetDevice(ctx->device));
+  const int64_t want = (ctx->d + 8 * kUpdThreads - 1) / (8 * kUpdThreads);
+  const int nb = int(std::max<int64_t>(1, std::min<int64_t>({want, int64_t(ctx->num_sms) * 8,
+                                                             int64_t(kUpdMaxBlocks)})));
+  if ((reinterpret_cast<uintptr_t>(update) & 15) == 0)
+    k_update_sumsq<true><<<nb, kUpdThreads, 0, st>>>(update, ctx->d, ctx->upd_norm + 1);
+  else
+    k_update_sumsq<false><<<nb, kUpdThreads, 0, st>>>(update, ctx->d, ctx->upd_norm + 1);
+  EFCP_LAUNCHED();
+  k_sum_parts<<<1, 256, 0, st>>>(ctx->upd_norm + 1, nb, ctx->upd_norm);
+  EFCP_LAUNCHED();
+  ctx->norm_t = ctx->t;
+  if (host_out) {
+    double s = 0.0;
+    EFCP_CUDA(cudaMemcpyAsync(&s, ctx->upd_norm, 8, cudaMemcpyDeviceToHost, st));
+    EFCP_CUDA(cudaStreamSynchronize(st));
+    *host_out = std::sqrt(s);
+  }
+  return EFCP_OK;
+}
+
+int efcp_apply_update(efcp_ctx* ctx, float* theta, const float* update, int64_t n, float eta,
+                      float gamma, float clip_norm, void* stream_) {
+  if (!ctx || !theta || !update || theta == update || n < 1 || n > ctx->d) return EFCP_EINVAL;
+  if (!(eta >= 0.f) || !(gamma >= 0.f) || !(clip_norm >= 0.f) || std::isinf(eta) ||
+      std::isinf(gamma) || std::isinf(clip_norm))
+    return EFCP_EINVAL;
+  if (clip_norm > 0.f && ctx->norm_t != ctx->t) return EFCP_EINVAL;  // no norm of this step's u
+  cudaStream_t st = static_cast<cudaStream_t>(stream_);
+  EFCP_CUDA(cudaSetDevice(ctx->device));
+  const float decay = float(1.0 - double(gamma) * double(eta));
+  const int64_t want = (n + 4 * kUpdThreads - 1) / (4 * kUpdThreads);
+  const int nb = int(std::max<int64_t>(1, std::min<int64_t>(want, int64_t(ctx->num_sms) * 16)));
+  const bool vec = ((reinterpret_cast<uintptr_t>(theta) | reinterpret_cast<uintptr_t>(update)) & 15) == 0;
+  if (vec)
+    k_apply_update<true><<<nb, kUpdThreads, 0, st>>>(theta, update, n, decay, double(eta),
+                                                     double(clip_norm), ctx->upd_norm);
+  else
+    k_apply_update<false><<<nb, kUpdThreads, 0, st>>>(theta, update, n, decay, double(eta),
+                                                      double(clip_norm), ctx->upd_norm);
+  EFCP_LAUNCHED();
+  return EFCP_OK;
+}
+
+int efcp_step_apply(efcp_ctx* ctx, const float* grad, float* theta, float* update, float eta,
+                    float gamma, float clip_norm, void* stream_) {
+  if (!ctx || !theta || theta == grad) return EFCP_EINVAL;
+  if (!(eta >= 0.f) || !(gamma >= 0.f) || !(clip_norm >= 0.f) || std::isinf(eta) ||
+      std::isinf(gamma) || std::isinf(clip_norm))
+    return EFCP_EINVAL;  // before the step: a rejected call leaves the state untouched
+  int rc = efcp_step(ctx, grad, update, stream_);
+  if (rc != EFCP_OK) return rc;
+  if (clip_norm > 0.f && (rc = efcp_update_norm(ctx, update, nullptr, stream_)) != EFCP_OK) return rc;
+  rc = efcp_apply_update(ctx, theta, update, ctx->d, eta, gamma, clip_norm, stream_);
+  return rc;
+}
+
 int efcp_step_host(efcp_ctx* ctx, const float* grad, float* update, void* stream_) {
   if (!ctx || !grad || !update) return EFCP_EINVAL;
   cudaStream_t st = static_cast<cudaStream_t>(stream_);
@@ -665,15 +729,6 @@ __global__ void __launch_bounds__(256) k_sumsq(const float* __restrict__ e, int6
   acc = block_sum(acc, sm);
   if (threadIdx.x == 0) part[blockIdx.x] = acc;
 }
-__global__ void __launch_bounds__(256) k_sum_parts(const double* __restrict__ part, int n,
-                                                    double* __restrict__ out) {
-  __shared__ double sm[32];
-  double acc = 0.0;
-  for (int i = threadIdx.x; i < n; i += blockDim.x) acc += part[i];
-  acc = block_sum(acc, sm);
-  if (threadIdx.x == 0) *out = acc;
-}
-
 }  // namespace
 
 namespace {
