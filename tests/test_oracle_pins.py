@@ -382,3 +382,82 @@ def test_ef_evolution_metric():
     from oracle import wrapper
     got = wrapper.ef_evolution([1.0, 1.0, 3.0], [2.0, 2.0, 2.0])
     assert np.allclose(got, [0.5, 0.25, 0.5])
+
+
+# ------------------------------------------------------------- Sparse GGT (appendix)
+def _ggt_definition(rows, x, eps):
+    """((sum_i c_i c_i^T)^(1/2) + eps I)^-1 x with a dense d x d eigendecomposition."""
+    C = np.asarray(rows, np.float64)
+    lam, Q = np.linalg.eigh(C.T @ C)
+    root = np.sqrt(np.maximum(lam, 0.0))
+    return Q @ ((Q.T @ x) / (root + eps))
+
+
+def test_ggt_matches_the_dense_definition():
+    from oracle import ggt
+    d, m, k, eps = 120, 5, 12, 0.05
+    rng = np.random.default_rng(50)
+    o = ggt.RefSparseGGT(d, m, k, eps)
+    sim = DenseSim(d, m, k, 1.0)  # for the window only: its own solve is not used
+    for t in range(13):  # the window fills and wraps twice
+        g = rng.standard_normal(d).astype(np.float32)
+        u = o.step(g)
+        sim.step(g)
+        rows = sim.G[:min(t + 1, m)]
+        x = sim.G[t % m]
+        want = _ggt_definition(rows, x, np.float64(np.float32(eps)))
+        assert rel(u, want) < 1e-6, t
+    o.close()
+
+
+def test_ggt_closed_forms():
+    from oracle import ggt
+    d, eps = 64, 0.25
+    rng = np.random.default_rng(51)
+    # m = 1: the window is x alone and u = x / (|x| + eps)
+    o = ggt.RefSparseGGT(d, 1, 8, eps)
+    for _ in range(3):
+        u = o.step(rng.standard_normal(d).astype(np.float32))
+        idx, val = o.row(0)
+        x = np.zeros(d)
+        x[idx] = val
+        assert rel(u, x / (np.linalg.norm(x) + eps)) < 1e-6
+    o.close()
+    # rows with disjoint supports are orthogonal: again u = x / (|x| + eps)
+    o = ggt.RefSparseGGT(d, 4, 4, eps)
+    for t in range(4):
+        g = np.zeros(d, np.float32)
+        g[8 * t:8 * t + 4] = 1.0 + rng.random(4)
+        u = o.step(g)
+        assert rel(u, g / (np.linalg.norm(g.astype(np.float64)) + eps)) < 1e-6
+    o.close()
+    # a repeated row (rank-deficient window): c c^T counted twice, u = x / (sqrt(2) |x| + eps)
+    o = ggt.RefSparseGGT(d, 3, 4, eps)
+    g = np.zeros(d, np.float32)
+    g[:4] = (1.0, -2.0, 3.0, 0.5)
+    o.step(g)
+    u = o.step(g)  # the error buffer is zero on the kept entries, so the same row again
+    assert rel(u, g / (np.sqrt(2.0) * np.linalg.norm(g.astype(np.float64)) + eps)) < 1e-6
+    o.close()
+
+
+def test_ggt_large_eps_limit_and_scaling():
+    from oracle import ggt
+    d, m, k = 80, 4, 8
+    rng = np.random.default_rng(52)
+    grads = [rng.standard_normal(d).astype(np.float32) for _ in range(6)]
+    big = ggt.RefSparseGGT(d, m, k, 1e6)
+    for g in grads:
+        u = big.step(g)
+    idx, val = big.row((len(grads) - 1) % m)
+    x = np.zeros(d)
+    x[idx] = val
+    assert rel(u * 1e6, x) < 1e-4  # eps -> infinity: u -> x / eps
+    big.close()
+    # (G G^T)^(1/2) is homogeneous of degree 1: scaling gradients and eps by s leaves u unchanged
+    a, b = ggt.RefSparseGGT(d, m, k, 0.125), ggt.RefSparseGGT(d, m, k, 0.5)
+    for g in grads:
+        ua, ub = a.step(g), b.step(4.0 * g)
+        assert rel(ua, ub.astype(np.float64)) < 1e-6
+    a.close()
+    b.close()
