@@ -2,7 +2,7 @@
  * efcp.h - C ABI of the B200 (sm_100a) EFCP / Sparse M-FAC step library.
  *
  * One handle owns the whole optimizer state of one parameter vector of
- * dimension d on one GPU: the error-feedback buffer xi (Algorithm 1, line 2),
+ * dimension d on one GPU: the error-feedback buffer xi (Algorithm 1),
  * the sparse ring buffer G = (I, V) of the last m compressed accumulators
  * (Section 3.1, "Sparsity format for G"), the m x m scalar-product matrix
  * S = G G^T (Section 2.1, "Scalar Products (SP)") and the inverse of
@@ -40,7 +40,7 @@ typedef struct efcp_ctx efcp_ctx;
 
 /* flags for efcp_create_ex */
 #define EFCP_RHS_COMPRESSED  0u /* u_t = A(c_t): precondition the compressed accumulator
-                                   (Algorithm 1, line 8) - the default                    */
+                                   (Algorithm 1) - the default                             */
 #define EFCP_RHS_ACCUMULATOR 1u /* precondition the full accumulator a_t = xi_t + c_t
                                    (u = F^-1 a_t; costs one more read of xi in SP and LCG)  */
 
@@ -51,8 +51,21 @@ typedef struct efcp_ctx efcp_ctx;
                                    then read 4 bytes per window entry instead of 6.  Cannot
                                    be combined with EFCP_RHS_ACCUMULATOR.                   */
 
+#define EFCP_PRECOND_GGT     4u /* Sparse GGT instead of Sparse M-FAC (appendix "Sparse GGT"):
+                                   u_t = ((sum_i c_i c_i^T)^(1/2) + eps I)^-1 c_t over the
+                                   window rows c_i, with eps passed in the `lambda` argument.
+                                   Error feedback, Top-k, the window and the scalar products
+                                   are unchanged; the m x m stage becomes a symmetric
+                                   eigendecomposition, held in one SM's shared memory, which
+                                   limits m to 112.  Not with EFCP_RHS_ACCUMULATOR (GGT
+                                   preconditions the compressed accumulator).  For this mode
+                                   efcp_get_weights returns the coefficients of u over the
+                                   window rows and efcp_last_residual the relative
+                                   off-diagonal norm the eigendecomposition stopped at;
+                                   EFCP_ENUMERIC means it did not converge.                  */
+
 /*
- * efcp_create / efcp_create_ex - Algorithm 1 lines 1-2: set up an empty window and
+ * efcp_create / efcp_create_ex - the initialisation of Algorithm 1: set up an empty window and
  * xi_0 = 0 for dimension d, window length m, k kept entries per step (Top-k of
  * Section 3.1, k given as a count) and damping lambda (F_0 = lambda I, Section 2.1).
  * Requires 1 <= k <= d < 2^31, 1 <= m <= 4096, lambda finite and > 0.
@@ -80,7 +93,7 @@ int efcp_create_blockwise(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float
 int64_t efcp_row_length(efcp_ctx* ctx);
 
 /*
- * efcp_step - Algorithm 1 lines 5-8 for one gradient:
+ * efcp_step - the body of Algorithm 1's loop for one gradient, without the parameter update:
  *     a = xi + g                      (fp32, one rounding per coordinate)
  *     c = TopK_k(a)                   (global over d, exact, ties to the lower index)
  *     xi = a - c                      (kept coordinates become +0)
@@ -92,7 +105,7 @@ int64_t efcp_row_length(efcp_ctx* ctx);
  *   update device, d floats, every element overwritten; must not alias grad.
  *   stream a cudaStream_t (NULL = default stream).  All work is enqueued on it and
  *          the call returns without waiting.  Learning rate, weight decay and the
- *          parameter update (Algorithm 1 line 9) are left to the caller.
+ *          parameter update are left to the caller (or to efcp_apply_update).
  * Errors detected on the device (EFCP_ENUMERIC, ...) are sticky and reported by
  * efcp_status or the next efcp_get_* call.
  */
@@ -232,7 +245,7 @@ int32_t efcp_launches_per_step(efcp_ctx* ctx);
  *   efcp_profile_end   : waits for the device, adds up the elapsed times of the steps
  *                        recorded since efcp_profile_begin and stops recording.
  *                        ms_out (host, 4 doubles) receives the totals in milliseconds:
- *                        [0] error feedback + Top-k + ring insert (Algorithm 1 lines 5-7),
+ *                        [0] error feedback + Top-k + ring insert (Algorithm 1),
  *                        [1] the scalar-product (SP) kernel alone,
  *                        [2] the m x m stage,
  *                        [3] the linear-combination (LCG) kernel alone;

@@ -8,7 +8,7 @@
 // smoke check and the CPU-baseline leg of the benchmark may use it.
 //
 // What each function follows:
-//   * step 1-3 (error feedback, Top-k compress, residual): Algorithm 1 lines 5-7
+//   * step 1-3 (error feedback, Top-k compress, residual): Algorithm 1, the error-feedback, compression and error-update statements
 //     and the "Overview" paragraph of Section 3.
 //   * Top-k: Section 3.1 (keep the k largest-magnitude entries as index/value
 //     pairs).  Global over d, ties go to the lower index, pairs stored by
@@ -29,7 +29,7 @@
 //   * linear combination of gradients: Section 2.1 "LCG" and Eq. (2).
 //   * optional bfloat16 window values: Section 3.1 "Format for V".  Reading taken (the paper
 //     only says the optimizer still converges with bfloat16 values): Compress returns the
-//     selected values rounded to bfloat16, and line 7 of Algorithm 1 is applied to that c,
+//     selected values rounded to bfloat16, and the error update of Algorithm 1 is applied to that c,
 //     so the rounding residue is fed back like any other compression error.
 //
 // Precision: the state (error buffer, window) is fp32 exactly as the method
@@ -337,11 +337,11 @@ int efcp_ref_step(efcp_ref* h, const float* grad, float* update) {
   const int32_t m = o->m;
   const double lambda = double(o->lambda);
 
-  // Algorithm 1 line 5: a = xi + g, one fp32 add per coordinate.
+  // Algorithm 1, error feedback: a = xi + g, one fp32 add per coordinate.
   // (built with -ffp-contract=off and without fast-math.)
   for (int64_t j = 0; j < d; ++j) o->a[size_t(j)] = o->e[size_t(j)] + grad[j];
 
-  // Algorithm 1 line 6: c = TopK(a); the row goes into ring slot i.
+  // Algorithm 1, compression: c = TopK(a); the row goes into ring slot i.
   const int32_t i = int32_t(o->t % m);
   int32_t* idx = &o->I[size_t(i) * size_t(k)];
   float* val = &o->V[size_t(i) * size_t(k)];
@@ -365,7 +365,7 @@ int efcp_ref_step(efcp_ref* h, const float* grad, float* update) {
   if (o->flags & kFlagValuesBf16)
     for (int64_t r = 0; r < k; ++r) val[r] = round_to_bf16(val[r]);
 
-  // Algorithm 1 line 7: xi = a - c.  At a kept coordinate a - a is +0; with rounded values
+  // Algorithm 1, error update: xi = a - c.  At a kept coordinate a - a is +0; with rounded values
   // the rounding residue a - bf16(a) (exact in fp32) stays in the error buffer.
   o->e = o->a;
   for (int64_t r = 0; r < k; ++r)

@@ -18,6 +18,7 @@
 #include "efcp_common.cuh"
 #include "efcp_blockwise.cuh"
 #include "efcp_update.cuh"
+#include "efcp_ggt.cuh"
 #include "efcp_mxm.cuh"
 #include "efcp_topk.cuh"
 #include "efcp_window.cuh"
@@ -256,8 +257,10 @@ int efcp_create_blockwise(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float
   if (!out) return EFCP_EINVAL;
   *out = nullptr;
   if (!valid_args(d, m, k) || !(lambda > 0.f) || !std::isfinite(lambda)) return EFCP_EINVAL;
-  if (flags & ~(EFCP_RHS_ACCUMULATOR | EFCP_VALUES_BF16)) return EFCP_EINVAL;
+  if (flags & ~(EFCP_RHS_ACCUMULATOR | EFCP_VALUES_BF16 | EFCP_PRECOND_GGT)) return EFCP_EINVAL;
   if ((flags & EFCP_RHS_ACCUMULATOR) && (flags & EFCP_VALUES_BF16)) return EFCP_EINVAL;
+  if ((flags & EFCP_PRECOND_GGT) && ((flags & EFCP_RHS_ACCUMULATOR) || m > kGgtMaxM))
+    return EFCP_EINVAL;
   if (block != 0 && (block < 32 || block > kBlkMax || (block & 31))) return EFCP_EINVAL;
   const int64_t k_req = k;
   int n_blocks = 0;
@@ -355,6 +358,8 @@ int efcp_create_blockwise(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float
       return cudaFuncSetAttribute(kern, attr, bs) == cudaSuccess;
     });
   }
+  if (flags & EFCP_PRECOND_GGT)
+    ok &= cudaFuncSetAttribute(k_ggt_weights, attr, int(ggt_smem_bytes(m))) == cudaSuccess;
   ok &= cudaFuncSetAttribute(k_sp_rows<false, float>, attr, int(smem)) == cudaSuccess;
   ok &= cudaFuncSetAttribute(k_sp_rows<true, float>, attr, int(smem)) == cudaSuccess;
   ok &= cudaFuncSetAttribute(k_sp_rows<false, bf16raw>, attr, int(smem)) == cudaSuccess;
@@ -500,6 +505,12 @@ int efcp_step(efcp_ctx* ctx, const float* grad, float* update, void* stream_) {
                                                aprime, acc_mode ? rhs : nullptr,
                                                double(ctx->lambda));
   EFCP_LAUNCHED();
+  if (ctx->flags & EFCP_PRECOND_GGT) {
+    // m x m: eigendecomposition of S and the weights of u over the window rows
+    k_ggt_weights<<<1, kGgtThreads, ggt_smem_bytes(m), st>>>(ctx->S, m, slot, double(ctx->lambda),
+                                                             w, ctx->wf, ctx->sc);
+    EFCP_LAUNCHED();
+  } else {
   // m x m: remove-and-border update of the inverse, weights, one refinement step
   const int gemv_grid = (m + 7) / 8;
   k_gemv<<<gemv_grid, 256, 0, st>>>(ctx->B, aprime, y, m);
@@ -520,6 +531,7 @@ int efcp_step(efcp_ctx* ctx, const float* grad, float* update, void* stream_) {
   EFCP_LAUNCHED();
   k_refine_finish<<<1, 1024, 0, st>>>(w, dw, res, ctx->wf, m, ctx->sc);
   EFCP_LAUNCHED();
+  }
   // linear combination of the window rows
   prof_mark(ctx, 3, st);
   const bool uvec = (reinterpret_cast<uintptr_t>(update) & 15) == 0;

@@ -1,4 +1,4 @@
-// Error feedback + exact global Top-k (Algorithm 1 lines 5-7, Section 3.1).
+// Error feedback + exact global Top-k (Algorithm 1: the error-feedback, compression and error-update statements; Section 3.1).
 //
 // Selection is a most-significant-digit radix select on the 31-bit magnitude key
 // (12 + 10 + 9 bits).  Digit 1 is histogrammed while a = xi + g is formed; every

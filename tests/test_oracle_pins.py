@@ -61,7 +61,7 @@ def test_topk_rejects_bad_arguments():
         ref.topk(a, 0)
 
 
-# ------------------------------------------- error feedback (Algorithm 1, lines 5-7)
+# ------------------------------------------- error feedback (Algorithm 1)
 def test_error_feedback_invariant_bitwise():
     rng = np.random.default_rng(3)
     d, m, k = 3001, 4, 37
