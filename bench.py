@@ -205,6 +205,8 @@ def main():
                     help="precondition c_t (Algorithm 1, default) or the whole accumulator a_t")
     ap.add_argument("--values", default="fp32", choices=["fp32", "bf16"],
                     help="window value format (bf16: Section 3.1 'Format for V', not the default)")
+    ap.add_argument("--precond", default="mfac", choices=["mfac", "ggt"],
+                    help="ggt: Sparse GGT (appendix), lambda of the workload is its eps; m <= 112")
     ap.add_argument("--block", type=int, default=0,
                     help="block-wise Top-k with blocks of this many coordinates (Section 3.1 "
                          "'Sparsity Pattern'); 0 = global Top-k, the default")
@@ -240,7 +242,8 @@ def main():
     bf16 = args.values == "bf16"
     opt = binding.Efcp(w.d, w.m, w.k, w.lam,
                        (binding.RHS_ACCUMULATOR if acc else binding.RHS_COMPRESSED) |
-                       (binding.VALUES_BF16 if bf16 else 0), args.block)
+                       (binding.VALUES_BF16 if bf16 else 0) |
+                       (binding.PRECOND_GGT if args.precond == "ggt" else 0), args.block)
     if args.block:  # rows are a little longer than k: count the bytes of what is really kept
         w = gradgen.Workload(w.name, w.d, w.m, opt.k, w.lam, w.steps, w.rank, w.scale_block,
                              w.seed, w.noise)
@@ -364,6 +367,7 @@ def main():
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": w.name, "d": w.d, "m": w.m, "k": w.k, "lambda": w.lam,
                        "rhs": args.rhs, "window_values": args.values,
+                       "preconditioner": {"mfac": "Sparse M-FAC", "ggt": "Sparse GGT"}[args.precond],
                        "topk": f"blockwise({args.block})" if args.block else "global",
                        "prefill_steps": prefill,
                        "parameter_update": (f"efcp_step_apply (eta 1e-3, gamma 1e-4, clip "

@@ -30,6 +30,8 @@ struct efcp_ctx {
   int64_t k_req = 0;     // the k of the create call (block-wise Top-k keeps a little more)
   int block = 0, n_blocks = 0;  // block-wise Top-k: block length in coordinates, number of blocks
   int blk_resident = 1;         // thread blocks of the block-wise kernel one SM holds
+  double* ggt_V = nullptr;      // Sparse GGT: eigenvectors of the last step's S (m x m)
+  double* ggt_T = nullptr;      // and an (m+1) x (m+1) scratch matrix
   double* upd_norm = nullptr;   // [0]: |u|^2 of the last efcp_update_norm, then its partial sums
   int64_t norm_t = -1;          // step count at that call
   int blk_threads = kBlkThreads;  // threads per thread block of the block-wise kernel
@@ -315,6 +317,10 @@ int efcp_create_blockwise(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float
   const int64_t sums = (flags & EFCP_RHS_ACCUMULATOR) ? 2 : 1;
   if ((rc = dev_alloc(ctx, &ctx->slab_part, int64_t(z.n_slabs) * m * 8 * sums))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->upd_norm, int64_t(kUpdMaxBlocks + 1) * 8))) return fail(rc);
+  if (flags & EFCP_PRECOND_GGT) {
+    if ((rc = dev_alloc(ctx, &ctx->ggt_V, int64_t(m) * m * 8))) return fail(rc);
+    if ((rc = dev_alloc(ctx, &ctx->ggt_T, int64_t(m + 1) * (m + 1) * 8))) return fail(rc);
+  }
   if ((rc = dev_alloc(ctx, &ctx->partial, int64_t(kSpParts) * m * 8 * sums))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->vecs, int64_t(9) * m * 8))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->wf, int64_t(m) * 4))) return fail(rc);
@@ -341,6 +347,7 @@ int efcp_create_blockwise(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float
   ok &= cudaMemset(ctx->wf, 0, size_t(m) * 4) == cudaSuccess;
   k_init_rows<<<ctx->num_sms * 4, 256>>>(ctx->I, k, mk);
   k_init_identity<<<ctx->num_sms * 2, 256>>>(ctx->B, m, 1.0 / (double(m) * double(lambda)));
+  if (ctx->ggt_V) k_init_identity<<<ctx->num_sms * 2, 256>>>(ctx->ggt_V, m, 1.0);
   const size_t smem = slab_smem_bytes(z.W, m);
   const auto attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
   if (block) {
@@ -508,7 +515,8 @@ int efcp_step(efcp_ctx* ctx, const float* grad, float* update, void* stream_) {
   if (ctx->flags & EFCP_PRECOND_GGT) {
     // m x m: eigendecomposition of S and the weights of u over the window rows
     k_ggt_weights<<<1, kGgtThreads, ggt_smem_bytes(m), st>>>(ctx->S, m, slot, double(ctx->lambda),
-                                                             w, ctx->wf, ctx->sc);
+                                                             w, ctx->wf, ctx->sc, ctx->ggt_V,
+                                                             ctx->ggt_T);
     EFCP_LAUNCHED();
   } else {
   // m x m: remove-and-border update of the inverse, weights, one refinement step
