@@ -206,7 +206,7 @@ def main():
     ap.add_argument("--values", default="fp32", choices=["fp32", "bf16"],
                     help="window value format (bf16: Section 3.1 'Format for V', not the default)")
     ap.add_argument("--precond", default="mfac", choices=["mfac", "ggt"],
-                    help="ggt: Sparse GGT (appendix), lambda of the workload is its eps; m <= 112")
+                    help="ggt: Sparse GGT (appendix), lambda of the workload is its eps; m <= 160")
     ap.add_argument("--block", type=int, default=0,
                     help="block-wise Top-k with blocks of this many coordinates (Section 3.1 "
                          "'Sparsity Pattern'); 0 = global Top-k, the default")

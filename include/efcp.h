@@ -57,7 +57,7 @@ typedef struct efcp_ctx efcp_ctx;
                                    Error feedback, Top-k, the window and the scalar products
                                    are unchanged; the m x m stage becomes a symmetric
                                    eigendecomposition, held in one SM's shared memory, which
-                                   limits m to 112.  Not with EFCP_RHS_ACCUMULATOR (GGT
+                                   limits m to 160.  Not with EFCP_RHS_ACCUMULATOR (GGT
                                    preconditions the compressed accumulator).  For this mode
                                    efcp_get_weights returns the coefficients of u over the
                                    window rows and efcp_last_residual the relative

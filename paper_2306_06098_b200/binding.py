@@ -16,7 +16,7 @@ LIB_PATH = os.path.join(_HERE, "csrc", "libefcp.so")
 OK, EINVAL, ENOMEM, ECUDA, ENUMERIC, ETIMEOUT, EINTERNAL, ETOOBIG = 0, -1, -2, -3, -4, -5, -6, -7
 TOPK_STATIC_MAX_D = 1 << 20
 RHS_COMPRESSED, RHS_ACCUMULATOR, VALUES_BF16, PRECOND_GGT = 0, 1, 2, 4
-GGT_MAX_M = 112
+GGT_MAX_M = 160
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(

@@ -30,8 +30,7 @@ struct efcp_ctx {
   int64_t k_req = 0;     // the k of the create call (block-wise Top-k keeps a little more)
   int block = 0, n_blocks = 0;  // block-wise Top-k: block length in coordinates, number of blocks
   int blk_resident = 1;         // thread blocks of the block-wise kernel one SM holds
-  double* ggt_V = nullptr;      // Sparse GGT: eigenvectors of the last step's S (m x m)
-  double* ggt_T = nullptr;      // and an (m+1) x (m+1) scratch matrix
+  double2* ggt_rot = nullptr;   // Sparse GGT: the rotations of one step's eigendecomposition
   double* upd_norm = nullptr;   // [0]: |u|^2 of the last efcp_update_norm, then its partial sums
   int64_t norm_t = -1;          // step count at that call
   int blk_threads = kBlkThreads;  // threads per thread block of the block-wise kernel
@@ -318,8 +317,7 @@ int efcp_create_blockwise(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float
   if ((rc = dev_alloc(ctx, &ctx->slab_part, int64_t(z.n_slabs) * m * 8 * sums))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->upd_norm, int64_t(kUpdMaxBlocks + 1) * 8))) return fail(rc);
   if (flags & EFCP_PRECOND_GGT) {
-    if ((rc = dev_alloc(ctx, &ctx->ggt_V, int64_t(m) * m * 8))) return fail(rc);
-    if ((rc = dev_alloc(ctx, &ctx->ggt_T, int64_t(m + 1) * (m + 1) * 8))) return fail(rc);
+    if ((rc = dev_alloc(ctx, &ctx->ggt_rot, ggt_log_entries(m) * 16))) return fail(rc);
   }
   if ((rc = dev_alloc(ctx, &ctx->partial, int64_t(kSpParts) * m * 8 * sums))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->vecs, int64_t(9) * m * 8))) return fail(rc);
@@ -347,7 +345,6 @@ int efcp_create_blockwise(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float
   ok &= cudaMemset(ctx->wf, 0, size_t(m) * 4) == cudaSuccess;
   k_init_rows<<<ctx->num_sms * 4, 256>>>(ctx->I, k, mk);
   k_init_identity<<<ctx->num_sms * 2, 256>>>(ctx->B, m, 1.0 / (double(m) * double(lambda)));
-  if (ctx->ggt_V) k_init_identity<<<ctx->num_sms * 2, 256>>>(ctx->ggt_V, m, 1.0);
   const size_t smem = slab_smem_bytes(z.W, m);
   const auto attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
   if (block) {
@@ -366,7 +363,8 @@ int efcp_create_blockwise(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float
     });
   }
   if (flags & EFCP_PRECOND_GGT)
-    ok &= cudaFuncSetAttribute(k_ggt_weights, attr, int(ggt_smem_bytes(m))) == cudaSuccess;
+    ok &= cudaFuncSetAttribute(ggt_slots(m) <= 2 ? k_ggt_weights<2> : k_ggt_weights<4>, attr,
+                               int(ggt_smem_bytes(m))) == cudaSuccess;
   ok &= cudaFuncSetAttribute(k_sp_rows<false, float>, attr, int(smem)) == cudaSuccess;
   ok &= cudaFuncSetAttribute(k_sp_rows<true, float>, attr, int(smem)) == cudaSuccess;
   ok &= cudaFuncSetAttribute(k_sp_rows<false, bf16raw>, attr, int(smem)) == cudaSuccess;
@@ -514,9 +512,12 @@ int efcp_step(efcp_ctx* ctx, const float* grad, float* update, void* stream_) {
   EFCP_LAUNCHED();
   if (ctx->flags & EFCP_PRECOND_GGT) {
     // m x m: eigendecomposition of S and the weights of u over the window rows
-    k_ggt_weights<<<1, kGgtThreads, ggt_smem_bytes(m), st>>>(ctx->S, m, slot, double(ctx->lambda),
-                                                             w, ctx->wf, ctx->sc, ctx->ggt_V,
-                                                             ctx->ggt_T);
+    if (ggt_slots(m) <= 2)
+      k_ggt_weights<2><<<1, kGgtThreads, ggt_smem_bytes(m), st>>>(
+          ctx->S, m, slot, double(ctx->lambda), w, ctx->wf, ctx->sc, ctx->ggt_rot);
+    else
+      k_ggt_weights<4><<<1, kGgtThreads, ggt_smem_bytes(m), st>>>(
+          ctx->S, m, slot, double(ctx->lambda), w, ctx->wf, ctx->sc, ctx->ggt_rot);
     EFCP_LAUNCHED();
   } else {
   // m x m: remove-and-border update of the inverse, weights, one refinement step

@@ -48,7 +48,7 @@ def run_ggt(d, m, k, eps, grads, flags=0, block=0):
         err = rel_l2(u, u_ref)
         worst = max(worst, err)
         assert err <= U_TOL, f"update rel-L2 {err:.3e} at step {t}"
-        assert gpu.last_residual() <= 1e-14  # off-diagonal norm the eigendecomposition reached
+        assert gpu.last_residual() <= 1e-13  # off-diagonal norm the eigendecomposition reached
         # the scalar products are those of the oracle's window
         Sg = gpu.gram()
         assert np.allclose(Sg, cpu.S, rtol=1e-12, atol=1e-12 * np.abs(cpu.S).max())
@@ -64,7 +64,8 @@ def run_ggt(d, m, k, eps, grads, flags=0, block=0):
     (20_000, 7, 200, 0.05, 20),      # odd m (padded pairing), the window wraps twice
     (100_003, 32, 1000, 0.01, 40),   # several slabs, ragged tail
     (272_474, 100, 2725, 0.01, 12),  # the paper's GGT setting: ResNet-20 size, m = 100, 1 %
-    (50_000, 112, 500, 0.02, 8),     # the largest window the mode takes
+    (50_000, 160, 500, 0.02, 6),     # the largest window the mode takes
+    (30_000, 113, 300, 0.02, 4),     # odd m above 112
 ])
 def test_ggt_parity(d, m, k, eps, steps):
     rng = np.random.default_rng(d + m)
@@ -94,7 +95,7 @@ def test_ggt_rank_deficient_window():
 
 def test_ggt_argument_errors():
     B = _binding()
-    for args in ((1000, 113, 10, 0.1, B.PRECOND_GGT),
+    for args in ((1000, 161, 10, 0.1, B.PRECOND_GGT),
                  (1000, 8, 10, 0.1, B.PRECOND_GGT | B.RHS_ACCUMULATOR),
                  (1000, 8, 10, 0.0, B.PRECOND_GGT)):
         with pytest.raises(B.EfcpError) as ei:
