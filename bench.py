@@ -130,10 +130,24 @@ def max_over_ranks(x, world, device):
     return float(t.item())
 
 
-def oracle_steps_per_sec(w, grads_host, n_steps):
+def make_oracle(d, m, k, lam, precond):
+    """The CPU oracle of the preconditioner being timed (None when it cannot hold the case:
+    the Sparse GGT oracle keeps a dense m x d window)."""
+    from oracle import ref
+    if precond == "ggt":
+        if d * m * 8 > (4 << 30):
+            return None
+        from oracle import ggt
+        return ggt.RefSparseGGT(d, m, k, lam)
+    return ref.RefEFCP(d, m, k, lam)
+
+
+def oracle_steps_per_sec(w, grads_host, n_steps, precond="mfac"):
     """Times the CPU oracle as it stands on `n_steps` gradients of workload w."""
     from oracle import ref
-    o = ref.RefEFCP(w.d, w.m, w.k, w.lam)
+    o = make_oracle(w.d, w.m, w.k, w.lam, precond)
+    if o is None:
+        return None
     t0 = time.perf_counter()
     for i in range(n_steps):
         o.step(grads_host[i % len(grads_host)])
@@ -159,7 +173,11 @@ def run_reference(args, world, rank):
     small = gradgen.Workload(w.name, d, w.m, k, w.lam, w.steps, w.rank, w.scale_block, w.seed)
     gs = gradgen.GradStream.for_workload(small, "cpu")
     from oracle import ref
-    o = ref.RefEFCP(d, w.m, k, w.lam)
+    o = make_oracle(d, w.m, k, w.lam, args.precond)
+    if o is None:
+        print(json.dumps({"impl": "reference",
+                          "unavailable": "the Sparse GGT oracle keeps a dense m x d window"}))
+        return
     grads = [gs.next().numpy() for _ in range(min(4, args.steps + args.warmup))]
     for i in range(args.warmup):
         o.step(grads[i % len(grads)])
@@ -175,7 +193,8 @@ def run_reference(args, world, rank):
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": 1e3 / value, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "d": w.d, "m": w.m, "k": w.k, "lambda": w.lam},
+        "config": {"workload": w.name, "d": w.d, "m": w.m, "k": w.k, "lambda": w.lam,
+                   "preconditioner": {"mfac": "Sparse M-FAC", "ggt": "Sparse GGT"}[args.precond]},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": ref.num_threads(),
                          "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -354,11 +373,13 @@ def main():
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline and args.cpu_steps > 0:
         grads_host = [pool[i].cpu().numpy() for i in range(min(2, pool_n))]
-        v, cores, dt = oracle_steps_per_sec(w, grads_host, args.cpu_steps)
-        cpu_baseline = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
-                        "sample": f"{args.cpu_steps} full steps of {w.name} from an empty window "
-                                  f"(the oracle loops over all m rows whether written or not), "
-                                  f"{dt:.1f} s"}
+        timed = oracle_steps_per_sec(w, grads_host, args.cpu_steps, args.precond)
+        if timed is not None:
+            v, cores, dt = timed
+            cpu_baseline = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
+                            "sample": f"{args.cpu_steps} full steps of {w.name} from an empty "
+                                      f"window (the oracle loops over all m rows whether written "
+                                      f"or not), {dt:.1f} s"}
 
     if rank == 0:
         line = {
