@@ -232,6 +232,9 @@ def main():
     ap.add_argument("--apply-update", action="store_true",
                     help="time efcp_step_apply: the step plus theta <- (1 - gamma eta) theta - "
                          "eta s u on a resident parameter vector (eta 1e-3, gamma 1e-4)")
+    ap.add_argument("--no-u", action="store_true",
+                    help="with --apply-update and no clipping: do not materialise u (the linear "
+                         "combination updates theta directly)")
     ap.add_argument("--clip", type=float, default=0.0,
                     help="with --apply-update: clip |u| to this norm (adds the norm kernels)")
     ap.add_argument("--prefill", type=int, default=-1,
@@ -275,7 +278,7 @@ def main():
         if theta is None:
             opt.step(g, ubuf, stream)
         else:
-            opt.step_apply(g, theta, ubuf, 1e-3, 1e-4, args.clip, stream)
+            opt.step_apply(g, theta, None if args.no_u else ubuf, 1e-3, 1e-4, args.clip, stream)
 
     prefill = w.m if args.prefill < 0 else args.prefill
     for _ in range(prefill):
@@ -363,7 +366,7 @@ def main():
     step_bytes = 2 * (4 + val_b) * mk + 16 * w.d + 8 * w.k + 2 * xi_read
     step_moved = 2 * (2 + val_b) * mk + 16 * w.d + 10 * w.k + 2 * xi_read
     if args.apply_update:  # theta read and written, u read; the norm reads u once more
-        extra = 12 * w.d + (4 * w.d if args.clip > 0 else 0)
+        extra = (4 * w.d if args.no_u else 12 * w.d) + (4 * w.d if args.clip > 0 else 0)
         step_bytes += extra
         step_moved += extra
     step_gbs = step_bytes / (ms_per_step * 1e-3) / 1e9
@@ -392,7 +395,8 @@ def main():
                        "topk": f"blockwise({args.block})" if args.block else "global",
                        "prefill_steps": prefill,
                        "parameter_update": (f"efcp_step_apply (eta 1e-3, gamma 1e-4, clip "
-                                            f"{args.clip:g})" if args.apply_update else "none"),
+                                            f"{args.clip:g}{', u not materialised' if args.no_u else ''})"
+                                            if args.apply_update else "none"),
                        "parallelism": f"replicas x{world}",
                        "l2": "inputs larger than L2 (window %.2f GB, gradient %.2f GB)" % (
                            8 * w.m * w.k / 1e9, 4 * w.d / 1e9)},

@@ -196,8 +196,12 @@ int efcp_error_norm(efcp_ctx* ctx, double* out);
  *                       eta) and eta s are formed in fp64 and rounded once, the update is one
  *                       multiply and one fused multiply-add per coordinate.  Asynchronous.
  *   efcp_step_apply   : efcp_step, then efcp_update_norm (if clip_norm > 0) and
- *                       efcp_apply_update over all d coordinates, on the same stream.
- *                       `update` still receives u.
+ *                       efcp_apply_update over all d coordinates, on the same stream;
+ *                       `update` receives u.  With update == NULL (and clip_norm == 0,
+ *                       EFCP_EINVAL otherwise: clipping needs |u| before any of it is applied)
+ *                       u is never written: the linear combination updates theta slab by
+ *                       slab from shared memory, which saves the write and one read of u.
+ *                       The arithmetic per coordinate is the same.
  * eta >= 0, gamma >= 0, clip_norm >= 0 and finite, 1 <= n <= d; EFCP_EINVAL otherwise.
  */
 int efcp_update_norm(efcp_ctx* ctx, const float* update, double* host_out, void* stream);

@@ -258,16 +258,18 @@ class Efcp:
                     "efcp_apply_update")
         return theta
 
-    def step_apply(self, grad: torch.Tensor, theta: torch.Tensor, update: torch.Tensor,
-                   eta: float, gamma: float = 0.0, clip_norm: float = 0.0, stream=None):
-        """efcp_step_apply: one optimizer step including the parameter update; asynchronous."""
-        for t in (grad, theta, update):
+    def step_apply(self, grad: torch.Tensor, theta: torch.Tensor, update, eta: float,
+                   gamma: float = 0.0, clip_norm: float = 0.0, stream=None):
+        """efcp_step_apply: one optimizer step including the parameter update; asynchronous.
+        update=None (only without clipping): u is not materialised, the linear combination
+        updates theta directly."""
+        for t in (grad, theta) + (() if update is None else (update,)):
             assert t.is_cuda and t.dtype == torch.float32 and t.is_contiguous()
             assert t.numel() == self.d
         s = torch.cuda.current_stream() if stream is None else stream
         self._check(_lib.efcp_step_apply(self._h, grad.data_ptr(), theta.data_ptr(),
-                                         update.data_ptr(), eta, gamma, clip_norm,
-                                         s.cuda_stream), "efcp_step_apply")
+                                         None if update is None else update.data_ptr(), eta,
+                                         gamma, clip_norm, s.cuda_stream), "efcp_step_apply")
         return theta
 
     def validate(self) -> int:

@@ -392,8 +392,10 @@ int efcp_destroy(efcp_ctx* ctx) {
   return EFCP_OK;
 }
 
-int efcp_step(efcp_ctx* ctx, const float* grad, float* update, void* stream_) {
-  if (!ctx || !grad || !update || grad == update) return EFCP_EINVAL;
+// One step; with ap.theta set the linear combination updates the parameters in place of
+// writing u (update may then be NULL).
+static int step_impl(efcp_ctx* ctx, const float* grad, float* update, void* stream_, LcgApply ap) {
+  if (!ctx || !grad || (!update && !ap.theta) || grad == update) return EFCP_EINVAL;
   cudaStream_t st = static_cast<cudaStream_t>(stream_);
   const int64_t d = ctx->d, k = ctx->k;
   const int m = ctx->m;
@@ -548,7 +550,7 @@ int efcp_step(efcp_ctx* ctx, const float* grad, float* update, void* stream_) {
 #define EFCP_LCG_LAUNCH(VEC, ACC, VT, VPTR)                                                    \
   k_lcg<VEC, ACC, VT><<<ctx->grid_slab, kSlabThreads, smem, st>>>(                             \
       ctx->R, VPTR, ctx->offs, k, m, ctx->W, ctx->n_slabs, ctx->wf, update, d,                 \
-      ctx->slab_ctr + 1, ctx->order, ctx->e, inv_lambda)
+      ctx->slab_ctr + 1, ctx->order, ctx->e, inv_lambda, ap)
   if (ctx->V16) {
     if (uvec) EFCP_LCG_LAUNCH(true, false, bf16raw, ctx->V16);
     else EFCP_LCG_LAUNCH(false, false, bf16raw, ctx->V16);
@@ -565,6 +567,11 @@ int efcp_step(efcp_ctx* ctx, const float* grad, float* update, void* stream_) {
   if (ctx->prof_on && ctx->prof_n < ctx->prof_cap) ++ctx->prof_n;
   ctx->t += 1;
   return EFCP_OK;
+}
+
+int efcp_step(efcp_ctx* ctx, const float* grad, float* update, void* stream) {
+  if (!update) return EFCP_EINVAL;
+  return step_impl(ctx, grad, update, stream, LcgApply{nullptr, 0.f, 0.f});
 }
 
 int efcp_update_norm(efcp_ctx* ctx, const float* update, double* host_out, void* stream_) {
@@ -620,6 +627,12 @@ int efcp_step_apply(efcp_ctx* ctx, const float* grad, float* theta, float* updat
   if (!(eta >= 0.f) || !(gamma >= 0.f) || !(clip_norm >= 0.f) || std::isinf(eta) ||
       std::isinf(gamma) || std::isinf(clip_norm))
     return EFCP_EINVAL;  // before the step: a rejected call leaves the state untouched
+  if (!update) {
+    // nobody wants u: the linear combination applies it to theta slab by slab
+    if (clip_norm > 0.f) return EFCP_EINVAL;  // clipping needs |u| before any of it is applied
+    const float decay = float(1.0 - double(gamma) * double(eta));
+    return step_impl(ctx, grad, nullptr, stream_, LcgApply{theta, decay, -eta});
+  }
   int rc = efcp_step(ctx, grad, update, stream_);
   if (rc != EFCP_OK) return rc;
   if (clip_norm > 0.f && (rc = efcp_update_norm(ctx, update, nullptr, stream_)) != EFCP_OK) return rc;

@@ -417,12 +417,19 @@ __global__ void __launch_bounds__(128) k_sp_finish(const double* __restrict__ pa
 // shared-memory accumulator (Eq. (2) in the form that has no x/lambda term, see
 // efcp_mxm.cuh).  Every element of u is written exactly once.
 // With ACC (x = a_t) the accumulator of a slab starts from xi_t / lambda instead of zero.
+// The parameter update fused into the write-out of the linear combination (theta == nullptr:
+// off, u is written instead): theta <- decay theta + neg_step u.
+struct LcgApply {
+  float* theta;
+  float decay, neg_step;
+};
+
 template <bool VEC, bool ACC, typename VT>
 __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_lcg(
     const uint16_t* __restrict__ R, const VT* __restrict__ V, const int32_t* __restrict__ offs,
     int64_t k, int m, int W, int n_slabs, const float* __restrict__ wf, float* __restrict__ u,
     int64_t d, int* ctr, const int32_t* __restrict__ order, const float* __restrict__ xi,
-    float inv_lambda) {
+    float inv_lambda, LcgApply ap) {
   extern __shared__ __align__(16) unsigned char smraw[];
   float* acc = reinterpret_cast<float*>(smraw);
   float* wc = reinterpret_cast<float*>(smraw + size_t(W) * 4);
@@ -484,7 +491,29 @@ __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_lcg(
     // write the slab out and clear it for the next one
     const int64_t gbase = int64_t(s) * W;
     const int n = int(min(int64_t(W), d - gbase));
-    if (VEC && (n & 3) == 0) {
+    if (ap.theta != nullptr) {
+      // the parameter update takes the finished slab of u straight from shared memory:
+      // theta <- decay theta + (-eta) u; u itself is not written
+      float* th = ap.theta + gbase;
+      if ((reinterpret_cast<uintptr_t>(th) & 15) == 0 && (n & 3) == 0) {
+        float4* th4 = reinterpret_cast<float4*>(th);
+        for (int i = tid; i < (n >> 2); i += blockDim.x) {
+          float4 t4 = th4[i];
+          const float4 a4 = acc4[i];
+          t4.x = __fmaf_rn(ap.neg_step, a4.x, __fmul_rn(ap.decay, t4.x));
+          t4.y = __fmaf_rn(ap.neg_step, a4.y, __fmul_rn(ap.decay, t4.y));
+          t4.z = __fmaf_rn(ap.neg_step, a4.z, __fmul_rn(ap.decay, t4.z));
+          t4.w = __fmaf_rn(ap.neg_step, a4.w, __fmul_rn(ap.decay, t4.w));
+          th4[i] = t4;
+          acc4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+      } else {
+        for (int i = tid; i < n; i += blockDim.x) {
+          th[i] = __fmaf_rn(ap.neg_step, acc[i], __fmul_rn(ap.decay, th[i]));
+          acc[i] = 0.f;
+        }
+      }
+    } else if (VEC && (n & 3) == 0) {
       // the slab is one contiguous, 16-byte aligned piece of u: a single bulk copy (the
       // copy engine reads shared memory itself) instead of a load and a store per thread
       if (tid == 0) {

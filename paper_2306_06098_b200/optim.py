@@ -67,7 +67,8 @@ class SparseMFAC(torch.optim.Optimizer):
 
     @property
     def last_update(self) -> torch.Tensor:
-        """u_t of the last step (flat, device)."""
+        """u_t of the last step (flat, device); not written when there is one parameter group
+        and no clipping (the update is then applied without materialising u)."""
         return self._u
 
     @torch.no_grad()
@@ -87,8 +88,10 @@ class SparseMFAC(torch.optim.Optimizer):
                 off += n
         groups = self.param_groups
         if len(groups) == 1:
-            self._h.step_apply(self._g, self._theta, self._u, float(groups[0]["lr"]),
-                               float(groups[0]["weight_decay"]), self._clip)
+            # without clipping nobody needs u: the library applies it to theta as it forms
+            self._h.step_apply(self._g, self._theta, self._u if self._clip > 0 else None,
+                               float(groups[0]["lr"]), float(groups[0]["weight_decay"]),
+                               self._clip)
         else:
             self._h.step(self._g, self._u)
             if self._clip > 0:

@@ -159,3 +159,39 @@ def test_torch_optimizer_front_end():
     # parameters are views of one flat vector: the model sees the library's in-place update
     assert all(p.data_ptr() >= opt._theta.data_ptr() for p in order)
     cpu.close()
+
+
+@pytest.mark.parametrize("flags_name,block,off", [("", 0, 0), ("", 0, 1), ("RHS_ACCUMULATOR", 0, 0),
+                                                   ("VALUES_BF16", 4096, 0)])
+def test_step_apply_without_materialising_u(flags_name, block, off):
+    """update = NULL: the linear combination updates theta slab by slab."""
+    B = _binding()
+    flags = getattr(B, flags_name) if flags_name else 0
+    d, m, k, lam = 150_001, 6, 1500, 1e-3
+    eta, gamma = 0.03, 0.02
+    rng = np.random.default_rng(8)
+    gpu = B.Efcp(d, m, k, lam, flags, block)
+    cpu = ref.RefEFCP(d, m, k, lam, flags, block)
+    theta = rng.standard_normal(d).astype(np.float32)
+    tbuf = torch.empty(d + 1, device="cuda")
+    t_dev = tbuf[off:d + off]  # off = 1: a parameter vector that is not 16-byte aligned
+    t_dev.copy_(torch.from_numpy(theta))
+    g_dev = torch.empty(d, device="cuda")
+    for t in range(9):
+        g = rng.standard_normal(d).astype(np.float32)
+        g_dev.copy_(torch.from_numpy(g))
+        before = t_dev.cpu().numpy()
+        gpu.step_apply(g_dev, t_dev, None, eta, gamma)
+        u_ref = cpu.step(g)
+        want = wrapper.apply_update(before, u_ref, eta, gamma)
+        got = t_dev.cpu().numpy().astype(np.float64)
+        step_len = np.linalg.norm(want - before)
+        assert np.linalg.norm(got - want) <= 1e-4 * step_len + 4 * EPS * np.linalg.norm(want), t
+        assert np.array_equal(gpu.error().view(np.uint32), cpu.error().view(np.uint32))
+    assert gpu.status() == 0 and gpu.validate() == 0
+    with pytest.raises(B.EfcpError) as ei:  # clipping needs u
+        gpu.step_apply(g_dev, t_dev, None, eta, gamma, 1.0)
+    assert ei.value.code == B.EINVAL
+    assert gpu.step_count == 9  # the rejected call did not step
+    gpu.close()
+    cpu.close()
