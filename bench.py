@@ -226,6 +226,9 @@ def main():
                     help="window value format (bf16: Section 3.1 'Format for V', not the default)")
     ap.add_argument("--precond", default="mfac", choices=["mfac", "ggt"],
                     help="ggt: Sparse GGT (appendix), lambda of the workload is its eps; m <= 160")
+    ap.add_argument("--lcg", default="fixed", choices=["fixed", "fp32"],
+                    help="accumulator of the linear combination: int32 fixed point with an fp32 "
+                         "fallback per slab (the library's default) or fp32 atomics (EFCP_LCG_FP32)")
     ap.add_argument("--block", type=int, default=0,
                     help="block-wise Top-k with blocks of this many coordinates (Section 3.1 "
                          "'Sparsity Pattern'); 0 = global Top-k, the default")
@@ -265,7 +268,8 @@ def main():
     opt = binding.Efcp(w.d, w.m, w.k, w.lam,
                        (binding.RHS_ACCUMULATOR if acc else binding.RHS_COMPRESSED) |
                        (binding.VALUES_BF16 if bf16 else 0) |
-                       (binding.PRECOND_GGT if args.precond == "ggt" else 0), args.block)
+                       (binding.PRECOND_GGT if args.precond == "ggt" else 0) |
+                       (binding.LCG_FP32 if args.lcg == "fp32" else 0), args.block)
     if args.block:  # rows are a little longer than k: count the bytes of what is really kept
         w = gradgen.Workload(w.name, w.d, w.m, opt.k, w.lam, w.steps, w.rank, w.scale_block,
                              w.seed, w.noise)
@@ -391,6 +395,9 @@ def main():
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": w.name, "d": w.d, "m": w.m, "k": w.k, "lambda": w.lam,
                        "rhs": args.rhs, "window_values": args.values,
+                       "lcg_accumulator": ("int32 fixed point, fp32 fallback per slab (%d slabs "
+                                           "fell back)" % opt.fixed_point_fallbacks()
+                                           if args.lcg == "fixed" and not acc else "fp32"),
                        "preconditioner": {"mfac": "Sparse M-FAC", "ggt": "Sparse GGT"}[args.precond],
                        "topk": f"blockwise({args.block})" if args.block else "global",
                        "prefill_steps": prefill,

@@ -64,6 +64,21 @@ typedef struct efcp_ctx efcp_ctx;
                                    off-diagonal norm the eigendecomposition stopped at;
                                    EFCP_ENUMERIC means it did not converge.                  */
 
+#define EFCP_LCG_FP32        8u /* The linear combination (Section 2.1 "LCG", Section 3.1 "Sparse
+                                   LCG") accumulates a slab of u in shared memory.  By default
+                                   the accumulator is int32 fixed point: the shared-memory adds
+                                   cost less than half of fp32 ones, and a slab's result does
+                                   not depend on the order of the adds.  The scale of a slab
+                                   comes from a bound that excludes overflow; a slab whose
+                                   rounding error (estimated from the number of entries and
+                                   the step of the grid) could exceed 1e-5 of its norm is
+                                   accumulated again in fp32, so the update stays within the
+                                   same 1e-4 of the exact one (efcp_fixed_point_fallbacks
+                                   counts those slabs).  This flag selects fp32 atomic adds
+                                   for every slab instead.  EFCP_RHS_ACCUMULATOR always uses
+                                   fp32 adds.  The choice is not part of the state: a state
+                                   exported with one setting imports into the other.          */
+
 /*
  * efcp_create / efcp_create_ex - the initialisation of Algorithm 1: set up an empty window and
  * xi_0 = 0 for dimension d, window length m, k kept entries per step (Top-k of
@@ -238,6 +253,10 @@ double efcp_last_residual(efcp_ctx* ctx);
 
 /* Device bytes a handle for (d, m, k) allocates (state + scratch); -1 if invalid. */
 int64_t efcp_state_bytes(int64_t d, int32_t m, int64_t k);
+
+/* Slabs of the update that the fixed-point accumulator handed to fp32 since the handle was
+ * created (0 with EFCP_LCG_FP32, -1 for a NULL handle or a CUDA error).  Waits for the device. */
+int64_t efcp_fixed_point_fallbacks(efcp_ctx* ctx);
 
 /* Number of kernels one efcp_step launches for this handle. */
 int32_t efcp_launches_per_step(efcp_ctx* ctx);

@@ -15,7 +15,7 @@ LIB_PATH = os.path.join(_HERE, "csrc", "libefcp.so")
 
 OK, EINVAL, ENOMEM, ECUDA, ENUMERIC, ETIMEOUT, EINTERNAL, ETOOBIG = 0, -1, -2, -3, -4, -5, -6, -7
 TOPK_STATIC_MAX_D = 1 << 20
-RHS_COMPRESSED, RHS_ACCUMULATOR, VALUES_BF16, PRECOND_GGT = 0, 1, 2, 4
+RHS_COMPRESSED, RHS_ACCUMULATOR, VALUES_BF16, PRECOND_GGT, LCG_FP32 = 0, 1, 2, 4, 8
 GGT_MAX_M = 160
 
 if not os.path.exists(LIB_PATH):
@@ -53,6 +53,7 @@ EXPORTS = {
     "efcp_last_residual": ([_vp], C.c_double),
     "efcp_state_bytes": ([_i64, _i32, _i64], _i64),
     "efcp_launches_per_step": ([_vp], _i32),
+    "efcp_fixed_point_fallbacks": ([_vp], _i64),
     "efcp_profile_begin": ([_vp, _i32], C.c_int),
     "efcp_profile_end": ([_vp, _vp, _vp], C.c_int),
     "efcp_topk_static": ([_vp, _i64, _i64, _vp, _vp, _vp], C.c_int),
@@ -271,6 +272,9 @@ class Efcp:
                                          None if update is None else update.data_ptr(), eta,
                                          gamma, clip_norm, s.cuda_stream), "efcp_step_apply")
         return theta
+
+    def fixed_point_fallbacks(self) -> int:
+        return int(_lib.efcp_fixed_point_fallbacks(self._h))
 
     def validate(self) -> int:
         """efcp_validate: raises EfcpError when the window's derived structures are

@@ -31,6 +31,8 @@ struct efcp_ctx {
   int block = 0, n_blocks = 0;  // block-wise Top-k: block length in coordinates, number of blocks
   int blk_resident = 1;         // thread blocks of the block-wise kernel one SM holds
   double2* ggt_rot = nullptr;   // Sparse GGT: the rotations of one step's eigendecomposition
+  float* vmax = nullptr;        // fixed-point LCG: max |V| per (slab, row)
+  unsigned long long* lcg_redo = nullptr;  // slabs the fixed-point LCG redid in fp32
   double* upd_norm = nullptr;   // [0]: |u|^2 of the last efcp_update_norm, then its partial sums
   int64_t norm_t = -1;          // step count at that call
   int blk_threads = kBlkThreads;  // threads per thread block of the block-wise kernel
@@ -258,8 +260,15 @@ int efcp_create_blockwise(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float
   if (!out) return EFCP_EINVAL;
   *out = nullptr;
   if (!valid_args(d, m, k) || !(lambda > 0.f) || !std::isfinite(lambda)) return EFCP_EINVAL;
-  if (flags & ~(EFCP_RHS_ACCUMULATOR | EFCP_VALUES_BF16 | EFCP_PRECOND_GGT)) return EFCP_EINVAL;
+  if (flags & ~(EFCP_RHS_ACCUMULATOR | EFCP_VALUES_BF16 | EFCP_PRECOND_GGT | EFCP_LCG_FP32))
+    return EFCP_EINVAL;
   if ((flags & EFCP_RHS_ACCUMULATOR) && (flags & EFCP_VALUES_BF16)) return EFCP_EINVAL;
+  // EFCP_LCG=fp32 / fixed in the environment overrides the flag (testing)
+  if (const char* env = getenv("EFCP_LCG")) {
+    if (!std::strcmp(env, "fp32")) flags |= EFCP_LCG_FP32;
+    if (!std::strcmp(env, "fixed")) flags &= ~EFCP_LCG_FP32;
+  }
+  const bool lcg_fixed = !(flags & EFCP_LCG_FP32) && !(flags & EFCP_RHS_ACCUMULATOR);
   if ((flags & EFCP_PRECOND_GGT) && ((flags & EFCP_RHS_ACCUMULATOR) || m > kGgtMaxM))
     return EFCP_EINVAL;
   if (block != 0 && (block < 32 || block > kBlkMax || (block & 31))) return EFCP_EINVAL;
@@ -316,6 +325,13 @@ int efcp_create_blockwise(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float
   const int64_t sums = (flags & EFCP_RHS_ACCUMULATOR) ? 2 : 1;
   if ((rc = dev_alloc(ctx, &ctx->slab_part, int64_t(z.n_slabs) * m * 8 * sums))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->upd_norm, int64_t(kUpdMaxBlocks + 1) * 8))) return fail(rc);
+  if (lcg_fixed) {
+    if ((rc = dev_alloc(ctx, &ctx->vmax, int64_t(z.n_slabs) * m * 4))) return fail(rc);
+    if ((rc = dev_alloc(ctx, &ctx->lcg_redo, 8))) return fail(rc);
+    if (cudaMemset(ctx->vmax, 0, size_t(z.n_slabs) * m * 4) != cudaSuccess ||
+        cudaMemset(ctx->lcg_redo, 0, 8) != cudaSuccess)
+      return fail(EFCP_ECUDA);
+  }
   if (flags & EFCP_PRECOND_GGT) {
     if ((rc = dev_alloc(ctx, &ctx->ggt_rot, ggt_log_entries(m) * 16))) return fail(rc);
   }
@@ -374,6 +390,10 @@ int efcp_create_blockwise(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float
   ok &= cudaFuncSetAttribute(k_lcg<false, true, float>, attr, int(smem)) == cudaSuccess;
   ok &= cudaFuncSetAttribute(k_lcg<true, false, bf16raw>, attr, int(smem)) == cudaSuccess;
   ok &= cudaFuncSetAttribute(k_lcg<false, false, bf16raw>, attr, int(smem)) == cudaSuccess;
+  ok &= cudaFuncSetAttribute(k_lcg<true, false, float, true>, attr, int(smem)) == cudaSuccess;
+  ok &= cudaFuncSetAttribute(k_lcg<false, false, float, true>, attr, int(smem)) == cudaSuccess;
+  ok &= cudaFuncSetAttribute(k_lcg<true, false, bf16raw, true>, attr, int(smem)) == cudaSuccess;
+  ok &= cudaFuncSetAttribute(k_lcg<false, false, bf16raw, true>, attr, int(smem)) == cudaSuccess;
   ok &= cudaDeviceSynchronize() == cudaSuccess;
   if (!ok) {
     ctx->last_cuda = int(cudaGetLastError());
@@ -486,7 +506,7 @@ static int step_impl(efcp_ctx* ctx, const float* grad, float* update, void* stre
   k_layout_row<<<ctx->n_slabs, kLayoutWarps * 32, 0, st>>>(
       ctx->sel_idx, ctx->sel_val, k, ctx->W, ctx->n_slabs, m, slot, ctx->offs, row_idx,
       ctx->R + int64_t(slot) * k, row_val, ctx->V16 ? ctx->V16 + int64_t(slot) * k : nullptr,
-      ctx->slab_ctr);
+      ctx->slab_ctr, ctx->vmax);
   EFCP_LAUNCHED();
   // scalar products with the new row, Gram row/column
   const bool acc_mode = (ctx->flags & EFCP_RHS_ACCUMULATOR) != 0;
@@ -551,7 +571,19 @@ static int step_impl(efcp_ctx* ctx, const float* grad, float* update, void* stre
   k_lcg<VEC, ACC, VT><<<ctx->grid_slab, kSlabThreads, smem, st>>>(                             \
       ctx->R, VPTR, ctx->offs, k, m, ctx->W, ctx->n_slabs, ctx->wf, update, d,                 \
       ctx->slab_ctr + 1, ctx->order, ctx->e, inv_lambda, ap)
-  if (ctx->V16) {
+#define EFCP_LCG_FIXED_LAUNCH(VEC, VT, VPTR)                                                    \
+  k_lcg<VEC, false, VT, true><<<ctx->grid_slab, kSlabThreads, smem, st>>>(                     \
+      ctx->R, VPTR, ctx->offs, k, m, ctx->W, ctx->n_slabs, ctx->wf, update, d,                 \
+      ctx->slab_ctr + 1, ctx->order, ctx->e, inv_lambda, ap, ctx->vmax, ctx->lcg_redo)
+  if (ctx->vmax) {
+    if (ctx->V16) {
+      if (uvec) EFCP_LCG_FIXED_LAUNCH(true, bf16raw, ctx->V16);
+      else EFCP_LCG_FIXED_LAUNCH(false, bf16raw, ctx->V16);
+    } else {
+      if (uvec) EFCP_LCG_FIXED_LAUNCH(true, float, ctx->V);
+      else EFCP_LCG_FIXED_LAUNCH(false, float, ctx->V);
+    }
+  } else if (ctx->V16) {
     if (uvec) EFCP_LCG_LAUNCH(true, false, bf16raw, ctx->V16);
     else EFCP_LCG_LAUNCH(false, false, bf16raw, ctx->V16);
   } else if (acc_mode) {
@@ -562,6 +594,7 @@ static int step_impl(efcp_ctx* ctx, const float* grad, float* update, void* stre
     else EFCP_LCG_LAUNCH(false, false, float, ctx->V);
   }
 #undef EFCP_LCG_LAUNCH
+#undef EFCP_LCG_FIXED_LAUNCH
   EFCP_LAUNCHED();
   prof_mark(ctx, 4, st);
   if (ctx->prof_on && ctx->prof_n < ctx->prof_cap) ++ctx->prof_n;
@@ -854,7 +887,7 @@ int efcp_state_import(efcp_ctx* ctx, const void* host_buf, int64_t bytes) {
   StateHeader h;
   std::memcpy(&h, host_buf, sizeof(h));
   if (h.magic != kStateMagic || h.d != ctx->d || h.k != ctx->k || h.m != ctx->m ||
-      h.W != ctx->W || h.n_slabs != ctx->n_slabs || h.flags != ctx->flags ||
+      h.W != ctx->W || h.n_slabs != ctx->n_slabs || (h.flags & ~EFCP_LCG_FP32) != (ctx->flags & ~EFCP_LCG_FP32) ||
       h.pad != uint32_t(ctx->block) ||
       std::memcmp(&h.lambda, &ctx->lambda, 4) != 0 || h.t < 0)
     return EFCP_EINVAL;
@@ -869,8 +902,23 @@ int efcp_state_import(efcp_ctx* ctx, const void* host_buf, int64_t bytes) {
   // two-pass route once; the selection does not depend on the route)
   EFCP_CUDA(cudaMemset(ctx->sc, 0, sizeof(Scalars)));
   EFCP_CUDA(cudaMemset(ctx->hist, 0, (kBins1 + kBins2 + kBins3) * 4));
+  if (ctx->vmax) {  // derived from the window: rebuilt rather than stored
+    k_vmax_all<<<ctx->n_slabs, 256>>>(ctx->V, ctx->offs, ctx->k, ctx->m, ctx->vmax);
+    EFCP_CUDA(cudaGetLastError());
+    EFCP_CUDA(cudaDeviceSynchronize());
+  }
   ctx->t = h.t;
   return EFCP_OK;
+}
+
+int64_t efcp_fixed_point_fallbacks(efcp_ctx* ctx) {
+  if (!ctx) return -1;
+  if (!ctx->lcg_redo) return 0;
+  unsigned long long v = 0;
+  if (cudaSetDevice(ctx->device) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess ||
+      cudaMemcpy(&v, ctx->lcg_redo, 8, cudaMemcpyDeviceToHost) != cudaSuccess)
+    return -1;
+  return int64_t(v);
 }
 
 int efcp_error_norm(efcp_ctx* ctx, double* out) {

@@ -95,7 +95,9 @@ __global__ void __launch_bounds__(kLayoutWarps * 32) k_layout_row(
     const int32_t* __restrict__ src_idx, const float* __restrict__ src_val, int64_t k, int W,
     int n_slabs, int m, int slot, const int32_t* __restrict__ offs,
     int32_t* __restrict__ dst_idx, uint16_t* __restrict__ dst_rel, float* __restrict__ dst_val,
-    bf16raw* __restrict__ dst_v16, int* __restrict__ slab_ctr) {
+    bf16raw* __restrict__ dst_v16, int* __restrict__ slab_ctr, float* __restrict__ vmax) {
+  __shared__ float s_max[kLayoutWarps];
+  float vm = 0.f;  // largest magnitude this thread staged (for the fixed-point LCG's bound)
   __shared__ int32_t s_idx[kLayoutWarps][kLayoutChunk];
   __shared__ float s_val[kLayoutWarps][kLayoutChunk];
   __shared__ uint16_t s_q[kLayoutWarps][kLayoutChunk];
@@ -118,6 +120,7 @@ __global__ void __launch_bounds__(kLayoutWarps * 32) k_layout_row(
     for (int a = lane; a < n; a += 32) {
       ci[a] = src_idx[c0 + a];
       cv[a] = src_val[c0 + a];
+      vm = fmaxf(vm, fabsf(cv[a]));
     }
     __syncwarp();
     for (int a0 = 0; a0 < n; a0 += 32) {
@@ -151,6 +154,31 @@ __global__ void __launch_bounds__(kLayoutWarps * 32) k_layout_row(
       }
     }
     __syncwarp();
+  }
+  if (vmax != nullptr) {  // max |value| of the row's segment in this slab (0 when empty)
+    for (int o = 16; o > 0; o >>= 1) vm = fmaxf(vm, __shfl_xor_sync(0xFFFFFFFFu, vm, o));
+    if (lane == 0) s_max[warp] = vm;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      float v = s_max[0];
+      for (int w2 = 1; w2 < kLayoutWarps; ++w2) v = fmaxf(v, s_max[w2]);
+      vmax[int64_t(s) * m + slot] = v;
+    }
+  }
+}
+
+// vmax[s][r] = max |V| over row r's segment in slab s, for every slab and row (after a state
+// import; a step keeps the table up to date through k_layout_row).
+__global__ void __launch_bounds__(256) k_vmax_all(const float* __restrict__ V,
+                                                  const int32_t* __restrict__ offs, int64_t k,
+                                                  int m, float* __restrict__ vmax) {
+  const int s = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int r = warp; r < m; r += 8) {
+    const int b = offs[int64_t(s) * m + r], e = offs[int64_t(s + 1) * m + r];
+    float vm = 0.f;
+    for (int j = b + lane; j < e; j += 32) vm = fmaxf(vm, fabsf(V[int64_t(r) * k + j]));
+    for (int o = 16; o > 0; o >>= 1) vm = fmaxf(vm, __shfl_xor_sync(0xFFFFFFFFu, vm, o));
+    if (lane == 0) vmax[int64_t(s) * m + r] = vm;
   }
 }
 
@@ -424,13 +452,26 @@ struct LcgApply {
   float decay, neg_step;
 };
 
-template <bool VEC, bool ACC, typename VT>
+// FIXED: the accumulator of a slab holds int32 fixed-point sums.  An fp32 atomicAdd on shared
+// memory is a compare-and-swap loop, the integer one is a single operation of less than half
+// the cost.  Per slab, bound = sum_r |w_r| max|V_r in the slab| is an upper bound of every
+// partial sum of every coordinate, so with scale = 2^e, bound * scale < 2^30, nothing can
+// overflow; each product is rounded to a multiple of q = 1 / scale (error at most q / 2, random
+// in sign), which over the slab's n entries adds up to a variance of n q^2 / 12.  The slab is
+// accepted if that is below (1e-5 |u_slab|)^2 - ten times inside the tolerance of the update,
+// slab by slab and therefore for the whole vector - and otherwise accumulated again with fp32
+// atomics (its 2.5 MB of entries are still in L2).  Integer sums do not depend on the order of
+// the adds: the accepted slabs of u are reproducible bit for bit.
+template <bool VEC, bool ACC, typename VT, bool FIXED = false>
 __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_lcg(
     const uint16_t* __restrict__ R, const VT* __restrict__ V, const int32_t* __restrict__ offs,
     int64_t k, int m, int W, int n_slabs, const float* __restrict__ wf, float* __restrict__ u,
     int64_t d, int* ctr, const int32_t* __restrict__ order, const float* __restrict__ xi,
-    float inv_lambda, LcgApply ap) {
+    float inv_lambda, LcgApply ap, const float* __restrict__ vmax = nullptr,
+    unsigned long long* __restrict__ redo_count = nullptr) {
+  static_assert(!(FIXED && ACC), "the fixed-point accumulator starts from zero");
   extern __shared__ __align__(16) unsigned char smraw[];
+  __shared__ double red[32];
   float* acc = reinterpret_cast<float*>(smraw);
   float* wc = reinterpret_cast<float*>(smraw + size_t(W) * 4);
   int32_t* seg = reinterpret_cast<int32_t*>(smraw + size_t(W) * 4 + size_t(m) * 8);
@@ -453,44 +494,81 @@ __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_lcg(
       for (int i = tid; i < n; i += blockDim.x) acc[i] = xi[int64_t(base) + i] * inv_lambda;
     }
     __syncthreads();
-    for (int r = warp; r < m; r += nwarps) {
-      const int b = seg[r], e = seg[m + r];
-      const float c = wc[r];
-      if (b >= e || c == 0.f) continue;
-      const uint16_t* Rr = R + int64_t(r) * k;
-      const VT* Vr = V + int64_t(r) * k;
-      if (r + nwarps < m) {
-        const int rn = r + nwarps;
-        prefetch_segment(R + int64_t(rn) * k, V + int64_t(rn) * k, seg[rn], seg[m + rn], lane);
-      }
-      int j0 = b + lane;
-      for (; j0 + 32 * (kDepth - 1) < e - 31 + lane; j0 += 32 * kDepth) {  // full passes
-        const uint16_t* pi = Rr + j0;
-        const VT* pv = Vr + j0;
-        int ii[kDepth];
-        float vv[kDepth];
-#pragma unroll
-        for (int q = 0; q < kDepth; ++q) {
-          ii[q] = __ldcs(pi + 32 * q);
-          vv[q] = load_value(pv + 32 * q);
+    // every row's segment of this slab, scaled by the row's weight, into the accumulator
+    auto accumulate = [&](auto add) {
+      for (int r = warp; r < m; r += nwarps) {
+        const int b = seg[r], e = seg[m + r];
+        const float c = wc[r];
+        if (b >= e || c == 0.f) continue;
+        const uint16_t* Rr = R + int64_t(r) * k;
+        const VT* Vr = V + int64_t(r) * k;
+        if (r + nwarps < m) {
+          const int rn = r + nwarps;
+          prefetch_segment(R + int64_t(rn) * k, V + int64_t(rn) * k, seg[rn], seg[m + rn], lane);
         }
-#pragma unroll
-        for (int q = 0; q < kDepth; ++q) atomicAdd(&acc[ii[q]], c * vv[q]);
+        int j0 = b + lane;
+        for (; j0 + 32 * (kDepth - 1) < e - 31 + lane; j0 += 32 * kDepth) {  // full passes
+          const uint16_t* pi = Rr + j0;
+          const VT* pv = Vr + j0;
+          int ii[kDepth];
+          float vv[kDepth];
+  #pragma unroll
+          for (int q = 0; q < kDepth; ++q) {
+            ii[q] = __ldcs(pi + 32 * q);
+            vv[q] = load_value(pv + 32 * q);
+          }
+  #pragma unroll
+          for (int q = 0; q < kDepth; ++q) add(ii[q], c * vv[q]);
+        }
+        const int rem = e - (j0 - lane);  // entries left for the last pass (warp-uniform)
+        if (rem > 0) {
+          const int groups = (rem + 31) >> 5;
+          tail_dispatch(groups, Rr + j0, Vr + j0, j0 + 32 * (groups - 1) < e, -1,
+                        [&](int, int i, float v) {
+                          if (i >= 0) add(i, c * v);
+                        });
+        }
       }
-      const int rem = e - (j0 - lane);  // entries left for the last pass (warp-uniform)
-      if (rem > 0) {
-        const int groups = (rem + 31) >> 5;
-        tail_dispatch(groups, Rr + j0, Vr + j0, j0 + 32 * (groups - 1) < e, -1,
-                      [&](int, int i, float v) {
-                        if (i >= 0) atomicAdd(&acc[i], c * v);
-                      });
+    };
+    const int64_t gbase = int64_t(s) * W;
+    const int n = int(min(int64_t(W), d - gbase));
+    bool by_float = true;
+    if (FIXED) {
+      double part = 0.0, cnt = 0.0;
+      for (int r = tid; r < m; r += blockDim.x) {
+        part += double(fabsf(wc[r])) * double(vmax[int64_t(s) * m + r]);
+        cnt += double(seg[m + r] - seg[r]);
+      }
+      const double bound = block_sum(part, red);
+      const double n_entries = block_sum(cnt, red);
+      if (bound > 0.0 && bound < 1e30) {
+        int ex;
+        (void)frexp(bound, &ex);  // bound < 2^ex
+        ex = max(ex, -90);
+        const float scale = ldexpf(1.0f, 30 - ex);
+        int* acci = reinterpret_cast<int*>(acc);
+        accumulate([&](int i, float t) { atomicAdd(acci + i, __float2int_rn(t * scale)); });
+        __syncthreads();
+        const float q = ldexpf(1.0f, ex - 30);
+        double nrm2 = 0.0;
+        for (int i = tid; i < n; i += blockDim.x) {
+          const float v = float(acci[i]) * q;
+          acc[i] = v;
+          nrm2 += double(v) * double(v);
+        }
+        nrm2 = block_sum(nrm2, red);
+        by_float = !(n_entries * double(q) * double(q) / 12.0 <= 1e-10 * nrm2);
+        if (by_float) {  // too coarse for this slab: start over
+          if (tid == 0 && redo_count) atomicAdd(redo_count, 1ULL);
+          for (int i = tid; i < (W >> 2); i += blockDim.x) acc4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+          __syncthreads();
+        }
       }
     }
+    if (by_float) accumulate([&](int i, float t) { atomicAdd(&acc[i], t); });
     if (VEC) bulk_store_fence();  // every thread's adds, before the barrier that orders them
     __syncthreads();
     // write the slab out and clear it for the next one
-    const int64_t gbase = int64_t(s) * W;
-    const int n = int(min(int64_t(W), d - gbase));
     if (ap.theta != nullptr) {
       // the parameter update takes the finished slab of u straight from shared memory:
       // theta <- decay theta + (-eta) u; u itself is not written

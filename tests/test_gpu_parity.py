@@ -46,13 +46,13 @@ def lincomb_amplification(cpu, u_ref):
 
 
 def run_parity(d, m, k, lam, grads, flags=0, check_rows="new", gram_every=0,
-               allow_amplified=False, block=0):
+               allow_amplified=False, block=0, gpu_flags=0):
     """grads: iterable of fp32 numpy arrays.  Returns the worst update error seen.
 
     allow_amplified: for deliberately degenerate windows only - the bound becomes
     U_TOL + 8 * 2^-24 * amplification (see lincomb_amplification)."""
     B = _binding()
-    gpu = B.Efcp(d, m, k, lam, flags, block)
+    gpu = B.Efcp(d, m, k, lam, flags | gpu_flags, block)  # gpu_flags: options the oracle has no part in
     cpu = ref.RefEFCP(d, m, k, lam, flags, block)
     assert gpu.k == cpu.k  # same row length (matters for block-wise Top-k)
     g_dev = torch.empty(d, dtype=torch.float32, device="cuda")
@@ -255,6 +255,83 @@ def test_blockwise_unaligned_gradient_and_side_stream():
     cpu.close()
 
 
+# ---- the two accumulators of the linear combination: int32 fixed point (default) and fp32
+# (EFCP_LCG_FP32).  Every other parity case runs the default; these run both.
+def _fp32():
+    return _binding().LCG_FP32
+
+
+def test_fp32_lcg_c1_full_run():
+    w = gradgen.C1
+    run_parity(w.d, w.m, w.k, w.lam, stream_grads(w, w.steps), check_rows="all",
+               gpu_flags=_fp32())
+
+
+@pytest.mark.parametrize("d,m,k,lam,steps,flags,block", [
+    (300_007, 16, 3000, 1e-3, 24, 0, 0),         # ragged tail, several slabs
+    (1_000_001, 8, 10_000, 1e-4, 10, 2, 0),      # bfloat16 values
+    (300_007, 4, 3000, 1e-3, 8, 0, 8192),        # block-wise Top-k
+    (3_000_017, 8, 30_000, 1e-4, 12, 0, 0),      # many slabs, the ring wraps
+])
+def test_both_lcg_accumulators_parity(d, m, k, lam, steps, flags, block):
+    rng = np.random.default_rng(d + m)
+    scale = np.exp(rng.standard_normal(d)).astype(np.float32)  # log-normal scales: heavy tail
+    grads = [(scale * rng.standard_normal(d)).astype(np.float32) for _ in range(steps)]
+    run_parity(d, m, k, lam, grads, flags=flags, block=block)
+    run_parity(d, m, k, lam, grads, flags=flags, block=block, gpu_flags=_fp32())
+
+
+def test_fixed_point_lcg_hard_inputs():
+    """Ties, threshold jumps of 1e3, an all-zero gradient, outliers 300 times the rest: slabs
+    whose grid is too coarse have to fall back to fp32, and the update stays in tolerance.
+    (The same inputs run through the fp32 accumulator first: they are inside what the m x m
+    solve can take, see the note on scale jumps in the tolerances.)"""
+    B = _binding()
+    d, m, k = 200_000, 8, 2000
+    rng = np.random.default_rng(81)
+    grads = [rng.integers(-2, 3, d).astype(np.float32) for _ in range(3)]
+    grads += [(s * rng.standard_normal(d)).astype(np.float32) for s in (1.0, 1e-3, 1e-3, 30.0, 1.0)]
+    g = rng.standard_normal(d).astype(np.float32)
+    g[::5000] *= 300.0
+    grads += [g, np.zeros(d, np.float32), rng.standard_normal(d).astype(np.float32)]
+    run_parity(d, m, k, 1e-2, grads, check_rows="all", gpu_flags=_fp32())
+    run_parity(d, m, k, 1e-2, grads, check_rows="all")
+
+
+def test_fixed_point_lcg_is_reproducible_and_survives_a_checkpoint():
+    B = _binding()
+    d, m, k, lam = 500_000, 8, 5000, 1e-3
+    rng = np.random.default_rng(82)
+    grads = [rng.standard_normal(d).astype(np.float32) for _ in range(12)]
+    a, b = B.Efcp(d, m, k, lam), B.Efcp(d, m, k, lam)
+    g_dev = torch.empty(d, device="cuda")
+    ua, ub = torch.empty(d, device="cuda"), torch.empty(d, device="cuda")
+    for t, g in enumerate(grads):
+        g_dev.copy_(torch.from_numpy(g))
+        a.step(g_dev, ua)
+        b.step(g_dev, ub)
+        if a.fixed_point_fallbacks() == 0 and b.fixed_point_fallbacks() == 0:
+            assert torch.equal(ua, ub), t  # integer sums do not depend on the order of the adds
+    assert a.fixed_point_fallbacks() == 0  # well-scaled data: every slab took the integer route
+    blob = a.state_export()
+    c = B.Efcp(d, m, k, lam)
+    c.state_import(blob)
+    g = rng.standard_normal(d).astype(np.float32)
+    g_dev.copy_(torch.from_numpy(g))
+    uc = torch.empty(d, device="cuda")
+    a.step(g_dev, ua)
+    c.step(g_dev, uc)
+    assert torch.equal(ua, uc)
+    assert c.validate() == 0 and c.status() == 0
+    for h in (a, b, c):
+        h.close()
+    # the accumulator is not part of the state: an fp32 handle takes the same blob
+    f = B.Efcp(d, m, k, lam, B.LCG_FP32)
+    f.state_import(blob)
+    assert f.fixed_point_fallbacks() == 0 and f.step_count == len(grads)
+    f.close()
+
+
 def test_blockwise_rejects_bad_block_sizes():
     B = _binding()
     for block in (16, 48, 20_000, -32):
@@ -390,8 +467,9 @@ def test_full_size_first_steps_match_oracle(w):
     cpu.close()
 
 
-@pytest.mark.parametrize("w,flags", [(gradgen.C3, 0), (gradgen.C4, 0), (gradgen.C3, 1)],
-                         ids=["c3", "c4", "c3_rhs_accumulator"])
+@pytest.mark.parametrize("w,flags", [(gradgen.C3, 0), (gradgen.C4, 0), (gradgen.C3, 1),
+                                     (gradgen.C3, 8), (gradgen.C4, 8)],
+                         ids=["c3", "c4", "c3_rhs_accumulator", "c3_fp32_lcg", "c4_fp32_lcg"])
 def test_full_size_steady_state_residual(w, flags):
     """With the window completely filled (the state the benchmark times) the update must
     solve the defining system (lambda I + (1/m) G^T G) u = x up to the rounding of u itself:
@@ -412,7 +490,7 @@ def test_full_size_steady_state_residual(w, flags):
     slot = (gpu.step_count - 1) % w.m
     ud = u.double()
     x = torch.zeros(w.d, dtype=torch.float64, device="cuda")
-    if flags:
+    if flags & 1:
         x += torch.from_numpy(gpu.error()).cuda().double()
     x.index_add_(0, I[slot].long(), V[slot].double())
     Gu = torch.empty(w.m, dtype=torch.float64, device="cuda")
@@ -433,6 +511,9 @@ def test_full_size_steady_state_residual(w, flags):
     print(f"{w.name}: |Fu - x| = {res:.3e}, rounding bound {lim:.3e}, |x| = {float(x.norm()):.3e}")
     assert res <= lim
     assert gpu.last_residual() < 1e-9
+    if not flags:
+        print(f"{w.name}: slabs redone in fp32 over {gpu.step_count} steps: {gpu.fixed_point_fallbacks()}")
+        assert gpu.fixed_point_fallbacks() == 0  # the benchmark workloads never need the fallback
     gpu.close()
 
 
