@@ -35,12 +35,12 @@ UNIT = "steps/s"
 # profiles/ (dram__bytes_read.sum + dram__bytes_write.sum), keyed by workload; None until
 # a capture of that workload exists.  Scaled from a smaller capture where noted there.
 # Captured on a quarter-size copy of c4_bert_base (same slab width and segment lengths, see
-# profiles/): DRAM traffic / bytes to move was 1.104 for k_sp_rows and 1.082 for k_lcg, and it
+# profiles/): DRAM traffic / bytes to move was 1.104 for k_sp_rows and 1.078 for k_lcg, and it
 # is proportional to the bytes streamed, so the C4 figures are those ratios times the C4 bytes
 # per launch.
 NCU_TRAFFIC_BYTES = {
     "c4_bert_base": {"sp": int(1.104 * 6 * 1024 * 1_094_822),
-                     "lcg": int(1.082 * (6 * 1024 * 1_094_822 + 4 * 109_482_240))},
+                     "lcg": int(1.078 * (6 * 1024 * 1_094_822 + 4 * 109_482_240))},
 }
 
 
@@ -363,7 +363,9 @@ def main():
     moved = mov[kern] / (avg_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": {"sp": "k_sp_rows", "lcg": "k_lcg"}[kern],
                 "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": None if (acc or bf16) else NCU_TRAFFIC_BYTES.get(w.name, {}).get(kern),
+                "traffic": (None if (acc or bf16 or args.block or args.precond != "mfac" or
+                                     (kern == "lcg" and (args.lcg != "fixed" or args.apply_update)))
+                            else NCU_TRAFFIC_BYTES.get(w.name, {}).get(kern)),
                 "peak_source": peak_src, "algorithmic_bytes_per_launch": alg[kern],
                 "avg_launch_ms": avg_ms,
                 "moved": {"bytes_per_launch": mov[kern], "achieved": moved, "frac": moved / peak}}
