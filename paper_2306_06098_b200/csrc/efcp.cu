@@ -33,6 +33,7 @@ struct efcp_ctx {
   double2* ggt_rot = nullptr;   // Sparse GGT: the rotations of one step's eigendecomposition
   float* vmax = nullptr;        // fixed-point LCG: max |V| per (slab, row)
   unsigned long long* lcg_redo = nullptr;  // slabs the fixed-point LCG redid in fp32
+  double lcg_tol2 = 1e-10;      // its acceptance bound, squared: (1e-5)^2
   double* upd_norm = nullptr;   // [0]: |u|^2 of the last efcp_update_norm, then its partial sums
   int64_t norm_t = -1;          // step count at that call
   int blk_threads = kBlkThreads;  // threads per thread block of the block-wise kernel
@@ -319,6 +320,12 @@ int efcp_create_blockwise(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float
   if ((rc = dev_alloc(ctx, &ctx->bk_off, int64_t(z.n_chunks) * kChunk * 2))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->bk_val, int64_t(z.n_chunks) * kChunk * 4))) return fail(rc);
   if (const char* env = getenv("EFCP_NO_SPEC")) ctx->spec = atoi(env) == 0;
+  // EFCP_LCG_FIXED_TOL: relative error a slab of the fixed-point LCG may have before it is redone
+  // in fp32 (default 1e-5; 0 sends every slab through the fallback, which a parity test does)
+  if (const char* env = getenv("EFCP_LCG_FIXED_TOL")) {
+    const double tol = atof(env);
+    if (tol >= 0.0 && tol <= 1e-4) ctx->lcg_tol2 = tol * tol;
+  }
   if ((rc = dev_alloc(ctx, &ctx->sel_idx, k * 4))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->sel_val, k * 4))) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->sc, sizeof(Scalars)))) return fail(rc);
@@ -574,7 +581,8 @@ static int step_impl(efcp_ctx* ctx, const float* grad, float* update, void* stre
 #define EFCP_LCG_FIXED_LAUNCH(VEC, VT, VPTR)                                                    \
   k_lcg<VEC, false, VT, true><<<ctx->grid_slab, kSlabThreads, smem, st>>>(                     \
       ctx->R, VPTR, ctx->offs, k, m, ctx->W, ctx->n_slabs, ctx->wf, update, d,                 \
-      ctx->slab_ctr + 1, ctx->order, ctx->e, inv_lambda, ap, ctx->vmax, ctx->lcg_redo)
+      ctx->slab_ctr + 1, ctx->order, ctx->e, inv_lambda, ap, ctx->vmax, ctx->lcg_redo,         \
+      ctx->lcg_tol2)
   if (ctx->vmax) {
     if (ctx->V16) {
       if (uvec) EFCP_LCG_FIXED_LAUNCH(true, bf16raw, ctx->V16);

@@ -468,7 +468,7 @@ __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_lcg(
     int64_t k, int m, int W, int n_slabs, const float* __restrict__ wf, float* __restrict__ u,
     int64_t d, int* ctr, const int32_t* __restrict__ order, const float* __restrict__ xi,
     float inv_lambda, LcgApply ap, const float* __restrict__ vmax = nullptr,
-    unsigned long long* __restrict__ redo_count = nullptr) {
+    unsigned long long* __restrict__ redo_count = nullptr, double fixed_tol2 = 1e-10) {
   static_assert(!(FIXED && ACC), "the fixed-point accumulator starts from zero");
   extern __shared__ __align__(16) unsigned char smraw[];
   __shared__ double red[32];
@@ -557,7 +557,7 @@ __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_lcg(
           nrm2 += double(v) * double(v);
         }
         nrm2 = block_sum(nrm2, red);
-        by_float = !(n_entries * double(q) * double(q) / 12.0 <= 1e-10 * nrm2);
+        by_float = !(n_entries * double(q) * double(q) / 12.0 <= fixed_tol2 * nrm2);
         if (by_float) {  // too coarse for this slab: start over
           if (tid == 0 && redo_count) atomicAdd(redo_count, 1ULL);
           for (int i = tid; i < (W >> 2); i += blockDim.x) acc4[i] = make_float4(0.f, 0.f, 0.f, 0.f);

@@ -298,6 +298,24 @@ def test_fixed_point_lcg_hard_inputs():
     run_parity(d, m, k, 1e-2, grads, check_rows="all")
 
 
+def test_fixed_point_lcg_fallback_path(monkeypatch):
+    """With the acceptance bound at zero every slab is accumulated in integers, rejected and
+    accumulated again in fp32: the second pass must start from a clean accumulator."""
+    B = _binding()
+    monkeypatch.setenv("EFCP_LCG_FIXED_TOL", "0")
+    d, m, k = 300_007, 8, 3000
+    rng = np.random.default_rng(83)
+    grads = [rng.standard_normal(d).astype(np.float32) for _ in range(10)]
+    run_parity(d, m, k, 1e-3, grads, check_rows="all")
+    run_parity(d, m, k, 1e-3, grads, flags=B.VALUES_BF16, block=4096)
+    h = B.Efcp(d, m, k, 1e-3)
+    g_dev = torch.from_numpy(grads[0]).cuda()
+    u_dev = torch.empty(d, device="cuda")
+    h.step(g_dev, u_dev)
+    assert h.fixed_point_fallbacks() > 0
+    h.close()
+
+
 def test_fixed_point_lcg_is_reproducible_and_survives_a_checkpoint():
     B = _binding()
     d, m, k, lam = 500_000, 8, 5000, 1e-3
