@@ -365,11 +365,17 @@ int efcp_ref_step(efcp_ref* h, const float* grad, float* update) {
   if (o->flags & kFlagValuesBf16)
     for (int64_t r = 0; r < k; ++r) val[r] = round_to_bf16(val[r]);
 
-  // Algorithm 1, error update: xi = a - c.  At a kept coordinate a - a is +0; with rounded values
-  // the rounding residue a - bf16(a) (exact in fp32) stays in the error buffer.
+  // Algorithm 1, error update: xi = a - c.  A kept coordinate becomes literally +0 (what a - a
+  // is for every finite a; a non-finite a would give NaN, and the method defines the kept
+  // coordinate as removed from the error); with rounded values the rounding residue
+  // a - bf16(a) (exact in fp32) stays in the error buffer.
   o->e = o->a;
-  for (int64_t r = 0; r < k; ++r)
-    o->e[size_t(idx[r])] = o->a[size_t(idx[r])] - val[r];
+  if (o->flags & kFlagValuesBf16) {
+    for (int64_t r = 0; r < k; ++r)
+      o->e[size_t(idx[r])] = o->a[size_t(idx[r])] - val[r];
+  } else {
+    for (int64_t r = 0; r < k; ++r) o->e[size_t(idx[r])] = 0.0f;
+  }
   o->t += 1;
 
   // Right-hand side x of the inverse-Fisher-vector product.
