@@ -38,6 +38,21 @@ typedef struct efcp_ctx efcp_ctx;
 #define EFCP_EINTERNAL -6 /* an internal consistency check failed (selection count != k)  */
 #define EFCP_ETOOBIG  -7  /* size beyond the fixed capacity of an allocation-free entry point */
 
+/*
+ * Environment variables read by efcp_create* (testing and tuning aids; none changes what a
+ * step computes beyond the rounding of the update):
+ *   EFCP_NO_SPEC=1        Top-k always takes the exact two-pass candidate route instead of the
+ *                         candidates set aside while a = xi + g is formed.  Same selection.
+ *   EFCP_LCG=fp32|fixed   overrides the EFCP_LCG_FP32 flag (accumulator of the linear combination).
+ *   EFCP_LCG_FIXED_TOL=x  0 <= x <= 1e-4: relative error a slab of the fixed-point accumulator
+ *                         may have before it is accumulated again in fp32 (default 1e-5; 0
+ *                         sends every slab through the fp32 route).
+ *   EFCP_SLAB_W=n         slab width in coordinates (multiple of 32, 256..49152) instead of the
+ *                         width chosen from d, m and the SM count.  The width is part of a
+ *                         checkpoint's header: a state imports only into a handle created with
+ *                         the same width.
+ */
+
 /* flags for efcp_create_ex */
 #define EFCP_RHS_COMPRESSED  0u /* u_t = A(c_t): precondition the compressed accumulator
                                    (Algorithm 1) - the default                             */
@@ -79,6 +94,12 @@ typedef struct efcp_ctx efcp_ctx;
                                    fp32 adds.  The choice is not part of the state: a state
                                    exported with one setting imports into the other.          */
 
+#define EFCP_DEBUG_CHECKS   16u /* After every step the library checks, on the device and on the
+                                   step's stream, what it derived from the new row (offset
+                                   table, slab membership of every entry, the 16-bit index
+                                   stream, the slab weights); a violation turns into the sticky
+                                   status EFCP_EINTERNAL.  Three more small launches per step.   */
+
 /*
  * efcp_create / efcp_create_ex - the initialisation of Algorithm 1: set up an empty window and
  * xi_0 = 0 for dimension d, window length m, k kept entries per step (Top-k of
@@ -103,6 +124,24 @@ int efcp_create_ex(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float lambda
  */
 int efcp_create_blockwise(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float lambda,
                           uint32_t flags, int32_t block);
+
+/*
+ * Caller-supplied memory (the ownership rule of the problem statement's create call: the
+ * handle owns its state, the caller may own the memory it lives in).
+ *   efcp_workspace_bytes : device bytes a handle for these arguments needs in total (state and
+ *                          scratch; the same list of buffers efcp_create_blockwise allocates,
+ *                          for the SM count of the current device, or of a B200 when there is
+ *                          no device); -1 for invalid arguments.  efcp_step_host needs
+ *                          8 d + 512 bytes more for its staging copies of grad and update.
+ *   efcp_create_in       : efcp_create_blockwise (block = 0: global Top-k) that takes every
+ *                          buffer from `workspace` (device, 256-byte aligned, workspace_bytes
+ *                          long) and never calls cudaMalloc; EFCP_ENOMEM when it is too
+ *                          small.  The workspace stays the caller's: efcp_destroy does not
+ *                          free it, and it must outlive the handle.
+ */
+int64_t efcp_workspace_bytes(int64_t d, int32_t m, int64_t k, uint32_t flags, int32_t block);
+int efcp_create_in(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float lambda, uint32_t flags,
+                   int32_t block, void* workspace, int64_t workspace_bytes);
 
 /* Entries per window row: k, or the block-wise total (-1 for a NULL handle). */
 int64_t efcp_row_length(efcp_ctx* ctx);
@@ -236,6 +275,18 @@ int efcp_step_apply(efcp_ctx* ctx, const float* grad, float* theta, float* updat
  */
 int efcp_validate(efcp_ctx* ctx, int64_t* bad);
 
+/*
+ * efcp_test_hook - switches for failure-detection tests; never needed in production.
+ *   EFCP_HOOK_DROP_BLOCK_LOADS (value 0/1): the block-wise Top-k kernel arms the barrier it
+ *       waits on for its bulk copies of xi and g but does not issue the copies, so nothing is
+ *       in flight and the kernel's bounded wait (about a second) runs out: the step ends with
+ *       the sticky status EFCP_ETIMEOUT and an undefined result, the context stays usable,
+ *       the handle can be destroyed.  Only handles from efcp_create_blockwise are affected.
+ * Returns EFCP_EINVAL for an unknown hook.
+ */
+#define EFCP_HOOK_DROP_BLOCK_LOADS 1
+int efcp_test_hook(efcp_ctx* ctx, int32_t hook, int32_t value);
+
 /* Number of completed efcp_step calls on this handle (-1 for a NULL handle). */
 int64_t efcp_step_count(efcp_ctx* ctx);
 
@@ -251,7 +302,7 @@ int efcp_last_cuda_error(efcp_ctx* ctx);
  */
 double efcp_last_residual(efcp_ctx* ctx);
 
-/* Device bytes a handle for (d, m, k) allocates (state + scratch); -1 if invalid. */
+/* efcp_workspace_bytes for the default mode (no flags, global Top-k). */
 int64_t efcp_state_bytes(int64_t d, int32_t m, int64_t k);
 
 /* Slabs of the update that the fixed-point accumulator handed to fp32 since the handle was
@@ -290,11 +341,16 @@ int efcp_profile_end(efcp_ctx* ctx, double* ms_out, int32_t* steps_out);
  * 8 bytes per element of `a`) lives in one fixed array inside the library image,
  * EFCP_TOPK_STATIC_MAX_D elements long: about 8.1 MiB that every GPU which loads the
  * library holds until the process exits.
- *   a      device, d floats, read only.
+ *   a      device, d floats, read only, 16-byte aligned (the kernels read it with vector
+ *          loads; a view that starts at an odd element of a larger buffer is refused
+ *          with EFCP_EINVAL rather than read).
  *   idx    device, k int32: receives the kept indices, ascending.
  *   val    device, k floats: receives a[idx[j]].
  *   stream a cudaStream_t (NULL = default stream); the work is enqueued, not awaited.
- * Returns EFCP_EINVAL for null pointers or k outside 1..d, EFCP_ETOOBIG when
+ * Non-finite entries are ranked, not reported: magnitudes are ordered by their IEEE bit
+ * pattern, so Inf ranks above every finite value and NaN above Inf, and unlike efcp_step
+ * this call has no handle whose status could record them.
+ * Returns EFCP_EINVAL for null pointers, a misaligned `a` or k outside 1..d, EFCP_ETOOBIG when
  * d > EFCP_TOPK_STATIC_MAX_D (nothing is enqueued), EFCP_ECUDA when a runtime call fails.
  * The first call on each device looks up the array's device address and the SM count;
  * make that first call outside any stream capture.  All calls on a device share the one

@@ -15,7 +15,8 @@ LIB_PATH = os.path.join(_HERE, "csrc", "libefcp.so")
 
 OK, EINVAL, ENOMEM, ECUDA, ENUMERIC, ETIMEOUT, EINTERNAL, ETOOBIG = 0, -1, -2, -3, -4, -5, -6, -7
 TOPK_STATIC_MAX_D = 1 << 20
-RHS_COMPRESSED, RHS_ACCUMULATOR, VALUES_BF16, PRECOND_GGT, LCG_FP32 = 0, 1, 2, 4, 8
+RHS_COMPRESSED, RHS_ACCUMULATOR, VALUES_BF16, PRECOND_GGT, LCG_FP32, DEBUG_CHECKS = 0, 1, 2, 4, 8, 16
+HOOK_DROP_BLOCK_LOADS = 1
 GGT_MAX_M = 160
 
 if not os.path.exists(LIB_PATH):
@@ -30,6 +31,9 @@ EXPORTS = {
     "efcp_create": ([C.POINTER(_vp), _i64, _i32, _i64, _f32], C.c_int),
     "efcp_create_ex": ([C.POINTER(_vp), _i64, _i32, _i64, _f32, _u32], C.c_int),
     "efcp_create_blockwise": ([C.POINTER(_vp), _i64, _i32, _i64, _f32, _u32, _i32], C.c_int),
+    "efcp_workspace_bytes": ([_i64, _i32, _i64, _u32, _i32], _i64),
+    "efcp_create_in": ([C.POINTER(_vp), _i64, _i32, _i64, _f32, _u32, _i32, _vp, _i64], C.c_int),
+    "efcp_test_hook": ([_vp, _i32, _i32], C.c_int),
     "efcp_row_length": ([_vp], _i64),
     "efcp_step": ([_vp, _vp, _vp, _vp], C.c_int),
     "efcp_step_host": ([_vp, _vp, _vp, _vp], C.c_int),
@@ -80,6 +84,10 @@ def state_bytes(d: int, m: int, k: int) -> int:
     return int(_lib.efcp_state_bytes(d, m, k))
 
 
+def workspace_bytes(d: int, m: int, k: int, flags: int = 0, block: int = 0) -> int:
+    return int(_lib.efcp_workspace_bytes(d, m, k, flags, block))
+
+
 def paper_state_bytes(d: int, m: int, k: int, value_bytes: int = 4) -> int:
     """Footprint of Sparse M-FAC as the paper's appendix "Memory savings" counts it:
     indices 4mk, values value_bytes*mk, error feedback 4d, SP result 4m, LCG result 4d."""
@@ -90,7 +98,8 @@ def topk_static(a: torch.Tensor, k: int, idx: torch.Tensor, val: torch.Tensor, s
     """efcp_topk_static: exact Top-k of the device vector `a` into the device tensors `idx`
     (int32, k) and `val` (fp32, k), ascending indices, using no allocation at all (the
     scratch memory is a fixed array inside the library; at most TOPK_STATIC_MAX_D elements).
-    For callers that must not allocate device memory; asynchronous on `stream`."""
+    For callers that must not allocate device memory; asynchronous on `stream`.  `a` must start
+    on a 16-byte boundary (the library refuses other pointers with EINVAL)."""
     assert a.is_cuda and idx.is_cuda and val.is_cuda
     assert a.dtype == torch.float32 and val.dtype == torch.float32 and idx.dtype == torch.int32
     assert a.is_contiguous() and idx.is_contiguous() and val.is_contiguous()
@@ -110,17 +119,26 @@ class Efcp:
     """One optimizer state (efcp_ctx) on the current CUDA device."""
 
     def __init__(self, d: int, m: int, k: int, lam: float, flags: int = RHS_COMPRESSED,
-                 block: int = 0):
+                 block: int = 0, workspace: torch.Tensor = None):
         """block > 0: Top-k in blocks of `block` coordinates (efcp_create_blockwise); self.k is
-        then the row length efcp_row_length reports, self.k_req the requested k."""
+        then the row length efcp_row_length reports, self.k_req the requested k.
+        workspace: a contiguous device tensor the handle takes all its memory from
+        (efcp_create_in; workspace_bytes() gives the size); it must outlive the handle."""
         self._h = None
         self.d, self.m, self.k, self.lam, self.flags = int(d), int(m), int(k), float(lam), flags
         self.k_req, self.block = int(k), int(block)
+        self._workspace = workspace
         h = _vp()
-        rc = _lib.efcp_create_blockwise(C.byref(h), self.d, self.m, self.k, self.lam, flags,
-                                        self.block)
+        if workspace is None:
+            rc = _lib.efcp_create_blockwise(C.byref(h), self.d, self.m, self.k, self.lam, flags,
+                                            self.block)
+        else:
+            assert workspace.is_cuda and workspace.is_contiguous()
+            rc = _lib.efcp_create_in(C.byref(h), self.d, self.m, self.k, self.lam, flags,
+                                     self.block, workspace.data_ptr(),
+                                     workspace.numel() * workspace.element_size())
         if rc != OK:
-            raise EfcpError(rc, "efcp_create_blockwise")
+            raise EfcpError(rc, "efcp_create_blockwise" if workspace is None else "efcp_create_in")
         self._h = h
         self.k = int(_lib.efcp_row_length(h))
 
@@ -170,6 +188,9 @@ class Efcp:
 
     def status(self) -> int:
         return int(_lib.efcp_status(self._h))
+
+    def test_hook(self, hook: int, value: int):
+        self._check(_lib.efcp_test_hook(self._h, hook, value), "efcp_test_hook")
 
     def last_residual(self) -> float:
         return float(_lib.efcp_last_residual(self._h))

@@ -79,11 +79,18 @@ struct efcp_ctx {
   float* stage_u = nullptr;
   int last_cuda = 0;
   int launches = 0;
+  unsigned long long* dbg_bad = nullptr;  // EFCP_DEBUG_CHECKS: violations found after a step
+  int hook_drop_loads = 0;  // efcp_test_hook: the block-wise kernel arms its wait, copies nothing
   // stage timing (efcp_profile_*): 5 events per recorded step
   std::vector<cudaEvent_t> prof_ev;
   int prof_cap = 0, prof_n = 0;
   bool prof_on = false;
   std::vector<void*> allocs;
+  // where the device memory comes from: cudaMalloc per buffer (ws_base == nullptr), or pieces
+  // of one caller-supplied workspace; ws_measure only adds the sizes up
+  unsigned char* ws_base = nullptr;
+  int64_t ws_cap = 0, ws_used = 0;
+  bool ws_measure = false;
 };
 
 namespace {
@@ -92,7 +99,6 @@ constexpr int kSpParts = 32;  // second-level partial sums of the scalar product
 
 struct Sizes {
   int W, n_slabs, n_chunks, grid_slab;
-  int64_t total;
 };
 
 int pick_slab_width(int64_t d, int m, int num_sms) {
@@ -113,29 +119,12 @@ int pick_slab_width(int64_t d, int m, int num_sms) {
 inline int64_t align256(int64_t b) { return (b + 255) & ~int64_t(255); }
 constexpr int64_t align256c(int64_t b) { return (b + 255) & ~int64_t(255); }
 
-Sizes compute_sizes(int64_t d, int32_t m, int64_t k, int num_sms) {
+Sizes compute_sizes(int64_t d, int32_t m, int num_sms) {
   Sizes z;
   z.W = pick_slab_width(d, m, num_sms);
   z.n_slabs = int((d + z.W - 1) / z.W);
   z.n_chunks = int((d + kChunk - 1) / kChunk);
   z.grid_slab = z.n_slabs < num_sms * kSlabBlocksPerSM ? z.n_slabs : num_sms * kSlabBlocksPerSM;
-  int64_t b = 0;
-  b += align256(d * 4);                                   // e
-  b += 2 * align256(int64_t(m) * k * 4) + align256(int64_t(m) * k * 2);  // I, V, R
-  b += align256(int64_t(z.n_slabs + 1) * m * 4);          // offs
-  b += 2 * align256(int64_t(m) * m * 8);                  // S, B
-  b += align256((kBins1 + kBins2 + kBins3) * 4);          // hist
-  b += 3 * align256(int64_t(z.n_chunks + 1) * 4);         // chunk_off, sel_gt, sel_eq
-  b += 2 * align256(d * 4);                               // cand_idx, cand_val
-  b += align256(int64_t(z.n_chunks) * kChunk * 2) + align256(int64_t(z.n_chunks) * kChunk * 4);  // buckets
-  b += 2 * align256(k * 4);                               // sel_idx, sel_val
-  b += align256(sizeof(Scalars));
-  b += align256(int64_t(z.n_slabs) * m * 8);              // slab_part
-  b += align256(int64_t(z.n_slabs + 1) * 8) + align256(int64_t(z.n_slabs) * 4);  // colsum, order
-  b += align256(int64_t(kSpParts) * m * 8);               // partial
-  b += align256(int64_t(9) * m * 8);                      // vecs
-  b += align256(int64_t(m) * 4);                          // wf
-  z.total = b;
   return z;
 }
 
@@ -170,8 +159,20 @@ __global__ void k_init_rows(int32_t* __restrict__ I, int64_t k, int64_t total) {
 
 template <typename T>
 int dev_alloc(efcp_ctx* ctx, T** p, int64_t bytes) {
+  const int64_t need = align256(bytes);
+  if (ctx->ws_measure) {
+    ctx->ws_used += need;
+    *p = nullptr;
+    return EFCP_OK;
+  }
+  if (ctx->ws_base) {
+    if (ctx->ws_used + need > ctx->ws_cap) return EFCP_ENOMEM;
+    *p = reinterpret_cast<T*>(ctx->ws_base + ctx->ws_used);
+    ctx->ws_used += need;
+    return EFCP_OK;
+  }
   void* q = nullptr;
-  cudaError_t err = cudaMalloc(&q, size_t(align256(bytes)));
+  cudaError_t err = cudaMalloc(&q, size_t(need));
   if (err != cudaSuccess) {
     ctx->last_cuda = int(err);
     (void)cudaGetLastError();
@@ -241,8 +242,7 @@ const char* efcp_strerror(int code) {
 }
 
 int64_t efcp_state_bytes(int64_t d, int32_t m, int64_t k) {
-  if (!valid_args(d, m, k)) return -1;
-  return compute_sizes(d, m, k, 148).total;
+  return efcp_workspace_bytes(d, m, k, EFCP_RHS_COMPRESSED, 0);
 }
 
 int efcp_create(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float lambda) {
@@ -256,12 +256,17 @@ int efcp_create_ex(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float lambda
 
 int64_t efcp_row_length(efcp_ctx* ctx) { return ctx ? ctx->k : -1; }
 
-int efcp_create_blockwise(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float lambda,
-                          uint32_t flags, int32_t block) {
-  if (!out) return EFCP_EINVAL;
-  *out = nullptr;
+}  // extern "C"
+
+namespace {
+
+// Checks the arguments of a create call and fills in everything of the handle that follows
+// from them and from the SM count (no device memory yet).
+int configure(efcp_ctx* ctx, int64_t d, int32_t m, int64_t k, float lambda, uint32_t flags,
+              int32_t block, int num_sms) {
   if (!valid_args(d, m, k) || !(lambda > 0.f) || !std::isfinite(lambda)) return EFCP_EINVAL;
-  if (flags & ~(EFCP_RHS_ACCUMULATOR | EFCP_VALUES_BF16 | EFCP_PRECOND_GGT | EFCP_LCG_FP32))
+  if (flags & ~(EFCP_RHS_ACCUMULATOR | EFCP_VALUES_BF16 | EFCP_PRECOND_GGT | EFCP_LCG_FP32 |
+                EFCP_DEBUG_CHECKS))
     return EFCP_EINVAL;
   if ((flags & EFCP_RHS_ACCUMULATOR) && (flags & EFCP_VALUES_BF16)) return EFCP_EINVAL;
   // EFCP_LCG=fp32 / fixed in the environment overrides the flag (testing)
@@ -269,7 +274,6 @@ int efcp_create_blockwise(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float
     if (!std::strcmp(env, "fp32")) flags |= EFCP_LCG_FP32;
     if (!std::strcmp(env, "fixed")) flags &= ~EFCP_LCG_FP32;
   }
-  const bool lcg_fixed = !(flags & EFCP_LCG_FP32) && !(flags & EFCP_RHS_ACCUMULATOR);
   if ((flags & EFCP_PRECOND_GGT) && ((flags & EFCP_RHS_ACCUMULATOR) || m > kGgtMaxM))
     return EFCP_EINVAL;
   if (block != 0 && (block < 32 || block > kBlkMax || (block & 31))) return EFCP_EINVAL;
@@ -280,45 +284,12 @@ int efcp_create_blockwise(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float
     const int64_t last = d - int64_t(n_blocks - 1) * block;
     k = int64_t(n_blocks - 1) * block_count(block, k_req, d) + block_count(last, k_req, d);
   }
-  efcp_ctx* ctx = new (std::nothrow) efcp_ctx();
-  if (!ctx) return EFCP_ENOMEM;
-  int rc = EFCP_OK;
-  auto fail = [&](int code) {
-    free_all(ctx);
-    delete ctx;
-    return code;
-  };
-  cudaError_t err = cudaGetDevice(&ctx->device);
-  if (err != cudaSuccess) { (void)cudaGetLastError(); return fail(EFCP_ECUDA); }
-  cudaDeviceProp prop;
-  err = cudaGetDeviceProperties(&prop, ctx->device);
-  if (err != cudaSuccess) { (void)cudaGetLastError(); return fail(EFCP_ECUDA); }
-  ctx->num_sms = prop.multiProcessorCount;
+  ctx->num_sms = num_sms;
   ctx->d = d; ctx->m = m; ctx->k = k; ctx->lambda = lambda; ctx->flags = flags;
   ctx->k_req = k_req; ctx->block = block; ctx->n_blocks = n_blocks;
-  const Sizes z = compute_sizes(d, m, k, ctx->num_sms);
+  const Sizes z = compute_sizes(d, m, ctx->num_sms);
   ctx->W = z.W; ctx->n_slabs = z.n_slabs; ctx->n_chunks = z.n_chunks;
   ctx->grid_slab = z.grid_slab;
-  const int64_t mk = int64_t(m) * k;
-  if ((rc = dev_alloc(ctx, &ctx->e, d * 4))) return fail(rc);
-  if ((rc = dev_alloc(ctx, &ctx->I, mk * 4))) return fail(rc);
-  if ((rc = dev_alloc(ctx, &ctx->R, mk * 2))) return fail(rc);
-  if (flags & EFCP_VALUES_BF16) {
-    if ((rc = dev_alloc(ctx, &ctx->V16, mk * 2))) return fail(rc);
-    if (cudaMemset(ctx->V16, 0, size_t(mk) * 2) != cudaSuccess) return fail(EFCP_ECUDA);
-  }
-  if ((rc = dev_alloc(ctx, &ctx->V, mk * 4))) return fail(rc);
-  if ((rc = dev_alloc(ctx, &ctx->offs, int64_t(z.n_slabs + 1) * m * 4))) return fail(rc);
-  if ((rc = dev_alloc(ctx, &ctx->S, int64_t(m) * m * 8))) return fail(rc);
-  if ((rc = dev_alloc(ctx, &ctx->B, int64_t(m) * m * 8))) return fail(rc);
-  if ((rc = dev_alloc(ctx, &ctx->hist, (kBins1 + kBins2 + kBins3) * 4))) return fail(rc);
-  if ((rc = dev_alloc(ctx, &ctx->chunk_off, int64_t(z.n_chunks + 1) * 4))) return fail(rc);
-  if ((rc = dev_alloc(ctx, &ctx->sel_gt, int64_t(z.n_chunks + 1) * 4))) return fail(rc);
-  if ((rc = dev_alloc(ctx, &ctx->sel_eq, int64_t(z.n_chunks + 1) * 4))) return fail(rc);
-  if ((rc = dev_alloc(ctx, &ctx->cand_idx, d * 4))) return fail(rc);
-  if ((rc = dev_alloc(ctx, &ctx->cand_val, d * 4))) return fail(rc);
-  if ((rc = dev_alloc(ctx, &ctx->bk_off, int64_t(z.n_chunks) * kChunk * 2))) return fail(rc);
-  if ((rc = dev_alloc(ctx, &ctx->bk_val, int64_t(z.n_chunks) * kChunk * 4))) return fail(rc);
   if (const char* env = getenv("EFCP_NO_SPEC")) ctx->spec = atoi(env) == 0;
   // EFCP_LCG_FIXED_TOL: relative error a slab of the fixed-point LCG may have before it is redone
   // in fp32 (default 1e-5; 0 sends every slab through the fallback, which a parity test does)
@@ -326,53 +297,95 @@ int efcp_create_blockwise(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float
     const double tol = atof(env);
     if (tol >= 0.0 && tol <= 1e-4) ctx->lcg_tol2 = tol * tol;
   }
-  if ((rc = dev_alloc(ctx, &ctx->sel_idx, k * 4))) return fail(rc);
-  if ((rc = dev_alloc(ctx, &ctx->sel_val, k * 4))) return fail(rc);
-  if ((rc = dev_alloc(ctx, &ctx->sc, sizeof(Scalars)))) return fail(rc);
+  return EFCP_OK;
+}
+
+// Every device buffer of a configured handle, in one fixed order (efcp_workspace_bytes runs
+// the same list with an arena that only adds up the sizes).
+int alloc_all(efcp_ctx* ctx) {
+  const int64_t d = ctx->d, k = ctx->k;
+  const int m = ctx->m, n_slabs = ctx->n_slabs, n_chunks = ctx->n_chunks;
+  const uint32_t flags = ctx->flags;
+  const int64_t mk = int64_t(m) * k;
+  const bool lcg_fixed = !(flags & EFCP_LCG_FP32) && !(flags & EFCP_RHS_ACCUMULATOR);
   const int64_t sums = (flags & EFCP_RHS_ACCUMULATOR) ? 2 : 1;
-  if ((rc = dev_alloc(ctx, &ctx->slab_part, int64_t(z.n_slabs) * m * 8 * sums))) return fail(rc);
-  if ((rc = dev_alloc(ctx, &ctx->upd_norm, int64_t(kUpdMaxBlocks + 1) * 8))) return fail(rc);
+  int rc = EFCP_OK;
+#define EFCP_ALLOC(field, bytes) \
+  if ((rc = dev_alloc(ctx, &ctx->field, (bytes)))) return rc
+  EFCP_ALLOC(e, d * 4);
+  EFCP_ALLOC(I, mk * 4);
+  EFCP_ALLOC(R, mk * 2);
+  if (flags & EFCP_VALUES_BF16) EFCP_ALLOC(V16, mk * 2);
+  EFCP_ALLOC(V, mk * 4);
+  EFCP_ALLOC(offs, int64_t(n_slabs + 1) * m * 4);
+  EFCP_ALLOC(S, int64_t(m) * m * 8);
+  EFCP_ALLOC(B, int64_t(m) * m * 8);
+  EFCP_ALLOC(hist, (kBins1 + kBins2 + kBins3) * 4);
+  EFCP_ALLOC(chunk_off, int64_t(n_chunks + 1) * 4);
+  EFCP_ALLOC(sel_gt, int64_t(n_chunks + 1) * 4);
+  EFCP_ALLOC(sel_eq, int64_t(n_chunks + 1) * 4);
+  EFCP_ALLOC(cand_idx, d * 4);
+  EFCP_ALLOC(cand_val, d * 4);
+  EFCP_ALLOC(bk_off, int64_t(n_chunks) * kChunk * 2);
+  EFCP_ALLOC(bk_val, int64_t(n_chunks) * kChunk * 4);
+  EFCP_ALLOC(sel_idx, k * 4);
+  EFCP_ALLOC(sel_val, k * 4);
+  EFCP_ALLOC(sc, sizeof(Scalars));
+  EFCP_ALLOC(slab_part, int64_t(n_slabs) * m * 8 * sums);
+  EFCP_ALLOC(upd_norm, int64_t(kUpdMaxBlocks + 1) * 8);
   if (lcg_fixed) {
-    if ((rc = dev_alloc(ctx, &ctx->vmax, int64_t(z.n_slabs) * m * 4))) return fail(rc);
-    if ((rc = dev_alloc(ctx, &ctx->lcg_redo, 8))) return fail(rc);
-    if (cudaMemset(ctx->vmax, 0, size_t(z.n_slabs) * m * 4) != cudaSuccess ||
-        cudaMemset(ctx->lcg_redo, 0, 8) != cudaSuccess)
-      return fail(EFCP_ECUDA);
+    EFCP_ALLOC(vmax, int64_t(n_slabs) * m * 4);
+    EFCP_ALLOC(lcg_redo, 8);
   }
-  if (flags & EFCP_PRECOND_GGT) {
-    if ((rc = dev_alloc(ctx, &ctx->ggt_rot, ggt_log_entries(m) * 16))) return fail(rc);
-  }
-  if ((rc = dev_alloc(ctx, &ctx->partial, int64_t(kSpParts) * m * 8 * sums))) return fail(rc);
-  if ((rc = dev_alloc(ctx, &ctx->vecs, int64_t(9) * m * 8))) return fail(rc);
-  if ((rc = dev_alloc(ctx, &ctx->wf, int64_t(m) * 4))) return fail(rc);
-  if ((rc = dev_alloc(ctx, &ctx->slab_ctr, 256))) return fail(rc);
-  if (block) {
-    // per block: last step's threshold key, then log2 of the candidate margin
-    if ((rc = dev_alloc(ctx, &ctx->blk_T, int64_t(n_blocks) * 8))) return fail(rc);
-    if (cudaMemset(ctx->blk_T, 0, size_t(n_blocks) * 8) != cudaSuccess) return fail(EFCP_ECUDA);
-  }
-  if ((rc = dev_alloc(ctx, &ctx->colsum, int64_t(z.n_slabs + 1) * 8))) return fail(rc);
-  if ((rc = dev_alloc(ctx, &ctx->order, int64_t(z.n_slabs) * 4))) return fail(rc);
+  if (flags & EFCP_PRECOND_GGT) EFCP_ALLOC(ggt_rot, ggt_log_entries(m) * 16);
+  EFCP_ALLOC(partial, int64_t(kSpParts) * m * 8 * sums);
+  EFCP_ALLOC(vecs, int64_t(9) * m * 8);
+  EFCP_ALLOC(wf, int64_t(m) * 4);
+  EFCP_ALLOC(slab_ctr, 256);
+  // block-wise Top-k, per block: last step's threshold key, then log2 of the candidate margin
+  if (ctx->block) EFCP_ALLOC(blk_T, int64_t(ctx->n_blocks) * 8);
+  EFCP_ALLOC(colsum, int64_t(n_slabs + 1) * 8);
+  EFCP_ALLOC(order, int64_t(n_slabs) * 4);
+  EFCP_ALLOC(dbg_bad, 8);
+#undef EFCP_ALLOC
+  return EFCP_OK;
+}
 
-
+// Initial contents (empty window, xi = 0, B = I / (m lambda)) and kernel attributes.
+bool init_state(efcp_ctx* ctx) {
+  const int64_t d = ctx->d, k = ctx->k;
+  const int m = ctx->m, n_slabs = ctx->n_slabs;
+  const int64_t mk = int64_t(m) * k;
   bool ok = true;
   ok &= cudaMemset(ctx->e, 0, size_t(d) * 4) == cudaSuccess;
   ok &= cudaMemset(ctx->V, 0, size_t(mk) * 4) == cudaSuccess;
   ok &= cudaMemset(ctx->R, 0, size_t(mk) * 2) == cudaSuccess;
-  ok &= cudaMemset(ctx->offs, 0, size_t(z.n_slabs + 1) * m * 4) == cudaSuccess;
+  if (ctx->V16) ok &= cudaMemset(ctx->V16, 0, size_t(mk) * 2) == cudaSuccess;
+  ok &= cudaMemset(ctx->offs, 0, size_t(n_slabs + 1) * m * 4) == cudaSuccess;
   ok &= cudaMemset(ctx->S, 0, size_t(m) * m * 8) == cudaSuccess;
-  ok &= cudaMemset(ctx->colsum, 0, size_t(z.n_slabs + 1) * 8) == cudaSuccess;
+  ok &= cudaMemset(ctx->colsum, 0, size_t(n_slabs + 1) * 8) == cudaSuccess;
   ok &= cudaMemset(ctx->hist, 0, (kBins1 + kBins2 + kBins3) * 4) == cudaSuccess;
   ok &= cudaMemset(ctx->sc, 0, sizeof(Scalars)) == cudaSuccess;
   ok &= cudaMemset(ctx->vecs, 0, size_t(9) * m * 8) == cudaSuccess;
   ok &= cudaMemset(ctx->wf, 0, size_t(m) * 4) == cudaSuccess;
+  // a step that gives up (EFCP_ETIMEOUT) leaves the selection buffers as they were; the
+  // kernels after it must still find indices inside [0, d)
+  ok &= cudaMemset(ctx->sel_idx, 0, size_t(k) * 4) == cudaSuccess;
+  ok &= cudaMemset(ctx->sel_val, 0, size_t(k) * 4) == cudaSuccess;
+  ok &= cudaMemset(ctx->dbg_bad, 0, 8) == cudaSuccess;
+  if (ctx->vmax) {
+    ok &= cudaMemset(ctx->vmax, 0, size_t(n_slabs) * m * 4) == cudaSuccess;
+    ok &= cudaMemset(ctx->lcg_redo, 0, 8) == cudaSuccess;
+  }
+  if (ctx->blk_T) ok &= cudaMemset(ctx->blk_T, 0, size_t(ctx->n_blocks) * 8) == cudaSuccess;
   k_init_rows<<<ctx->num_sms * 4, 256>>>(ctx->I, k, mk);
-  k_init_identity<<<ctx->num_sms * 2, 256>>>(ctx->B, m, 1.0 / (double(m) * double(lambda)));
-  const size_t smem = slab_smem_bytes(z.W, m);
+  k_init_identity<<<ctx->num_sms * 2, 256>>>(ctx->B, m,
+                                             1.0 / (double(m) * double(ctx->lambda)));
+  const size_t smem = slab_smem_bytes(ctx->W, m);
   const auto attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
-  if (block) {
-    const int bs = int(block_select_smem(block));
-    ctx->blk_threads = block_select_threads(block, block_count(block, k_req, d));
+  if (ctx->block) {
+    const int bs = int(block_select_smem(ctx->block));
+    ctx->blk_threads = block_select_threads(ctx->block, block_count(ctx->block, ctx->k_req, d));
     ok &= for_block_kernel(ctx->blk_threads, true, [&](auto kern) {
       int resident = 0;
       bool good = cudaFuncSetAttribute(kern, attr, bs) == cudaSuccess;
@@ -385,7 +398,7 @@ int efcp_create_blockwise(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float
       return cudaFuncSetAttribute(kern, attr, bs) == cudaSuccess;
     });
   }
-  if (flags & EFCP_PRECOND_GGT)
+  if (ctx->flags & EFCP_PRECOND_GGT)
     ok &= cudaFuncSetAttribute(ggt_slots(m) <= 2 ? k_ggt_weights<2> : k_ggt_weights<4>, attr,
                                int(ggt_smem_bytes(m))) == cudaSuccess;
   ok &= cudaFuncSetAttribute(k_sp_rows<false, float>, attr, int(smem)) == cudaSuccess;
@@ -402,12 +415,73 @@ int efcp_create_blockwise(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float
   ok &= cudaFuncSetAttribute(k_lcg<true, false, bf16raw, true>, attr, int(smem)) == cudaSuccess;
   ok &= cudaFuncSetAttribute(k_lcg<false, false, bf16raw, true>, attr, int(smem)) == cudaSuccess;
   ok &= cudaDeviceSynchronize() == cudaSuccess;
-  if (!ok) {
+  return ok;
+}
+
+int current_sm_count(int* device) {
+  int dev = 0, n = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) {
+    (void)cudaGetLastError();
+    return 0;
+  }
+  if (device) *device = dev;
+  return n;
+}
+
+int create_impl(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float lambda, uint32_t flags,
+                int32_t block, void* workspace, int64_t workspace_bytes, bool own_memory) {
+  if (!out) return EFCP_EINVAL;
+  *out = nullptr;
+  if (!own_memory && (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) ||
+                      workspace_bytes < 0))
+    return EFCP_EINVAL;
+  efcp_ctx* ctx = new (std::nothrow) efcp_ctx();
+  if (!ctx) return EFCP_ENOMEM;
+  auto fail = [&](int code) {
+    free_all(ctx);
+    delete ctx;
+    return code;
+  };
+  const int sms = current_sm_count(&ctx->device);
+  if (sms < 1) return fail(EFCP_ECUDA);
+  int rc = configure(ctx, d, m, k, lambda, flags, block, sms);
+  if (rc != EFCP_OK) return fail(rc);
+  if (!own_memory) {
+    ctx->ws_base = static_cast<unsigned char*>(workspace);
+    ctx->ws_cap = workspace_bytes;
+  }
+  if ((rc = alloc_all(ctx)) != EFCP_OK) return fail(rc);
+  if (!init_state(ctx)) {
     ctx->last_cuda = int(cudaGetLastError());
     return fail(EFCP_ECUDA);
   }
   *out = ctx;
   return EFCP_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int efcp_create_blockwise(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float lambda,
+                          uint32_t flags, int32_t block) {
+  return create_impl(out, d, m, k, lambda, flags, block, nullptr, 0, true);
+}
+
+int64_t efcp_workspace_bytes(int64_t d, int32_t m, int64_t k, uint32_t flags, int32_t block) {
+  efcp_ctx tmp;
+  tmp.ws_measure = true;
+  int sms = current_sm_count(nullptr);
+  if (sms < 1) sms = 148;  // no device: the SM count of a B200
+  if (configure(&tmp, d, m, k, 1.0f, flags, block, sms) != EFCP_OK) return -1;
+  if (alloc_all(&tmp) != EFCP_OK) return -1;
+  return tmp.ws_used;
+}
+
+int efcp_create_in(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float lambda, uint32_t flags,
+                   int32_t block, void* workspace, int64_t workspace_bytes) {
+  return create_impl(out, d, m, k, lambda, flags, block, workspace, workspace_bytes, false);
 }
 
 int efcp_destroy(efcp_ctx* ctx) {
@@ -424,6 +498,7 @@ int efcp_destroy(efcp_ctx* ctx) {
 static int step_impl(efcp_ctx* ctx, const float* grad, float* update, void* stream_, LcgApply ap) {
   if (!ctx || !grad || (!update && !ap.theta) || grad == update) return EFCP_EINVAL;
   cudaStream_t st = static_cast<cudaStream_t>(stream_);
+  EFCP_CUDA(cudaSetDevice(ctx->device));  // the launches below go to the handle's device
   const int64_t d = ctx->d, k = ctx->k;
   const int m = ctx->m;
   const int slot = int(ctx->t % m);
@@ -452,7 +527,8 @@ static int step_impl(efcp_ctx* ctx, const float* grad, float* update, void* stre
                      [&](auto kern) {
                        kern<<<grid, ctx->blk_threads, bs, st>>>(
                            ctx->e, grad, d, ctx->k_req, ctx->block, ctx->n_blocks, ctx->blk_T,
-                           ctx->sel_idx, ctx->sel_val, ctx->sc, ctx->V16 ? 1 : 0);
+                           ctx->sel_idx, ctx->sel_val, ctx->sc, ctx->V16 ? 1 : 0,
+                           ctx->hook_drop_loads);
                        return true;
                      });
     EFCP_LAUNCHED();
@@ -605,6 +681,19 @@ static int step_impl(efcp_ctx* ctx, const float* grad, float* update, void* stre
 #undef EFCP_LCG_FIXED_LAUNCH
   EFCP_LAUNCHED();
   prof_mark(ctx, 4, st);
+  if (ctx->flags & EFCP_DEBUG_CHECKS) {
+    // the new row's offsets, slab membership and 16-bit stream, and the slab weights; a
+    // violation becomes the sticky internal-error status
+    k_validate_rows<<<dim3(ctx->n_slabs, 1), 128, 0, st>>>(ctx->I, ctx->R, ctx->offs, k, d, m,
+                                                           ctx->W, ctx->n_slabs, slot, slot + 1,
+                                                           ctx->dbg_bad);
+    EFCP_LAUNCHED();
+    k_validate_colsum<<<ctx->n_slabs + 1, 256, 0, st>>>(ctx->offs, ctx->colsum, m, ctx->n_slabs,
+                                                        ctx->dbg_bad);
+    EFCP_LAUNCHED();
+    k_fold_bad<<<1, 1, 0, st>>>(ctx->dbg_bad, ctx->sc);
+    EFCP_LAUNCHED();
+  }
   if (ctx->prof_on && ctx->prof_n < ctx->prof_cap) ++ctx->prof_n;
   ctx->t += 1;
   return EFCP_OK;
@@ -684,6 +773,7 @@ int efcp_step_apply(efcp_ctx* ctx, const float* grad, float* theta, float* updat
 int efcp_step_host(efcp_ctx* ctx, const float* grad, float* update, void* stream_) {
   if (!ctx || !grad || !update) return EFCP_EINVAL;
   cudaStream_t st = static_cast<cudaStream_t>(stream_);
+  EFCP_CUDA(cudaSetDevice(ctx->device));
   if (!ctx->stage_g) {
     int rc;
     if ((rc = dev_alloc(ctx, &ctx->stage_g, ctx->d * 4))) return rc;
@@ -806,45 +896,6 @@ __global__ void __launch_bounds__(256) k_sumsq(const float* __restrict__ e, int6
 }
 }  // namespace
 
-namespace {
-
-// One block per (slab, written row): offsets monotone, entries inside the slab, R == I - s W.
-__global__ void __launch_bounds__(128) k_validate_rows(
-    const int32_t* __restrict__ I, const uint16_t* __restrict__ R, const int32_t* __restrict__ offs,
-    int64_t k, int64_t d, int m, int W, int n_slabs, int rows_written,
-    unsigned long long* __restrict__ bad) {
-  const int s = blockIdx.x, r = blockIdx.y;
-  if (r >= rows_written) return;
-  const int b = offs[int64_t(s) * m + r], e = offs[int64_t(s + 1) * m + r];
-  unsigned long long v = 0;
-  if (threadIdx.x == 0) {
-    if (b > e || b < 0 || e > k) ++v;
-    if (s == 0 && b != 0) ++v;
-    if (s == n_slabs - 1 && e != k) ++v;
-  }
-  const int64_t lo = int64_t(s) * W, hi = lo + W < d ? lo + W : d;
-  for (int j = b + threadIdx.x; j < e && j < k; j += blockDim.x) {
-    const int64_t idx = I[int64_t(r) * k + j];
-    if (idx < lo || idx >= hi) ++v;
-    else if (int64_t(R[int64_t(r) * k + j]) != idx - lo) ++v;
-  }
-  if (v) atomicAdd(bad, v);
-}
-
-// colsum[s] == sum over rows of offs[s][r]
-__global__ void __launch_bounds__(256) k_validate_colsum(const int32_t* __restrict__ offs,
-                                                          const int64_t* __restrict__ colsum,
-                                                          int m, int n_slabs,
-                                                          unsigned long long* __restrict__ bad) {
-  __shared__ double sm[32];
-  const int s = blockIdx.x;
-  double acc = 0.0;  // exact: sums stay far below 2^53
-  for (int r = threadIdx.x; r < m; r += blockDim.x) acc += double(offs[int64_t(s) * m + r]);
-  acc = block_sum(acc, sm);
-  if (threadIdx.x == 0 && int64_t(acc) != colsum[s]) atomicAdd(bad, 1ull);
-}
-
-}  // namespace
 
 int efcp_validate(efcp_ctx* ctx, int64_t* bad_out) {
   if (!ctx) return EFCP_EINVAL;
@@ -856,7 +907,7 @@ int efcp_validate(efcp_ctx* ctx, int64_t* bad_out) {
   const int rows = int(ctx->t < ctx->m ? ctx->t : ctx->m);
   if (rows > 0) {
     k_validate_rows<<<dim3(ctx->n_slabs, rows), 128>>>(ctx->I, ctx->R, ctx->offs, ctx->k, ctx->d,
-                                                       ctx->m, ctx->W, ctx->n_slabs, rows, bad);
+                                                       ctx->m, ctx->W, ctx->n_slabs, 0, rows, bad);
   }
   k_validate_colsum<<<ctx->n_slabs + 1, 256>>>(ctx->offs, ctx->colsum, ctx->m, ctx->n_slabs, bad);
   unsigned long long h = 0;
@@ -953,6 +1004,12 @@ int efcp_error_norm(efcp_ctx* ctx, double* out) {
 }
 
 int64_t efcp_step_count(efcp_ctx* ctx) { return ctx ? ctx->t : -1; }
+
+int efcp_test_hook(efcp_ctx* ctx, int32_t hook, int32_t value) {
+  if (!ctx || hook != EFCP_HOOK_DROP_BLOCK_LOADS) return EFCP_EINVAL;
+  ctx->hook_drop_loads = value ? 1 : 0;
+  return EFCP_OK;
+}
 
 int efcp_status(efcp_ctx* ctx) {
   if (!ctx) return EFCP_EINVAL;
@@ -1104,6 +1161,8 @@ __global__ void __launch_bounds__(kChunkThreads) k_write_sel_only(
 extern "C" int efcp_topk_static(const float* a, int64_t d, int64_t k, int32_t* idx, float* val,
                                 void* stream_) {
   if (!a || !idx || !val || d < 1 || k < 1 || k > d) return EFCP_EINVAL;
+  // the selection kernels read `a` with 16-byte vector loads
+  if (reinterpret_cast<uintptr_t>(a) & 15) return EFCP_EINVAL;
   if (d > kStaticMaxD) return EFCP_ETOOBIG;
   cudaStream_t st = static_cast<cudaStream_t>(stream_);
   int dev = 0;

@@ -24,8 +24,11 @@
 // crowded range) the bisection and the ranking run over all keys of the block.  Either way T
 // and the selection are exact.
 //
-// The wait on the mbarrier is bounded; if it runs out the kernel raises the sticky time-out
-// status and stops once the copies it started have finished.
+// The wait on the mbarrier is bounded (a poll count and a wall-clock limit).  If it runs out
+// the thread block raises the sticky time-out status, starts no further copy, gives the loads
+// it had started a second bounded wait to land (so that nothing is written into shared memory
+// the block has already given up), lets its stores finish and returns.  The step's result is
+// then undefined and the handle reports EFCP_ETIMEOUT.
 #pragma once
 
 #include "efcp_common.cuh"
@@ -39,6 +42,7 @@ constexpr int kBlkMax = 16384;             // largest block (coordinates) the ke
 // entries (2^20 is 1/8 binade)
 constexpr int kBlkMarginInit = 20, kBlkMarginMin = 12, kBlkMarginMax = 22;
 constexpr uint32_t kBlkSpin = 1u << 22;    // polls before the wait for a bulk load gives up
+constexpr uint64_t kBlkWaitNs = 1000000000ull;  // and the wall-clock limit of that wait: 1 s
 constexpr int kBlkWarpCap = 256;           // candidates one warp can set aside per block
 
 // dynamic shared memory of k_ef_block_select: two blocks of xi and one of g
@@ -76,6 +80,22 @@ __device__ __forceinline__ bool blk_mbar_try(uint64_t* bar, uint32_t parity) {
   return ok != 0u;
 }
 
+__device__ __forceinline__ uint64_t blk_now_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+
+// polls the mbarrier's phase until it completes, kBlkSpin polls were made or kBlkWaitNs went by
+__device__ __forceinline__ bool blk_mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
+  const uint64_t t0 = blk_now_ns();
+  for (uint32_t it = 0; it < kBlkSpin; ++it) {
+    if (blk_mbar_try(bar, parity)) return true;
+    if ((it & 255u) == 255u && blk_now_ns() - t0 > kBlkWaitNs) break;
+  }
+  return false;
+}
+
 // barrier 1 for the first `nthr` threads of the block (whole warps); returns how many of them
 // passed a true predicate
 __device__ __forceinline__ int blk_bar_count(int nthr, bool pred) {
@@ -107,7 +127,9 @@ template <bool ALIGNED, int NT>
 __global__ void __launch_bounds__(NT) k_ef_block_select(
     float* __restrict__ e, const float* __restrict__ g, int64_t d, int64_t k_req, int B,
     int n_blocks, uint32_t* __restrict__ blk_T, int32_t* __restrict__ sel_idx,
-    float* __restrict__ sel_val, Scalars* sc, int values_bf16) {
+    float* __restrict__ sel_val, Scalars* sc, int values_bf16, int drop_loads) {
+  // drop_loads (failure-detection test only): the mbarrier is armed but the copies are not
+  // issued, so nothing is in flight and the bounded wait below runs out
   constexpr int NW = NT / 32;
   extern __shared__ __align__(128) unsigned char blk_smraw[];
   float* ebuf0 = reinterpret_cast<float*>(blk_smraw);  // two buffers for xi / a / the new xi
@@ -135,6 +157,7 @@ __global__ void __launch_bounds__(NT) k_ef_block_select(
                      blk_smem_u32(&mbar)),
                  "r"(2u * bytes)
                  : "memory");
+    if (drop_loads) return;
     blk_bulk_g2s(eb, e + bn0, bytes, &mbar);
     blk_bulk_g2s(gbuf, g + bn0, bytes, &mbar);
   };
@@ -160,13 +183,19 @@ __global__ void __launch_bounds__(NT) k_ef_block_select(
     const bool bulk = is_bulk(b);
     // ---- the block of xi and of g: started one block ahead, or fetched here
     if (bulk) {
-      bool landed = tid != 0;  // one thread polls, the rest wait at the barrier below
-      for (uint32_t it = 0; it < kBlkSpin && !landed; ++it) landed = blk_mbar_try(&mbar, phase);
-      phase ^= 1u;
+      // one thread polls, the rest wait at the barrier below
+      bool landed = tid != 0 || blk_mbar_wait_bounded(&mbar, phase);
       if (!__syncthreads_and(landed)) {  // one verdict for the whole thread block
-        if (tid == 0) atomicOr(&sc->status, kStTimeout);
+        if (tid == 0) {
+          atomicOr(&sc->status, kStTimeout);
+          // no further loads are started; the ones in flight (this block's two) may still
+          // land in shared memory: give them a second bounded wait before the block leaves
+          (void)blk_mbar_wait_bounded(&mbar, phase);
+        }
+        __syncthreads();
         break;
       }
+      phase ^= 1u;
     } else {
       // the copy engine must have read this buffer's last contents before it is refilled
       if (tid == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");

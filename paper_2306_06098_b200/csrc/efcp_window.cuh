@@ -621,4 +621,48 @@ __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_lcg(
   }
 }
 
+// ---- consistency checks of the window's derived structures (efcp_validate, EFCP_DEBUG_CHECKS)
+
+// One block per (slab, row) for the rows [row0, row_end): offsets monotone, entries inside the
+// slab, R == I - s W.
+__global__ void __launch_bounds__(128) k_validate_rows(
+    const int32_t* __restrict__ I, const uint16_t* __restrict__ R, const int32_t* __restrict__ offs,
+    int64_t k, int64_t d, int m, int W, int n_slabs, int row0, int row_end,
+    unsigned long long* __restrict__ bad) {
+  const int s = blockIdx.x, r = row0 + blockIdx.y;
+  if (r >= row_end) return;
+  const int b = offs[int64_t(s) * m + r], e = offs[int64_t(s + 1) * m + r];
+  unsigned long long v = 0;
+  if (threadIdx.x == 0) {
+    if (b > e || b < 0 || e > k) ++v;
+    if (s == 0 && b != 0) ++v;
+    if (s == n_slabs - 1 && e != k) ++v;
+  }
+  const int64_t lo = int64_t(s) * W, hi = lo + W < d ? lo + W : d;
+  for (int j = b + threadIdx.x; j < e && j < k; j += blockDim.x) {
+    const int64_t idx = I[int64_t(r) * k + j];
+    if (idx < lo || idx >= hi) ++v;
+    else if (int64_t(R[int64_t(r) * k + j]) != idx - lo) ++v;
+  }
+  if (v) atomicAdd(bad, v);
+}
+
+// colsum[s] == sum over rows of offs[s][r]
+__global__ void __launch_bounds__(256) k_validate_colsum(const int32_t* __restrict__ offs,
+                                                          const int64_t* __restrict__ colsum,
+                                                          int m, int n_slabs,
+                                                          unsigned long long* __restrict__ bad) {
+  __shared__ double sm[32];
+  const int s = blockIdx.x;
+  double acc = 0.0;  // exact: sums stay far below 2^53
+  for (int r = threadIdx.x; r < m; r += blockDim.x) acc += double(offs[int64_t(s) * m + r]);
+  acc = block_sum(acc, sm);
+  if (threadIdx.x == 0 && int64_t(acc) != colsum[s]) atomicAdd(bad, 1ull);
+}
+
+// EFCP_DEBUG_CHECKS: a step's consistency checks found violations -> sticky internal error.
+__global__ void k_fold_bad(const unsigned long long* __restrict__ bad, Scalars* sc) {
+  if (*bad != 0ull) atomicOr(&sc->status, kStCount);
+}
+
 }  // namespace efcp

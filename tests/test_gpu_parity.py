@@ -46,18 +46,21 @@ def lincomb_amplification(cpu, u_ref):
 
 
 def run_parity(d, m, k, lam, grads, flags=0, check_rows="new", gram_every=0,
-               allow_amplified=False, block=0, gpu_flags=0):
+               allow_amplified=False, block=0, gpu_flags=0, gram_at=(), resid_from=None):
     """grads: iterable of fp32 numpy arrays.  Returns the worst update error seen.
 
     allow_amplified: for deliberately degenerate windows only - the bound becomes
-    U_TOL + 8 * 2^-24 * amplification (see lincomb_amplification)."""
+    U_TOL + 8 * 2^-24 * amplification (see lincomb_amplification).
+    gram_at: steps after which the whole scalar-product matrix is compared with the oracle's.
+    resid_from: from this step on, the residual of the m x m solve (the drift monitor of the
+    incrementally updated inverse) must stay below 1e-9 at every step."""
     B = _binding()
     gpu = B.Efcp(d, m, k, lam, flags | gpu_flags, block)  # gpu_flags: options the oracle has no part in
     cpu = ref.RefEFCP(d, m, k, lam, flags, block)
     assert gpu.k == cpu.k  # same row length (matters for block-wise Top-k)
     g_dev = torch.empty(d, dtype=torch.float32, device="cuda")
     u_dev = torch.empty(d, dtype=torch.float32, device="cuda")
-    worst = 0.0
+    worst = worst_resid = 0.0
     for t, g in enumerate(grads):
         g = np.ascontiguousarray(g, np.float32)
         g_dev.copy_(torch.from_numpy(g))
@@ -79,7 +82,11 @@ def run_parity(d, m, k, lam, grads, flags=0, check_rows="new", gram_every=0,
         if allow_amplified and err > U_TOL:
             tol = U_TOL + 8 * 2.0 ** -24 * lincomb_amplification(cpu, u_ref)
         assert err <= tol, f"update rel-L2 {err:.3e} (tol {tol:.3e}) at step {t}"
-        if gram_every and (t % gram_every == 0):
+        if resid_from is not None and t >= resid_from:
+            r = gpu.last_residual()
+            worst_resid = max(worst_resid, r)
+            assert r < 1e-9, f"m x m residual {r:.3e} at step {t}"
+        if (gram_every and (t % gram_every == 0)) or t in gram_at:
             Sg, Sc = gpu.gram(), cpu.gram()
             assert np.array_equal(Sg, Sg.T)
             assert np.allclose(Sg, Sc, rtol=1e-12, atol=1e-12 * np.abs(Sc).max())
@@ -90,7 +97,8 @@ def run_parity(d, m, k, lam, grads, flags=0, check_rows="new", gram_every=0,
             assert np.array_equal(gi, ci) and np.array_equal(bits(gv), bits(cv))
     assert gpu.step_count == cpu.step_count
     assert gpu.validate() == 0  # offset table, 16-bit stream and slab weights are consistent
-    print(f"parity d={d} m={m} k={k}: worst update rel-L2 {worst:.3e}")
+    print(f"parity d={d} m={m} k={k}: worst update rel-L2 {worst:.3e}" +
+          (f", worst m x m residual {worst_resid:.3e}" if resid_from is not None else ""))
     gpu.close()
     cpu.close()
     return worst
@@ -110,6 +118,18 @@ def test_c1_full_run():
 def test_c2_shape_first_steps():
     w = gradgen.C2
     run_parity(w.d, w.m, w.k, w.lam, stream_grads(w, 24), gram_every=8)
+
+
+def test_c2_full_run_ring_wraps_at_m1024():
+    """The whole ResNet-20-shaped run: 2000 steps of an m = 1024 ring, so the window fills, wraps,
+    and from step 1024 on every step removes a row from the explicitly kept inverse and borders
+    it with the new one (976 replacements).  Error buffer, the new row and the update are
+    compared with the oracle at every step, the scalar-product matrix around each wrap and at
+    the end, and the residual of the m x m solve must not drift."""
+    w = gradgen.C2
+    assert w.steps == 2000 and w.m == 1024
+    run_parity(w.d, w.m, w.k, w.lam, stream_grads(w, w.steps), check_rows="all",
+               gram_at={w.m - 1, w.m, w.m + 1, 1500, w.steps - 1}, resid_from=w.m)
 
 
 @pytest.mark.parametrize("d,m,k,steps", [
@@ -460,13 +480,21 @@ def _device_stream(w, device="cuda"):
     return gradgen.GradStream.for_workload(w, device)
 
 
-@pytest.mark.parametrize("w", [gradgen.C3, gradgen.C4], ids=lambda w: w.name)
-def test_full_size_first_steps_match_oracle(w):
+def _c5_corners():
+    """The corners of the density x window sweep: densities 0.1 % and 10 %, windows 128 and 1024."""
+    want = {"c5_dens0.001_m128", "c5_dens0.001_m1024", "c5_dens0.1_m128", "c5_dens0.1_m1024"}
+    pts = [w for w in gradgen.sweep_points() if w.name in want]
+    assert len(pts) == 4
+    return pts
+
+
+@pytest.mark.parametrize("w,steps", [(gradgen.C3, 20), (gradgen.C4, 3)] +
+                         [(w, 3) for w in _c5_corners()], ids=lambda x: getattr(x, "name", None))
+def test_full_size_first_steps_match_oracle(w, steps):
     """Element by element at the full dimension: every coordinate of the error buffer, the
     inserted rows and the update, for the first steps of the workload's own gradient stream
     (generated on the device, the same bytes copied to the oracle)."""
     B = _binding()
-    steps = 3
     gs = _device_stream(w)
     gpu = B.Efcp(w.d, w.m, w.k, w.lam)
     cpu = ref.RefEFCP(w.d, w.m, w.k, w.lam)
@@ -486,8 +514,10 @@ def test_full_size_first_steps_match_oracle(w):
 
 
 @pytest.mark.parametrize("w,flags", [(gradgen.C3, 0), (gradgen.C4, 0), (gradgen.C3, 1),
-                                     (gradgen.C3, 8), (gradgen.C4, 8)],
-                         ids=["c3", "c4", "c3_rhs_accumulator", "c3_fp32_lcg", "c4_fp32_lcg"])
+                                     (gradgen.C3, 8), (gradgen.C4, 8)] +
+                         [(w, 0) for w in _c5_corners()],
+                         ids=["c3", "c4", "c3_rhs_accumulator", "c3_fp32_lcg", "c4_fp32_lcg"] +
+                         [w.name for w in _c5_corners()])
 def test_full_size_steady_state_residual(w, flags):
     """With the window completely filled (the state the benchmark times) the update must
     solve the defining system (lambda I + (1/m) G^T G) u = x up to the rounding of u itself:
@@ -532,6 +562,27 @@ def test_full_size_steady_state_residual(w, flags):
     if not flags:
         print(f"{w.name}: slabs redone in fp32 over {gpu.step_count} steps: {gpu.fixed_point_fallbacks()}")
         assert gpu.fixed_point_fallbacks() == 0  # the benchmark workloads never need the fallback
+    if not flags & 1:
+        # The accumulation of the linear combination alone, range by range: u against the same
+        # combination sum_r w_r row_r formed in fp64 from the library's window and weights.
+        # With the fixed-point accumulator every range of coordinates must stay well inside
+        # the update's tolerance even where a coordinate collects a hundred terms (10 %
+        # density, m = 1024); the worst range is printed.
+        wts = torch.from_numpy(gpu.weights()).cuda()
+        exact = torch.zeros(w.d, dtype=torch.float64, device="cuda")
+        for r in range(w.m):
+            exact.index_add_(0, I[r].long(), V[r].double() * wts[r])
+        span = 32_768
+        pad = (-w.d) % span
+        diff2 = torch.nn.functional.pad((ud - exact) ** 2, (0, pad)).view(-1, span).sum(1)
+        ref2 = torch.nn.functional.pad(exact ** 2, (0, pad)).view(-1, span).sum(1)
+        whole = float(diff2.sum().sqrt() / ref2.sum().sqrt())
+        live = ref2 > 0
+        per_range = (diff2[live] / ref2[live]).sqrt()
+        print(f"{w.name}: linear combination vs fp64, whole vector {whole:.2e}, worst range of "
+              f"{span} coordinates {float(per_range.max()):.2e} (of {int(live.sum())} ranges)")
+        assert whole <= 2e-5
+        assert float(per_range.max()) <= U_TOL
     gpu.close()
 
 

@@ -58,6 +58,11 @@ def test_static_topk_matches_step_selection_twice_in_a_row():
         assert np.array_equal(got_i, want_i)                                   # bit-exact,
         assert np.array_equal(got_v.view(np.uint32), want_v.view(np.uint32))  # as for all state
         assert np.all(np.diff(got_i) > 0)
+        # and directly against the CPU oracle's Top-k (stable-sort definition)
+        from oracle import ref
+        ora_i, ora_v = ref.topk(g.cpu().numpy(), k)
+        assert np.array_equal(got_i, ora_i)
+        assert np.array_equal(got_v.view(np.uint32), ora_v.view(np.uint32))
 
 
 def test_static_topk_rejects_what_it_cannot_hold():
@@ -73,6 +78,11 @@ def test_static_topk_rejects_what_it_cannot_hold():
     with pytest.raises(B.EfcpError) as ei:
         B.topk_static(a[:8], 9, torch.empty(9, dtype=torch.int32, device="cuda"),
                       torch.empty(9, dtype=torch.float32, device="cuda"))
+    assert ei.value.code == B.EINVAL
+    # a vector that does not start on a 16-byte boundary (a view into a larger buffer) is
+    # refused before anything is launched: the kernels would read it with vector loads
+    with pytest.raises(B.EfcpError) as ei:
+        B.topk_static(a[1:1001], 4, idx, val)
     assert ei.value.code == B.EINVAL
     # the largest size it accepts
     a = torch.randn(B.TOPK_STATIC_MAX_D, device="cuda")
