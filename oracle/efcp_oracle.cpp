@@ -522,4 +522,14 @@ int efcp_ref_num_threads(void) {
 #endif
 }
 
+// Size of the OpenMP team for the calls that follow (timing the single-thread baseline);
+// no result depends on it.
+void efcp_ref_set_num_threads(int32_t n) {
+#ifdef _OPENMP
+  if (n >= 1) omp_set_num_threads(n);
+#else
+  (void)n;
+#endif
+}
+
 }  // extern "C"

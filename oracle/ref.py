@@ -43,6 +43,8 @@ def lib():
         L.efcp_ref_round_bf16.argtypes = [vp, vp, i64]
         L.efcp_ref_round_bf16.restype = None
         L.efcp_ref_num_threads.argtypes = []
+        L.efcp_ref_set_num_threads.argtypes = [i32]
+        L.efcp_ref_set_num_threads.restype = None
         _lib = L
     return _lib
 
@@ -53,6 +55,11 @@ def _ptr(a):
 
 def num_threads() -> int:
     return int(lib().efcp_ref_num_threads())
+
+
+def set_num_threads(n: int) -> None:
+    """Size of the OpenMP team of the following calls (results do not depend on it)."""
+    lib().efcp_ref_set_num_threads(int(n))
 
 
 def topk(a: np.ndarray, k: int, fullsort: bool = False):

@@ -22,6 +22,7 @@
 #include "efcp_mxm.cuh"
 #include "efcp_topk.cuh"
 #include "efcp_window.cuh"
+#include "efcp_select.cuh"
 
 using namespace efcp;
 
@@ -70,7 +71,10 @@ struct efcp_ctx {
   Scalars* sc = nullptr;
   double* slab_part = nullptr;  // SP: one partial sum per (slab, row)
   double* partial = nullptr;    // SP: kSpParts x m sums of slab partials
-  double* vecs = nullptr;  // 9 m-vectors: delta, aprime, y, bold, z, w, res, dw, rhs
+  double* vecs = nullptr;  // 10 m-vectors: delta, aprime, y, bold, z, w, res, dw, rhs, final w
+  int32_t* blk_tot = nullptr;   // selection kernel: per-block totals
+  unsigned int* bar = nullptr;  // grid barriers of the two cooperative kernels (2 words each)
+  int sel_grid = 0, mxm_grid = 0;  // their grids: every block resident
   float* wf = nullptr;
   int* slab_ctr = nullptr;   // work counters of the slab kernels (SP, LCG)
   int64_t* colsum = nullptr; // n_slabs + 1 column sums of offs
@@ -96,6 +100,7 @@ struct efcp_ctx {
 namespace {
 
 constexpr int kSpParts = 32;  // second-level partial sums of the scalar products
+constexpr int kMaxCoopBlocks = 1024;  // largest grid of the cooperative kernels
 
 struct Sizes {
   int W, n_slabs, n_chunks, grid_slab;
@@ -339,7 +344,9 @@ int alloc_all(efcp_ctx* ctx) {
   }
   if (flags & EFCP_PRECOND_GGT) EFCP_ALLOC(ggt_rot, ggt_log_entries(m) * 16);
   EFCP_ALLOC(partial, int64_t(kSpParts) * m * 8 * sums);
-  EFCP_ALLOC(vecs, int64_t(9) * m * 8);
+  EFCP_ALLOC(vecs, int64_t(10) * m * 8);
+  EFCP_ALLOC(blk_tot, int64_t(2) * kMaxCoopBlocks * 4);
+  EFCP_ALLOC(bar, 64);
   EFCP_ALLOC(wf, int64_t(m) * 4);
   EFCP_ALLOC(slab_ctr, 256);
   // block-wise Top-k, per block: last step's threshold key, then log2 of the candidate margin
@@ -366,7 +373,9 @@ bool init_state(efcp_ctx* ctx) {
   ok &= cudaMemset(ctx->colsum, 0, size_t(n_slabs + 1) * 8) == cudaSuccess;
   ok &= cudaMemset(ctx->hist, 0, (kBins1 + kBins2 + kBins3) * 4) == cudaSuccess;
   ok &= cudaMemset(ctx->sc, 0, sizeof(Scalars)) == cudaSuccess;
-  ok &= cudaMemset(ctx->vecs, 0, size_t(9) * m * 8) == cudaSuccess;
+  ok &= cudaMemset(ctx->vecs, 0, size_t(10) * m * 8) == cudaSuccess;
+  ok &= cudaMemset(ctx->bar, 0, 64) == cudaSuccess;
+  ok &= cudaMemset(ctx->blk_tot, 0, size_t(2) * kMaxCoopBlocks * 4) == cudaSuccess;
   ok &= cudaMemset(ctx->wf, 0, size_t(m) * 4) == cudaSuccess;
   // a step that gives up (EFCP_ETIMEOUT) leaves the selection buffers as they were; the
   // kernels after it must still find indices inside [0, d)
@@ -397,6 +406,21 @@ bool init_state(efcp_ctx* ctx) {
     ok &= for_block_kernel(ctx->blk_threads, false, [&](auto kern) {
       return cudaFuncSetAttribute(kern, attr, bs) == cudaSuccess;
     });
+  }
+  {
+    // the cooperative kernels: as many blocks as are resident together, at most 2 per SM
+    // (a grid-wide barrier costs in proportion to the number of blocks)
+    int occ = 0;
+    ok &= cudaFuncSetAttribute(k_mxm, attr, int(mxm_smem_bytes(m))) == cudaSuccess;
+    ok &= cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_mxm, kMxmThreads,
+                                                        mxm_smem_bytes(m)) == cudaSuccess;
+    ok &= occ >= 1;
+    ctx->mxm_grid = std::min(kMaxCoopBlocks, ctx->num_sms * std::min(occ, 2));
+    occ = 0;
+    ok &= cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_select_insert, kSelThreads,
+                                                        kSelSmemBytes) == cudaSuccess;
+    ok &= occ >= 1;
+    ctx->sel_grid = std::min(kMaxCoopBlocks, ctx->num_sms * std::min(occ, 2));
   }
   if (ctx->flags & EFCP_PRECOND_GGT)
     ok &= cudaFuncSetAttribute(ggt_slots(m) <= 2 ? k_ggt_weights<2> : k_ggt_weights<4>, attr,
@@ -519,6 +543,26 @@ static int step_impl(efcp_ctx* ctx, const float* grad, float* update, void* stre
   const double mlambda = double(m) * double(ctx->lambda);
 
   prof_mark(ctx, 0, st);
+  SelectArgs sa{};
+  sa.e = ctx->e; sa.d = d;
+  sa.hist1 = hist1; sa.hist2 = hist2; sa.hist3 = hist3;
+  sa.sc = ctx->sc;
+  sa.cnt = ctx->chunk_off; sa.bk_off = ctx->bk_off; sa.bk_val = ctx->bk_val;
+  sa.n_chunks = ctx->n_chunks;
+  sa.k_total = uint32_t(k);
+  sa.spec_limit = uint32_t(std::min<int64_t>(d, 3 * k + 65536));
+  sa.cnt_gt = ctx->sel_gt; sa.cnt_eq = ctx->sel_eq; sa.blk_tot = ctx->blk_tot;
+  sa.shard_tot = nullptr; sa.shard = 0; sa.n_shards = 1;
+  sa.sel_idx = ctx->sel_idx; sa.sel_val = ctx->sel_val;
+  sa.row_cap = k;
+  sa.values_bf16 = ctx->V16 ? 1 : 0;
+  sa.W = ctx->W; sa.n_slabs = ctx->n_slabs; sa.m = m; sa.slot = slot;
+  sa.offs = ctx->offs; sa.colsum = ctx->colsum; sa.order = ctx->order;
+  sa.row_idx = row_idx; sa.row_rel = ctx->R + int64_t(slot) * k; sa.row_val = row_val;
+  sa.row_v16 = ctx->V16 ? ctx->V16 + int64_t(slot) * k : nullptr;
+  sa.slab_ctr = ctx->slab_ctr; sa.vmax = ctx->vmax;
+  sa.bar = ctx->bar;
+  sa.phase_begin = 0; sa.phase_end = kSelPhases;
   if (ctx->block) {
     // block-wise Top-k: a = xi + g, the selection and xi = a - c in one kernel
     const size_t bs = block_select_smem(ctx->block);
@@ -532,6 +576,7 @@ static int step_impl(efcp_ctx* ctx, const float* grad, float* update, void* stre
                        return true;
                      });
     EFCP_LAUNCHED();
+    sa.phase_begin = 4;  // the selection is complete: only the ring insert is left
   } else {
     // a = xi + g, digit-1 histogram, speculative candidate buckets
     const int chunk_grid = ctx->n_chunks < ctx->num_sms * 8 ? ctx->n_chunks : ctx->num_sms * 8;
@@ -545,56 +590,19 @@ static int step_impl(efcp_ctx* ctx, const float* grad, float* update, void* stre
                                                              ctx->chunk_off, ctx->bk_off,
                                                              ctx->bk_val, ctx->n_chunks, spec);
     EFCP_LAUNCHED();
-    const uint32_t spec_limit = uint32_t(std::min<int64_t>(d, 3 * k + 65536));
-    k_pick<kBins1, 1><<<1, 1024, 0, st>>>(hist1, ctx->sc, uint32_t(k), spec, spec_limit);
-    EFCP_LAUNCHED();
-    // candidates: everything at or above the threshold bin, in index order.  The two-pass
-    // kernels return at once when the buckets are good, k_compact_buckets when they are not.
-    k_count_chunks<<<chunk_grid, kChunkThreads, 0, st>>>(ctx->e, d, ctx->sc, ctx->chunk_off,
-                                                         ctx->n_chunks);
-    EFCP_LAUNCHED();
-    k_scan_counts<<<1, 1024, 0, st>>>(ctx->chunk_off, ctx->n_chunks, &ctx->sc->n_cand);
-    EFCP_LAUNCHED();
-    k_compact_cand<<<chunk_grid, kChunkThreads, 0, st>>>(ctx->e, d, ctx->sc, ctx->chunk_off,
-                                                         ctx->cand_idx, ctx->cand_val, hist2,
-                                                         ctx->n_chunks);
-    EFCP_LAUNCHED();
-    k_compact_buckets<<<ctx->num_sms * 4, 256, 0, st>>>(ctx->bk_off, ctx->bk_val, ctx->sc,
-                                                        ctx->chunk_off, ctx->cand_idx,
-                                                        ctx->cand_val, hist2, ctx->n_chunks);
-    EFCP_LAUNCHED();
-    k_pick<kBins2, 2><<<1, 1024, 0, st>>>(hist2, ctx->sc, uint32_t(k));
-    EFCP_LAUNCHED();
-    const int cand_grid = ctx->num_sms * 4;
-    k_hist3<<<cand_grid, 256, 0, st>>>(ctx->cand_val, ctx->sc, hist3);
-    EFCP_LAUNCHED();
-    k_pick<kBins3, 3><<<1, 1024, 0, st>>>(hist3, ctx->sc, uint32_t(k));
-    EFCP_LAUNCHED();
-    // exact selection, ring insert, residual
-    k_count_sel<<<cand_grid, kChunkThreads, 0, st>>>(ctx->cand_val, ctx->sc, ctx->sel_gt,
-                                                     ctx->sel_eq);
-    EFCP_LAUNCHED();
-    k_scan_sel<<<1, 1024, 0, st>>>(ctx->sel_gt, ctx->sel_eq, ctx->sc, uint32_t(k));
-    EFCP_LAUNCHED();
-    k_write_sel<<<cand_grid, kChunkThreads, 0, st>>>(ctx->cand_idx, ctx->cand_val, ctx->sc,
-                                                     ctx->sel_gt, ctx->sel_eq, ctx->sel_idx,
-                                                     ctx->sel_val, ctx->e, k, ctx->V16 ? 1 : 0);
+  }
+  {
+    // exact selection (global Top-k), residual, ring insert: one cooperative kernel
+    void* args[] = {&sa};
+    EFCP_CUDA(cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(k_select_insert),
+                                          dim3(ctx->sel_grid), dim3(kSelThreads), args,
+                                          kSelSmemBytes, st));
     EFCP_LAUNCHED();
   }
-  k_row_offsets<<<ctx->num_sms * 4, 256, 0, st>>>(ctx->sel_idx, k, ctx->W, ctx->n_slabs, m, slot,
-                                                  ctx->offs, ctx->colsum);
-  EFCP_LAUNCHED();
-  k_slab_order<<<1, 1024, 0, st>>>(ctx->colsum, ctx->n_slabs, ctx->order);
-  EFCP_LAUNCHED();
-  k_layout_row<<<ctx->n_slabs, kLayoutWarps * 32, 0, st>>>(
-      ctx->sel_idx, ctx->sel_val, k, ctx->W, ctx->n_slabs, m, slot, ctx->offs, row_idx,
-      ctx->R + int64_t(slot) * k, row_val, ctx->V16 ? ctx->V16 + int64_t(slot) * k : nullptr,
-      ctx->slab_ctr, ctx->vmax);
-  EFCP_LAUNCHED();
   // scalar products with the new row, Gram row/column
   const bool acc_mode = (ctx->flags & EFCP_RHS_ACCUMULATOR) != 0;
-  const int m2 = acc_mode ? 2 * m : m;  // sums per slab: <row, c> and, for x = a, <row, xi>
   double* rhs = dw + m;
+  double* wfin = rhs + m;
   const size_t smem = slab_smem_bytes(ctx->W, m);
   prof_mark(ctx, 1, st);
 #define EFCP_SP_LAUNCH(ACC, VT, VPTR)                                                          \
@@ -607,15 +615,29 @@ static int step_impl(efcp_ctx* ctx, const float* grad, float* update, void* stre
 #undef EFCP_SP_LAUNCH
   EFCP_LAUNCHED();
   prof_mark(ctx, 2, st);
-  const int sp_parts = ctx->n_slabs < kSpParts ? ctx->n_slabs : kSpParts;
-  k_sp_reduce<<<dim3((m2 + 127) / 128, sp_parts), 128, 0, st>>>(ctx->slab_part, ctx->n_slabs, m2,
-                                                                ctx->partial);
-  EFCP_LAUNCHED();
-  k_sp_finish<<<(m + 127) / 128, 128, 0, st>>>(ctx->partial, sp_parts, m, slot, delta, ctx->S,
-                                               aprime, acc_mode ? rhs : nullptr,
-                                               double(ctx->lambda));
-  EFCP_LAUNCHED();
-  if (ctx->flags & EFCP_PRECOND_GGT) {
+  const bool ggt = (ctx->flags & EFCP_PRECOND_GGT) != 0;
+  {
+    // m x m: sums of the slab partials, S row/column, remove-and-border update of the
+    // inverse, weights, residual and the refinement's correction: one cooperative kernel
+    // (Sparse GGT: only the sums and S, its eigendecomposition follows)
+    MxmArgs ma{};
+    ma.slab_part = ctx->slab_part; ma.partial = ctx->partial;
+    ma.n_slabs = ctx->n_slabs;
+    ma.parts = ctx->n_slabs < kSpParts ? ctx->n_slabs : kSpParts;
+    ma.m = m; ma.slot = slot; ma.acc = acc_mode ? 1 : 0;
+    ma.mlambda = mlambda; ma.lambda = double(ctx->lambda);
+    ma.S = ctx->S; ma.B = ctx->B;
+    ma.delta = delta; ma.aprime = aprime; ma.y = y; ma.bold = bold; ma.w = w; ma.res = res;
+    ma.dw = dw; ma.rhs = rhs;
+    ma.sc = ctx->sc; ma.bar = ctx->bar + 2;
+    ma.phase_begin = 0; ma.phase_end = ggt ? 3 : kMxmPhases;
+    void* args[] = {&ma};
+    EFCP_CUDA(cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(k_mxm),
+                                          dim3(ctx->mxm_grid), dim3(kMxmThreads), args,
+                                          mxm_smem_bytes(m), st));
+    EFCP_LAUNCHED();
+  }
+  if (ggt) {
     // m x m: eigendecomposition of S and the weights of u over the window rows
     if (ggt_slots(m) <= 2)
       k_ggt_weights<2><<<1, kGgtThreads, ggt_smem_bytes(m), st>>>(
@@ -624,27 +646,6 @@ static int step_impl(efcp_ctx* ctx, const float* grad, float* update, void* stre
       k_ggt_weights<4><<<1, kGgtThreads, ggt_smem_bytes(m), st>>>(
           ctx->S, m, slot, double(ctx->lambda), w, ctx->wf, ctx->sc, ctx->ggt_rot);
     EFCP_LAUNCHED();
-  } else {
-  // m x m: remove-and-border update of the inverse, weights, one refinement step
-  const int gemv_grid = (m + 7) / 8;
-  k_gemv<<<gemv_grid, 256, 0, st>>>(ctx->B, aprime, y, m);
-  EFCP_LAUNCHED();
-  k_border_scalars<<<1, 1024, 0, st>>>(y, ctx->B + int64_t(slot) * m, delta, aprime, m, slot,
-                                       mlambda, bold, z, w, ctx->sc);
-  EFCP_LAUNCHED();
-  k_rank2<<<ctx->num_sms * 2, 256, 0, st>>>(ctx->B, bold, z, ctx->sc, m, slot);
-  EFCP_LAUNCHED();
-  if (acc_mode) {  // w = B' rhs replaces the column of B' that k_border_scalars wrote
-    k_gemv<<<gemv_grid, 256, 0, st>>>(ctx->B, rhs, w, m);
-    EFCP_LAUNCHED();
-  }
-  k_residual<<<gemv_grid, 256, 0, st>>>(ctx->S, w, res, m, slot, mlambda,
-                                        acc_mode ? rhs : nullptr);
-  EFCP_LAUNCHED();
-  k_gemv<<<gemv_grid, 256, 0, st>>>(ctx->B, res, dw, m);
-  EFCP_LAUNCHED();
-  k_refine_finish<<<1, 1024, 0, st>>>(w, dw, res, ctx->wf, m, ctx->sc);
-  EFCP_LAUNCHED();
   }
   // linear combination of the window rows
   prof_mark(ctx, 3, st);
@@ -652,12 +653,12 @@ static int step_impl(efcp_ctx* ctx, const float* grad, float* update, void* stre
   const float inv_lambda = 1.0f / ctx->lambda;
 #define EFCP_LCG_LAUNCH(VEC, ACC, VT, VPTR)                                                    \
   k_lcg<VEC, ACC, VT><<<ctx->grid_slab, kSlabThreads, smem, st>>>(                             \
-      ctx->R, VPTR, ctx->offs, k, m, ctx->W, ctx->n_slabs, ctx->wf, update, d,                 \
-      ctx->slab_ctr + 1, ctx->order, ctx->e, inv_lambda, ap)
+      ctx->R, VPTR, ctx->offs, k, m, ctx->W, ctx->n_slabs, w, ggt ? nullptr : dw, wfin, update, \
+      d, ctx->slab_ctr + 1, ctx->order, ctx->e, inv_lambda, ap)
 #define EFCP_LCG_FIXED_LAUNCH(VEC, VT, VPTR)                                                    \
   k_lcg<VEC, false, VT, true><<<ctx->grid_slab, kSlabThreads, smem, st>>>(                     \
-      ctx->R, VPTR, ctx->offs, k, m, ctx->W, ctx->n_slabs, ctx->wf, update, d,                 \
-      ctx->slab_ctr + 1, ctx->order, ctx->e, inv_lambda, ap, ctx->vmax, ctx->lcg_redo,         \
+      ctx->R, VPTR, ctx->offs, k, m, ctx->W, ctx->n_slabs, w, ggt ? nullptr : dw, wfin, update, \
+      d, ctx->slab_ctr + 1, ctx->order, ctx->e, inv_lambda, ap, ctx->vmax, ctx->lcg_redo,      \
       ctx->lcg_tol2)
   if (ctx->vmax) {
     if (ctx->V16) {
@@ -833,7 +834,7 @@ int efcp_get_weights(efcp_ctx* ctx, double* host_w) {
   if (!ctx || !host_w) return EFCP_EINVAL;
   const int rc = sync_status(ctx);
   if (rc == EFCP_ECUDA) return rc;
-  EFCP_CUDA(cudaMemcpy(host_w, ctx->vecs + int64_t(5) * ctx->m, size_t(ctx->m) * 8,
+  EFCP_CUDA(cudaMemcpy(host_w, ctx->vecs + int64_t(9) * ctx->m, size_t(ctx->m) * 8,
                        cudaMemcpyDeviceToHost));
   return rc;
 }

@@ -35,7 +35,7 @@ struct Scalars {
   uint32_t status;  // sticky status bits
   uint32_t have_prev;  // b1 holds the previous step's threshold bin
   uint32_t spec_ok;    // this step's speculative candidate buckets cover the threshold bin
-  uint32_t pad;
+  uint32_t guess;      // the bin from which this step's error-feedback kernel set entries aside
   double schur;     // Schur complement of the bordered inverse (1 / B_ii)
   double beta;      // B_ii before the row was replaced
   double resid;     // max-norm residual of the m x m solve, relative to m
@@ -93,6 +93,54 @@ __device__ __forceinline__ T block_excl_scan(T v, T* total, T* sm) {
   *total = sm[32];
   __syncthreads();
   return res;
+}
+
+__device__ __forceinline__ uint64_t now_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+
+// Barrier across all thread blocks of a kernel that was launched cooperatively (every block
+// resident).  bar[0] counts arrivals, bar[1] exits; both are zero between launches: the
+// n-th barrier of a launch (n = 1, 2, ...) completes when bar[0] reaches n * gridDim.x, and
+// grid_exit(), called by every block as its last action, lets the last block out clear both
+// words for the next launch.  The wait is bounded (kGridWaitNs): if it runs out the call
+// returns false for the whole block, which must then return from the kernel at once; the
+// caller raises the sticky time-out status.
+constexpr uint64_t kGridWaitNs = 2000000000ull;  // 2 s
+__device__ __forceinline__ bool grid_barrier(unsigned int* bar, unsigned int n) {
+  __syncthreads();
+  bool ok = true;
+  if (threadIdx.x == 0) {
+    const unsigned int target = n * gridDim.x;
+    __threadfence();  // this block's writes before the arrival
+    atomicAdd(&bar[0], 1u);
+    const uint64_t t0 = now_ns();
+    unsigned int it = 0;
+    for (;;) {
+      unsigned int seen;
+      asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(&bar[0]) : "memory");
+      if (seen >= target) break;
+      if ((++it & 1023u) == 0u && now_ns() - t0 > kGridWaitNs) {
+        ok = false;
+        break;
+      }
+    }
+    __threadfence();
+  }
+  return __syncthreads_and(ok) != 0;
+}
+__device__ __forceinline__ void grid_exit(unsigned int* bar) {
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    if (atomicAdd(&bar[1], 1u) == gridDim.x - 1u) {  // everyone else has left
+      bar[0] = 0u;
+      __threadfence();
+      bar[1] = 0u;
+    }
+  }
 }
 
 __device__ __forceinline__ double warp_sum(double v) {

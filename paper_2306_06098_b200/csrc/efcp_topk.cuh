@@ -41,6 +41,7 @@ __global__ void __launch_bounds__(kChunkThreads, 8) k_ef_spec(
   __shared__ int sm[33];
   for (int i = threadIdx.x; i < kBins1; i += blockDim.x) h[i] = 0u;
   const uint32_t guess = spec_guess(sc, enable);
+  if (blockIdx.x == 0 && threadIdx.x == 0) sc->guess = guess;  // for the selection kernel
   __syncthreads();
   bool bad = false;
   for (int ch = blockIdx.x; ch < n_chunks; ch += gridDim.x) {

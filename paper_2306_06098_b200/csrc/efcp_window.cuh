@@ -36,41 +36,45 @@
 namespace efcp {
 
 constexpr int kLayoutChunk = 512;   // entries permuted together (a multiple of 32)
-constexpr int kLayoutWarps = 4;     // warps per block of k_layout_row (one block per slab)
 
-// offs[s][slot] for the new row from its ascending index list: entry `pos` starts every
-// slab between its predecessor's slab (exclusive) and its own (inclusive); the last entry
-// also closes all slabs behind it.  One thread per entry, no searches.  colsum[s] =
-// sum over the rows of offs[s][.] is kept up to date (one writer per s), so that
-// colsum[s + 1] - colsum[s] is the number of window entries in slab s.
-__global__ void __launch_bounds__(256) k_row_offsets(const int32_t* __restrict__ idx, int64_t k,
-                                                      int W, int n_slabs, int m, int slot,
-                                                      int32_t* __restrict__ offs,
-                                                      int64_t* __restrict__ colsum) {
+// offs[s][slot] for the new row from its ascending index list of n entries: entry `pos`
+// starts every slab between its predecessor's slab (exclusive) and its own (inclusive); the
+// last entry also closes all slabs behind it.  One thread per entry, no searches (`first`
+// and `stride` spread the entries over the calling threads).  colsum[s] = sum over the rows
+// of offs[s][.] is kept up to date (one writer per s), so that colsum[s + 1] - colsum[s] is
+// the number of window entries in slab s.  An empty row (n == 0: a shard of the coordinates
+// that keeps nothing this step) has offset 0 everywhere.
+__device__ __forceinline__ void row_offsets(const int32_t* __restrict__ idx, int64_t n, int W,
+                                            int n_slabs, int m, int slot,
+                                            int32_t* __restrict__ offs,
+                                            int64_t* __restrict__ colsum, int64_t first,
+                                            int64_t stride) {
   auto put = [&](int s, int32_t v) {
     int32_t* p = offs + int64_t(s) * m + slot;
     colsum[s] += int64_t(v) - int64_t(*p);
     *p = v;
   };
-  for (int64_t pos = int64_t(blockIdx.x) * blockDim.x + threadIdx.x; pos < k;
-       pos += int64_t(gridDim.x) * blockDim.x) {
+  if (n == 0) {
+    for (int64_t s = first; s <= n_slabs; s += stride) put(int(s), 0);
+    return;
+  }
+  for (int64_t pos = first; pos < n; pos += stride) {
     const int s1 = idx[pos] / W;
     const int s0 = pos > 0 ? idx[pos - 1] / W : -1;
     for (int s = s0 + 1; s <= s1; ++s) put(s, int32_t(pos));
-    if (pos == k - 1)
-      for (int s = s1 + 1; s <= n_slabs; ++s) put(s, int32_t(k));
+    if (pos == n - 1)
+      for (int s = s1 + 1; s <= n_slabs; ++s) put(s, int32_t(n));
   }
 }
 
 // order[] = the slabs, heaviest first up to a factor 2^(1/4): a counting sort on the top
 // bits of the slab weight colsum[s + 1] - colsum[s].  The slab kernels hand out slabs in
 // this order, so the heavy slabs are never the last ones a block starts.  The order inside
-// a weight class is arbitrary; no result depends on it.  One block.
+// a weight class is arbitrary; no result depends on it.  Called by all threads of one
+// block; cnt: kOrderBins ints of shared memory, sm: 33.
 constexpr int kOrderBins = 1024;
-__global__ void __launch_bounds__(1024) k_slab_order(const int64_t* __restrict__ colsum,
-                                                      int n_slabs, int32_t* __restrict__ order) {
-  __shared__ int cnt[kOrderBins];
-  __shared__ int sm[33];
+__device__ __forceinline__ void slab_order_block(const int64_t* __restrict__ colsum, int n_slabs,
+                                                 int32_t* __restrict__ order, int* cnt, int* sm) {
   for (int i = threadIdx.x; i < kOrderBins; i += blockDim.x) cnt[i] = 0;
   __syncthreads();
   auto bin_of = [&](int s) {
@@ -80,95 +84,101 @@ __global__ void __launch_bounds__(1024) k_slab_order(const int64_t* __restrict__
   };
   for (int s = threadIdx.x; s < n_slabs; s += blockDim.x) atomicAdd(&cnt[bin_of(s)], 1);
   __syncthreads();
-  int total;
-  const int mine = cnt[threadIdx.x];
-  const int start = block_excl_scan<int>(mine, &total, sm);
-  cnt[threadIdx.x] = start;
+  int carry = 0;
+  for (int b0 = 0; b0 < kOrderBins; b0 += blockDim.x) {  // exclusive prefix of the bin counts
+    const int b = b0 + threadIdx.x;
+    const int mine = b < kOrderBins ? cnt[b] : 0;
+    int total;
+    const int start = block_excl_scan<int>(mine, &total, sm);
+    if (b < kOrderBins) cnt[b] = carry + start;
+    carry += total;
+  }
   __syncthreads();
   for (int s = threadIdx.x; s < n_slabs; s += blockDim.x) order[atomicAdd(&cnt[bin_of(s)], 1)] = s;
+  __syncthreads();
 }
 
 // Insert of the new row: from the ascending (index, value) list of the selection,
 //   ring slot <- the row, every segment [offs[s][slot], offs[s+1][slot]) in the
-//   bank-interleaved order described above.  One block per slab, one warp per chunk.
-__global__ void __launch_bounds__(kLayoutWarps * 32) k_layout_row(
-    const int32_t* __restrict__ src_idx, const float* __restrict__ src_val, int64_t k, int W,
-    int n_slabs, int m, int slot, const int32_t* __restrict__ offs,
-    int32_t* __restrict__ dst_idx, uint16_t* __restrict__ dst_rel, float* __restrict__ dst_val,
-    bf16raw* __restrict__ dst_v16, int* __restrict__ slab_ctr, float* __restrict__ vmax) {
-  __shared__ float s_max[kLayoutWarps];
-  float vm = 0.f;  // largest magnitude this thread staged (for the fixed-point LCG's bound)
-  __shared__ int32_t s_idx[kLayoutWarps][kLayoutChunk];
-  __shared__ float s_val[kLayoutWarps][kLayoutChunk];
-  __shared__ uint16_t s_q[kLayoutWarps][kLayoutChunk];
-  __shared__ int s_cnt[kLayoutWarps][32];
+//   bank-interleaved order described above.  The calling block (NW warps) takes the slabs
+//   block_id, block_id + n_blocks, ...; its warps share the chunks of a segment.  smraw: NW *
+//   (kLayoutChunk * 10 + 128) bytes of shared memory, s_max: NW floats.
+template <int NW>
+__device__ __forceinline__ void layout_row_slabs(
+    const int32_t* __restrict__ src_idx, const float* __restrict__ src_val, int W, int n_slabs,
+    int m, int slot, const int32_t* __restrict__ offs, int32_t* __restrict__ dst_idx,
+    uint16_t* __restrict__ dst_rel, float* __restrict__ dst_val, bf16raw* __restrict__ dst_v16,
+    float* __restrict__ vmax, unsigned char* smraw, float* s_max, int block_id, int n_blocks) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  if (blockIdx.x == 0 && threadIdx.x < 2) slab_ctr[threadIdx.x] = 0;  // SP and LCG work counters
-  const int s = blockIdx.x;  // one block per slab, its warps share the chunks of the segment
-  const int seg_b = offs[int64_t(s) * m + slot];
-  const int seg_e = offs[int64_t(s + 1) * m + slot];
-  int32_t* ci = s_idx[warp];
-  float* cv = s_val[warp];
-  uint16_t* cq = s_q[warp];
-  int* cnt = s_cnt[warp];
-  for (int c0 = seg_b + warp * kLayoutChunk; c0 < seg_e; c0 += kLayoutWarps * kLayoutChunk) {
-    const int n = min(kLayoutChunk, seg_e - c0);
-    cnt[lane] = 0;
-    __syncwarp();
-    // stage the chunk (all loads in flight together), then number every entry within its
-    // bank in ascending index order
-    for (int a = lane; a < n; a += 32) {
-      ci[a] = src_idx[c0 + a];
-      cv[a] = src_val[c0 + a];
-      vm = fmaxf(vm, fabsf(cv[a]));
-    }
-    __syncwarp();
-    for (int a0 = 0; a0 < n; a0 += 32) {
-      const int a = a0 + lane;
-      const bool on = a < n;
-      const int bank = on ? (ci[a] & 31) : 0;
-      const unsigned same = __match_any_sync(0xFFFFFFFFu, on ? bank : 32 + lane);
-      const int before = on ? cnt[bank] : 0;
+  int32_t* ci = reinterpret_cast<int32_t*>(smraw) + warp * kLayoutChunk;
+  float* cv = reinterpret_cast<float*>(smraw + size_t(NW) * kLayoutChunk * 4) + warp * kLayoutChunk;
+  uint16_t* cq =
+      reinterpret_cast<uint16_t*>(smraw + size_t(NW) * kLayoutChunk * 8) + warp * kLayoutChunk;
+  int* cnt = reinterpret_cast<int*>(smraw + size_t(NW) * kLayoutChunk * 10) + warp * 32;
+  for (int s = block_id; s < n_slabs; s += n_blocks) {
+    float vm = 0.f;  // largest magnitude this thread staged (for the fixed-point LCG's bound)
+    const int seg_b = offs[int64_t(s) * m + slot];
+    const int seg_e = offs[int64_t(s + 1) * m + slot];
+    for (int c0 = seg_b + warp * kLayoutChunk; c0 < seg_e; c0 += NW * kLayoutChunk) {
+      const int n = min(kLayoutChunk, seg_e - c0);
+      cnt[lane] = 0;
       __syncwarp();
-      if (on) {
-        cq[a] = uint16_t(before + __popc(same & ((1u << lane) - 1u)));
-        if ((same & ((1u << lane) - 1u)) == 0u) cnt[bank] = before + __popc(same);
+      // stage the chunk (all loads in flight together), then number every entry within its
+      // bank in ascending index order
+      for (int a = lane; a < n; a += 32) {
+        ci[a] = src_idx[c0 + a];
+        cv[a] = src_val[c0 + a];
+        vm = fmaxf(vm, fabsf(cv[a]));
       }
       __syncwarp();
-    }
-    // position in the (occurrence, bank) order
-    for (int a0 = 0; a0 < n; a0 += 32) {
-      const int a = a0 + lane;
-      if (a < n) {
-        const int idx = ci[a], bank = idx & 31, q = cq[a];
-        int pos = 0;
-#pragma unroll 8
-        for (int bb = 0; bb < 32; ++bb) {
-          const int c = cnt[bb];
-          pos += min(c, q) + ((bb < bank && c > q) ? 1 : 0);
+      for (int a0 = 0; a0 < n; a0 += 32) {
+        const int a = a0 + lane;
+        const bool on = a < n;
+        const int bank = on ? (ci[a] & 31) : 0;
+        const unsigned same = __match_any_sync(0xFFFFFFFFu, on ? bank : 32 + lane);
+        const int before = on ? cnt[bank] : 0;
+        __syncwarp();
+        if (on) {
+          cq[a] = uint16_t(before + __popc(same & ((1u << lane) - 1u)));
+          if ((same & ((1u << lane) - 1u)) == 0u) cnt[bank] = before + __popc(same);
         }
-        dst_idx[c0 + pos] = idx;
-        dst_rel[c0 + pos] = uint16_t(idx - s * W);
-        dst_val[c0 + pos] = cv[a];
-        if (dst_v16) dst_v16[c0 + pos].bits = bf16_bits_rn(cv[a]);  // exact: already rounded
+        __syncwarp();
       }
+      // position in the (occurrence, bank) order
+      for (int a0 = 0; a0 < n; a0 += 32) {
+        const int a = a0 + lane;
+        if (a < n) {
+          const int idx = ci[a], bank = idx & 31, q = cq[a];
+          int pos = 0;
+#pragma unroll 8
+          for (int bb = 0; bb < 32; ++bb) {
+            const int c = cnt[bb];
+            pos += min(c, q) + ((bb < bank && c > q) ? 1 : 0);
+          }
+          dst_idx[c0 + pos] = idx;
+          dst_rel[c0 + pos] = uint16_t(idx - s * W);
+          dst_val[c0 + pos] = cv[a];
+          if (dst_v16) dst_v16[c0 + pos].bits = bf16_bits_rn(cv[a]);  // exact: already rounded
+        }
+      }
+      __syncwarp();
     }
-    __syncwarp();
-  }
-  if (vmax != nullptr) {  // max |value| of the row's segment in this slab (0 when empty)
-    for (int o = 16; o > 0; o >>= 1) vm = fmaxf(vm, __shfl_xor_sync(0xFFFFFFFFu, vm, o));
-    if (lane == 0) s_max[warp] = vm;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      float v = s_max[0];
-      for (int w2 = 1; w2 < kLayoutWarps; ++w2) v = fmaxf(v, s_max[w2]);
-      vmax[int64_t(s) * m + slot] = v;
+    if (vmax != nullptr) {  // max |value| of the row's segment in this slab (0 when empty)
+      for (int o = 16; o > 0; o >>= 1) vm = fmaxf(vm, __shfl_xor_sync(0xFFFFFFFFu, vm, o));
+      __syncthreads();  // the previous slab's maxima have been read
+      if (lane == 0) s_max[warp] = vm;
+      __syncthreads();
+      if (threadIdx.x == 0) {
+        float v = s_max[0];
+        for (int w2 = 1; w2 < NW; ++w2) v = fmaxf(v, s_max[w2]);
+        vmax[int64_t(s) * m + slot] = v;
+      }
     }
   }
 }
 
 // vmax[s][r] = max |V| over row r's segment in slab s, for every slab and row (after a state
-// import; a step keeps the table up to date through k_layout_row).
+// import; a step keeps the table up to date when it inserts the row).
 __global__ void __launch_bounds__(256) k_vmax_all(const float* __restrict__ V,
                                                   const int32_t* __restrict__ offs, int64_t k,
                                                   int m, float* __restrict__ vmax) {
@@ -271,9 +281,9 @@ __device__ __forceinline__ void bulk_store_wait_read() {
 // Slab scheduling of the two slab kernels.  Slabs differ in weight (the kept entries
 // cluster where the gradient is large), so blocks do not take a fixed share: block b starts
 // with slab b and then draws the next unprocessed slab from a counter in global memory
-// (cleared by k_layout_row earlier in the step).  The draw for the next slab is issued at
+// (cleared by the insert earlier in the step).  The draw for the next slab is issued at
 // the start of the current one, so its latency is hidden.  Results do not depend on which
-// block processes which slab, nor on the order k_slab_order puts the slabs in: LCG slabs are disjoint outputs, and SP writes one partial
+// block processes which slab, nor on the order the slabs are handed out in: LCG slabs are disjoint outputs, and SP writes one partial
 // sum per (slab, row) that is reduced afterwards in slab order.
 
 // Scalar products of every window row with the newest row c_t:
@@ -465,7 +475,8 @@ struct LcgApply {
 template <bool VEC, bool ACC, typename VT, bool FIXED = false>
 __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_lcg(
     const uint16_t* __restrict__ R, const VT* __restrict__ V, const int32_t* __restrict__ offs,
-    int64_t k, int m, int W, int n_slabs, const float* __restrict__ wf, float* __restrict__ u,
+    int64_t k, int m, int W, int n_slabs, const double* __restrict__ w64,
+    const double* __restrict__ dw64, double* __restrict__ w_out, float* __restrict__ u,
     int64_t d, int* ctr, const int32_t* __restrict__ order, const float* __restrict__ xi,
     float inv_lambda, LcgApply ap, const float* __restrict__ vmax = nullptr,
     unsigned long long* __restrict__ redo_count = nullptr, double fixed_tol2 = 1e-10) {
@@ -476,7 +487,12 @@ __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_lcg(
   float* wc = reinterpret_cast<float*>(smraw + size_t(W) * 4);
   int32_t* seg = reinterpret_cast<int32_t*>(smraw + size_t(W) * 4 + size_t(m) * 8);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
-  for (int r = tid; r < m; r += blockDim.x) wc[r] = wf[r];
+  // the weights: the m x m stage's solution plus its refinement step (dw64 == nullptr: none)
+  for (int r = tid; r < m; r += blockDim.x) {
+    const double v = w64[r] + (dw64 ? dw64[r] : 0.0);
+    wc[r] = float(v);
+    if (blockIdx.x == 0) w_out[r] = v;
+  }
   float4* acc4 = reinterpret_cast<float4*>(acc);
   for (int i = tid; i < (W >> 2); i += blockDim.x) acc4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
   __shared__ int s_next;
