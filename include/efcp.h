@@ -276,6 +276,44 @@ int efcp_step_apply(efcp_ctx* ctx, const float* grad, float* theta, float* updat
 int efcp_validate(efcp_ctx* ctx, int64_t* bad);
 
 /*
+ * Coordinate-sharded state: one optimizer state spread over several GPUs by ranges of
+ * coordinates.  The paper runs on one GPU and has no counterpart of this; the split follows
+ * from the method: error feedback, the window rows and the update are separable by
+ * coordinate, the Top-k threshold and the scalar products are sums over the shards.  Shard r of
+ * n holds the coordinates [d_lo, d_hi) (ranges ascending with r, disjoint, covering
+ * [0, d_global)): its part of xi, of every window row and of u; S and the m x m stage are
+ * replicated.  k_global is the number of entries kept over all shards; a row of a shard holds
+ * as many of them as fall into its range, at most row_cap (<= 0: min(k_global, d_hi - d_lo),
+ * the worst case; a step that would need more raises EFCP_EINTERNAL).  Indices inside a shard
+ * are relative to d_lo.  Flags: EFCP_VALUES_BF16, EFCP_LCG_FP32, EFCP_DEBUG_CHECKS.
+ *
+ * A step is six phases.  Every shard runs efcp_shard_phase(p), then buffer p of all shards
+ * (efcp_shard_buffer) is summed element-wise over the shards and the sum stored back in every
+ * shard's buffer - an all-reduce, e.g. NCCL's on the step's stream - then phase p + 1 runs:
+ *   p = 0  a = xi + g (needs grad: device, d_hi - d_lo floats)    buffer: 4096 uint32
+ *   p = 1  first digit of the threshold key                         buffer: 1024 uint32
+ *   p = 2  second digit                                             buffer: 512 uint32
+ *   p = 3  the key; entries above / equal to it on this shard       buffer: 2 n uint32
+ *   p = 4  selection (ties at the key go to lower coordinates first), residual, ring insert,
+ *          this shard's part of the scalar products                 buffer: m doubles
+ *   p = 5  S, coefficients, this shard's part of u (needs update: device, d_hi - d_lo floats)
+ * Unsigned sums may be formed as signed 32-bit sums (the bits are the same).  Nothing in the
+ * library reads another GPU's memory; the exchanges are the caller's.  Phases must be called
+ * in order (EFCP_EINVAL otherwise).  The state (xi, rows) equals that of an unsharded handle
+ * bit for bit; u agrees up to the rounding of the summed scalar products.
+ *   efcp_row_count : entries ring slot `slot` holds (k for an unsharded handle); efcp_get_row
+ *                    returns that many, then (0, 0) up to the row capacity.  Waits for the device.
+ */
+int efcp_create_shard(efcp_ctx** out, int64_t d_global, int64_t d_lo, int64_t d_hi, int32_t m,
+                      int64_t k_global, int64_t row_cap, float lambda, uint32_t flags,
+                      int32_t shard, int32_t n_shards);
+int efcp_shard_phase(efcp_ctx* ctx, int32_t phase, const float* grad, float* update,
+                     void* stream);
+int efcp_shard_buffer(efcp_ctx* ctx, int32_t phase, void** dev_ptr, int64_t* count,
+                      int32_t* is_f64);
+int64_t efcp_row_count(efcp_ctx* ctx, int32_t slot);
+
+/*
  * efcp_test_hook - switches for failure-detection tests; never needed in production.
  *   EFCP_HOOK_DROP_BLOCK_LOADS (value 0/1): the block-wise Top-k kernel arms the barrier it
  *       waits on for its bulk copies of xi and g but does not issue the copies, so nothing is

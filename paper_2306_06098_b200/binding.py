@@ -34,6 +34,11 @@ EXPORTS = {
     "efcp_workspace_bytes": ([_i64, _i32, _i64, _u32, _i32], _i64),
     "efcp_create_in": ([C.POINTER(_vp), _i64, _i32, _i64, _f32, _u32, _i32, _vp, _i64], C.c_int),
     "efcp_test_hook": ([_vp, _i32, _i32], C.c_int),
+    "efcp_create_shard": ([C.POINTER(_vp), _i64, _i64, _i64, _i32, _i64, _i64, _f32, _u32, _i32,
+                           _i32], C.c_int),
+    "efcp_shard_phase": ([_vp, _i32, _vp, _vp, _vp], C.c_int),
+    "efcp_shard_buffer": ([_vp, _i32, C.POINTER(_vp), C.POINTER(_i64), C.POINTER(_i32)], C.c_int),
+    "efcp_row_count": ([_vp, _i32], _i64),
     "efcp_row_length": ([_vp], _i64),
     "efcp_step": ([_vp, _vp, _vp, _vp], C.c_int),
     "efcp_step_host": ([_vp, _vp, _vp, _vp], C.c_int),
@@ -119,17 +124,25 @@ class Efcp:
     """One optimizer state (efcp_ctx) on the current CUDA device."""
 
     def __init__(self, d: int, m: int, k: int, lam: float, flags: int = RHS_COMPRESSED,
-                 block: int = 0, workspace: torch.Tensor = None):
+                 block: int = 0, workspace: torch.Tensor = None, shard=None):
         """block > 0: Top-k in blocks of `block` coordinates (efcp_create_blockwise); self.k is
         then the row length efcp_row_length reports, self.k_req the requested k.
         workspace: a contiguous device tensor the handle takes all its memory from
-        (efcp_create_in; workspace_bytes() gives the size); it must outlive the handle."""
+        (efcp_create_in; workspace_bytes() gives the size); it must outlive the handle.
+        shard: (d_global, d_lo, d_hi, k_global, index, count) makes the handle one coordinate
+        shard of a larger state (efcp_create_shard); d is then d_hi - d_lo and k the row
+        capacity (<= 0: the worst case)."""
         self._h = None
         self.d, self.m, self.k, self.lam, self.flags = int(d), int(m), int(k), float(lam), flags
         self.k_req, self.block = int(k), int(block)
         self._workspace = workspace
         h = _vp()
-        if workspace is None:
+        if shard is not None:
+            d_global, d_lo, d_hi, k_global, index, count = shard
+            assert d_hi - d_lo == self.d and workspace is None and not block
+            rc = _lib.efcp_create_shard(C.byref(h), d_global, d_lo, d_hi, self.m, k_global,
+                                        self.k, self.lam, flags, index, count)
+        elif workspace is None:
             rc = _lib.efcp_create_blockwise(C.byref(h), self.d, self.m, self.k, self.lam, flags,
                                             self.block)
         else:
@@ -188,6 +201,33 @@ class Efcp:
 
     def status(self) -> int:
         return int(_lib.efcp_status(self._h))
+
+    def shard_phase(self, phase: int, grad=None, update=None, stream=None):
+        """efcp_shard_phase: phase 0 takes the shard's gradient, phase 5 its update tensor."""
+        s = torch.cuda.current_stream() if stream is None else stream
+        self._check(_lib.efcp_shard_phase(self._h, phase,
+                                          None if grad is None else grad.data_ptr(),
+                                          None if update is None else update.data_ptr(),
+                                          s.cuda_stream), "efcp_shard_phase")
+
+    def shard_buffer(self, phase: int) -> torch.Tensor:
+        """The device buffer to be summed over the shards after `phase`, as a tensor aliasing
+        the library's memory (int32 for the counts - same bits as uint32 - or float64)."""
+        p, n, f = _vp(), _i64(), _i32()
+        self._check(_lib.efcp_shard_buffer(self._h, phase, C.byref(p), C.byref(n), C.byref(f)),
+                    "efcp_shard_buffer")
+
+        class _Alias:
+            def __init__(self, ptr, typestr, count):
+                self.__cuda_array_interface__ = {"shape": (count,), "typestr": typestr,
+                                                 "data": (ptr, False), "version": 3}
+
+        dev = torch.device("cuda", torch.cuda.current_device())
+        return torch.as_tensor(_Alias(p.value, "<f8" if f.value else "<i4", int(n.value)),
+                               device=dev)
+
+    def row_count(self, slot: int) -> int:
+        return int(_lib.efcp_row_count(self._h, slot))
 
     def test_hook(self, hook: int, value: int):
         self._check(_lib.efcp_test_hook(self._h, hook, value), "efcp_test_hook")

@@ -75,6 +75,12 @@ struct efcp_ctx {
   int32_t* blk_tot = nullptr;   // selection kernel: per-block totals
   unsigned int* bar = nullptr;  // grid barriers of the two cooperative kernels (2 words each)
   int sel_grid = 0, mxm_grid = 0;  // their grids: every block resident
+  // a coordinate shard of a larger state (efcp_create_shard); otherwise d_global == d etc.
+  int64_t d_global = 0, k_global = 0;
+  int shard = 0, n_shards = 1;
+  uint32_t* shard_tot = nullptr;  // per shard: entries above / at the threshold key
+  int next_phase = 0;             // of efcp_shard_phase
+  bool is_shard = false;
   float* wf = nullptr;
   int* slab_ctr = nullptr;   // work counters of the slab kernels (SP, LCG)
   int64_t* colsum = nullptr; // n_slabs + 1 column sums of offs
@@ -292,6 +298,7 @@ int configure(efcp_ctx* ctx, int64_t d, int32_t m, int64_t k, float lambda, uint
   ctx->num_sms = num_sms;
   ctx->d = d; ctx->m = m; ctx->k = k; ctx->lambda = lambda; ctx->flags = flags;
   ctx->k_req = k_req; ctx->block = block; ctx->n_blocks = n_blocks;
+  ctx->d_global = d; ctx->k_global = k; ctx->shard = 0; ctx->n_shards = 1;
   const Sizes z = compute_sizes(d, m, ctx->num_sms);
   ctx->W = z.W; ctx->n_slabs = z.n_slabs; ctx->n_chunks = z.n_chunks;
   ctx->grid_slab = z.grid_slab;
@@ -354,6 +361,7 @@ int alloc_all(efcp_ctx* ctx) {
   EFCP_ALLOC(colsum, int64_t(n_slabs + 1) * 8);
   EFCP_ALLOC(order, int64_t(n_slabs) * 4);
   EFCP_ALLOC(dbg_bad, 8);
+  if (ctx->is_shard) EFCP_ALLOC(shard_tot, int64_t(ctx->n_shards) * 8);
 #undef EFCP_ALLOC
   return EFCP_OK;
 }
@@ -382,6 +390,8 @@ bool init_state(efcp_ctx* ctx) {
   ok &= cudaMemset(ctx->sel_idx, 0, size_t(k) * 4) == cudaSuccess;
   ok &= cudaMemset(ctx->sel_val, 0, size_t(k) * 4) == cudaSuccess;
   ok &= cudaMemset(ctx->dbg_bad, 0, 8) == cudaSuccess;
+  if (ctx->shard_tot)
+    ok &= cudaMemset(ctx->shard_tot, 0, size_t(ctx->n_shards) * 8) == cudaSuccess;
   if (ctx->vmax) {
     ok &= cudaMemset(ctx->vmax, 0, size_t(n_slabs) * m * 4) == cudaSuccess;
     ok &= cudaMemset(ctx->lcg_redo, 0, 8) == cudaSuccess;
@@ -453,8 +463,15 @@ int current_sm_count(int* device) {
   return n;
 }
 
+// what efcp_create_shard adds to a create call
+struct ShardSpec {
+  int64_t d_global, k_global;
+  int shard, n_shards;
+};
+
 int create_impl(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float lambda, uint32_t flags,
-                int32_t block, void* workspace, int64_t workspace_bytes, bool own_memory) {
+                int32_t block, void* workspace, int64_t workspace_bytes, bool own_memory,
+                const ShardSpec* shard = nullptr) {
   if (!out) return EFCP_EINVAL;
   *out = nullptr;
   if (!own_memory && (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) ||
@@ -471,6 +488,11 @@ int create_impl(efcp_ctx** out, int64_t d, int32_t m, int64_t k, float lambda, u
   if (sms < 1) return fail(EFCP_ECUDA);
   int rc = configure(ctx, d, m, k, lambda, flags, block, sms);
   if (rc != EFCP_OK) return fail(rc);
+  if (shard) {
+    ctx->d_global = shard->d_global; ctx->k_global = shard->k_global;
+    ctx->shard = shard->shard; ctx->n_shards = shard->n_shards;
+    ctx->is_shard = true;
+  }
   if (!own_memory) {
     ctx->ws_base = static_cast<unsigned char*>(workspace);
     ctx->ws_cap = workspace_bytes;
@@ -517,54 +539,26 @@ int efcp_destroy(efcp_ctx* ctx) {
   return EFCP_OK;
 }
 
-// One step; with ap.theta set the linear combination updates the parameters in place of
-// writing u (update may then be NULL).
-static int step_impl(efcp_ctx* ctx, const float* grad, float* update, void* stream_, LcgApply ap) {
-  if (!ctx || !grad || (!update && !ap.theta) || grad == update) return EFCP_EINVAL;
-  cudaStream_t st = static_cast<cudaStream_t>(stream_);
-  EFCP_CUDA(cudaSetDevice(ctx->device));  // the launches below go to the handle's device
-  const int64_t d = ctx->d, k = ctx->k;
-  const int m = ctx->m;
-  const int slot = int(ctx->t % m);
-  ctx->launches = 0;
-  uint32_t* hist1 = ctx->hist;
-  uint32_t* hist2 = ctx->hist + kBins1;
-  uint32_t* hist3 = ctx->hist + kBins1 + kBins2;
-  int32_t* row_idx = ctx->I + int64_t(slot) * k;
-  float* row_val = ctx->V + int64_t(slot) * k;
-  double* delta = ctx->vecs;
-  double* aprime = delta + m;
-  double* y = aprime + m;
-  double* bold = y + m;
-  double* z = bold + m;
-  double* w = z + m;
-  double* res = w + m;
-  double* dw = res + m;
-  const double mlambda = double(m) * double(ctx->lambda);
+}  // extern "C"
 
-  prof_mark(ctx, 0, st);
-  SelectArgs sa{};
-  sa.e = ctx->e; sa.d = d;
-  sa.hist1 = hist1; sa.hist2 = hist2; sa.hist3 = hist3;
-  sa.sc = ctx->sc;
-  sa.cnt = ctx->chunk_off; sa.bk_off = ctx->bk_off; sa.bk_val = ctx->bk_val;
-  sa.n_chunks = ctx->n_chunks;
-  sa.k_total = uint32_t(k);
-  sa.spec_limit = uint32_t(std::min<int64_t>(d, 3 * k + 65536));
-  sa.cnt_gt = ctx->sel_gt; sa.cnt_eq = ctx->sel_eq; sa.blk_tot = ctx->blk_tot;
-  sa.shard_tot = nullptr; sa.shard = 0; sa.n_shards = 1;
-  sa.sel_idx = ctx->sel_idx; sa.sel_val = ctx->sel_val;
-  sa.row_cap = k;
-  sa.values_bf16 = ctx->V16 ? 1 : 0;
-  sa.W = ctx->W; sa.n_slabs = ctx->n_slabs; sa.m = m; sa.slot = slot;
-  sa.offs = ctx->offs; sa.colsum = ctx->colsum; sa.order = ctx->order;
-  sa.row_idx = row_idx; sa.row_rel = ctx->R + int64_t(slot) * k; sa.row_val = row_val;
-  sa.row_v16 = ctx->V16 ? ctx->V16 + int64_t(slot) * k : nullptr;
-  sa.slab_ctr = ctx->slab_ctr; sa.vmax = ctx->vmax;
-  sa.bar = ctx->bar;
-  sa.phase_begin = 0; sa.phase_end = kSelPhases;
+namespace {
+
+// The m-vectors of the m x m stage inside ctx->vecs.
+struct Vecs {
+  double *delta, *aprime, *y, *bold, *z, *w, *res, *dw, *rhs, *wfin;
+};
+Vecs vecs_of(efcp_ctx* ctx) {
+  double* v = ctx->vecs;
+  const int m = ctx->m;
+  return Vecs{v, v + m, v + 2 * m, v + 3 * m, v + 4 * m, v + 5 * m, v + 6 * m, v + 7 * m,
+              v + 8 * m, v + 9 * m};
+}
+
+// a = xi + g with the digit-1 histogram and the speculative candidate buckets, or, with
+// block-wise Top-k, the whole selection.
+int launch_ef(efcp_ctx* ctx, const float* grad, cudaStream_t st) {
+  const int64_t d = ctx->d;
   if (ctx->block) {
-    // block-wise Top-k: a = xi + g, the selection and xi = a - c in one kernel
     const size_t bs = block_select_smem(ctx->block);
     const int grid = std::min(ctx->n_blocks, ctx->num_sms * ctx->blk_resident);
     for_block_kernel(ctx->blk_threads, (reinterpret_cast<uintptr_t>(grad) & 15) == 0,
@@ -575,36 +569,60 @@ static int step_impl(efcp_ctx* ctx, const float* grad, float* update, void* stre
                            ctx->hook_drop_loads);
                        return true;
                      });
-    EFCP_LAUNCHED();
-    sa.phase_begin = 4;  // the selection is complete: only the ring insert is left
   } else {
-    // a = xi + g, digit-1 histogram, speculative candidate buckets
     const int chunk_grid = ctx->n_chunks < ctx->num_sms * 8 ? ctx->n_chunks : ctx->num_sms * 8;
     const int spec = ctx->spec ? 1 : 0;
     if ((reinterpret_cast<uintptr_t>(grad) & 15) == 0)
-      k_ef_spec<true><<<chunk_grid, kChunkThreads, 0, st>>>(ctx->e, grad, d, hist1, ctx->sc,
+      k_ef_spec<true><<<chunk_grid, kChunkThreads, 0, st>>>(ctx->e, grad, d, ctx->hist, ctx->sc,
                                                             ctx->chunk_off, ctx->bk_off,
                                                             ctx->bk_val, ctx->n_chunks, spec);
     else
-      k_ef_spec<false><<<chunk_grid, kChunkThreads, 0, st>>>(ctx->e, grad, d, hist1, ctx->sc,
+      k_ef_spec<false><<<chunk_grid, kChunkThreads, 0, st>>>(ctx->e, grad, d, ctx->hist, ctx->sc,
                                                              ctx->chunk_off, ctx->bk_off,
                                                              ctx->bk_val, ctx->n_chunks, spec);
-    EFCP_LAUNCHED();
   }
-  {
-    // exact selection (global Top-k), residual, ring insert: one cooperative kernel
-    void* args[] = {&sa};
-    EFCP_CUDA(cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(k_select_insert),
-                                          dim3(ctx->sel_grid), dim3(kSelThreads), args,
-                                          kSelSmemBytes, st));
-    EFCP_LAUNCHED();
-  }
-  // scalar products with the new row, Gram row/column
+  EFCP_LAUNCHED();
+  return EFCP_OK;
+}
+
+// Phases [pb, pe) of the selection / ring-insert kernel for ring slot `slot`.
+int launch_select(efcp_ctx* ctx, int slot, int pb, int pe, cudaStream_t st) {
+  const int64_t k = ctx->k;
+  SelectArgs sa{};
+  sa.e = ctx->e; sa.d = ctx->d;
+  sa.hist1 = ctx->hist; sa.hist2 = ctx->hist + kBins1; sa.hist3 = ctx->hist + kBins1 + kBins2;
+  sa.sc = ctx->sc;
+  sa.cnt = ctx->chunk_off; sa.bk_off = ctx->bk_off; sa.bk_val = ctx->bk_val;
+  sa.n_chunks = ctx->n_chunks;
+  sa.k_total = uint32_t(ctx->k_global);
+  sa.spec_limit = uint32_t(std::min<int64_t>(ctx->d_global, 3 * ctx->k_global + 65536));
+  sa.cnt_gt = ctx->sel_gt; sa.cnt_eq = ctx->sel_eq; sa.blk_tot = ctx->blk_tot;
+  sa.shard_tot = ctx->shard_tot; sa.shard = ctx->shard; sa.n_shards = ctx->n_shards;
+  sa.sel_idx = ctx->sel_idx; sa.sel_val = ctx->sel_val;
+  sa.row_cap = k;
+  sa.values_bf16 = ctx->V16 ? 1 : 0;
+  sa.W = ctx->W; sa.n_slabs = ctx->n_slabs; sa.m = ctx->m; sa.slot = slot;
+  sa.offs = ctx->offs; sa.colsum = ctx->colsum; sa.order = ctx->order;
+  sa.row_idx = ctx->I + int64_t(slot) * k; sa.row_rel = ctx->R + int64_t(slot) * k;
+  sa.row_val = ctx->V + int64_t(slot) * k;
+  sa.row_v16 = ctx->V16 ? ctx->V16 + int64_t(slot) * k : nullptr;
+  sa.slab_ctr = ctx->slab_ctr; sa.vmax = ctx->vmax;
+  sa.bar = ctx->bar;
+  sa.phase_begin = pb; sa.phase_end = pe;
+  void* args[] = {&sa};
+  EFCP_CUDA(cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(k_select_insert),
+                                        dim3(ctx->sel_grid), dim3(kSelThreads), args,
+                                        kSelSmemBytes, st));
+  EFCP_LAUNCHED();
+  return EFCP_OK;
+}
+
+// Scalar products of every window row with the new row (one partial per slab and row).
+int launch_sp(efcp_ctx* ctx, int slot, cudaStream_t st) {
+  const int64_t k = ctx->k, d = ctx->d;
+  const int m = ctx->m;
   const bool acc_mode = (ctx->flags & EFCP_RHS_ACCUMULATOR) != 0;
-  double* rhs = dw + m;
-  double* wfin = rhs + m;
   const size_t smem = slab_smem_bytes(ctx->W, m);
-  prof_mark(ctx, 1, st);
 #define EFCP_SP_LAUNCH(ACC, VT, VPTR)                                                          \
   k_sp_rows<ACC, VT><<<ctx->grid_slab, kSlabThreads, smem, st>>>(                              \
       ctx->R, VPTR, ctx->V, ctx->offs, k, m, ctx->W, ctx->n_slabs, slot, ctx->slab_part,       \
@@ -614,51 +632,65 @@ static int step_impl(efcp_ctx* ctx, const float* grad, float* update, void* stre
   else EFCP_SP_LAUNCH(false, float, ctx->V);
 #undef EFCP_SP_LAUNCH
   EFCP_LAUNCHED();
-  prof_mark(ctx, 2, st);
+  return EFCP_OK;
+}
+
+// Phases [pb, pe) of the m x m kernel.
+int launch_mxm(efcp_ctx* ctx, int slot, int pb, int pe, cudaStream_t st) {
+  const int m = ctx->m;
+  const Vecs v = vecs_of(ctx);
+  MxmArgs ma{};
+  ma.slab_part = ctx->slab_part; ma.partial = ctx->partial;
+  ma.n_slabs = ctx->n_slabs;
+  ma.parts = ctx->n_slabs < kSpParts ? ctx->n_slabs : kSpParts;
+  ma.m = m; ma.slot = slot; ma.acc = (ctx->flags & EFCP_RHS_ACCUMULATOR) ? 1 : 0;
+  ma.mlambda = double(m) * double(ctx->lambda); ma.lambda = double(ctx->lambda);
+  ma.S = ctx->S; ma.B = ctx->B;
+  ma.delta = v.delta; ma.aprime = v.aprime; ma.y = v.y; ma.bold = v.bold; ma.w = v.w;
+  ma.res = v.res; ma.dw = v.dw; ma.rhs = v.rhs;
+  ma.sc = ctx->sc; ma.bar = ctx->bar + 2;
+  ma.phase_begin = pb; ma.phase_end = pe;
+  void* args[] = {&ma};
+  EFCP_CUDA(cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(k_mxm),
+                                        dim3(ctx->mxm_grid), dim3(kMxmThreads), args,
+                                        mxm_smem_bytes(m), st));
+  EFCP_LAUNCHED();
+  return EFCP_OK;
+}
+
+// Sparse GGT: eigendecomposition of S and the weights of u over the window rows.
+int launch_ggt(efcp_ctx* ctx, int slot, cudaStream_t st) {
+  const int m = ctx->m;
+  const Vecs v = vecs_of(ctx);
+  if (ggt_slots(m) <= 2)
+    k_ggt_weights<2><<<1, kGgtThreads, ggt_smem_bytes(m), st>>>(
+        ctx->S, m, slot, double(ctx->lambda), v.w, ctx->wf, ctx->sc, ctx->ggt_rot);
+  else
+    k_ggt_weights<4><<<1, kGgtThreads, ggt_smem_bytes(m), st>>>(
+        ctx->S, m, slot, double(ctx->lambda), v.w, ctx->wf, ctx->sc, ctx->ggt_rot);
+  EFCP_LAUNCHED();
+  return EFCP_OK;
+}
+
+// Linear combination of the window rows into `update` (or straight into the parameters).
+int launch_lcg(efcp_ctx* ctx, float* update, LcgApply ap, cudaStream_t st) {
+  const int64_t k = ctx->k, d = ctx->d;
+  const int m = ctx->m;
+  const Vecs v = vecs_of(ctx);
+  const bool acc_mode = (ctx->flags & EFCP_RHS_ACCUMULATOR) != 0;
   const bool ggt = (ctx->flags & EFCP_PRECOND_GGT) != 0;
-  {
-    // m x m: sums of the slab partials, S row/column, remove-and-border update of the
-    // inverse, weights, residual and the refinement's correction: one cooperative kernel
-    // (Sparse GGT: only the sums and S, its eigendecomposition follows)
-    MxmArgs ma{};
-    ma.slab_part = ctx->slab_part; ma.partial = ctx->partial;
-    ma.n_slabs = ctx->n_slabs;
-    ma.parts = ctx->n_slabs < kSpParts ? ctx->n_slabs : kSpParts;
-    ma.m = m; ma.slot = slot; ma.acc = acc_mode ? 1 : 0;
-    ma.mlambda = mlambda; ma.lambda = double(ctx->lambda);
-    ma.S = ctx->S; ma.B = ctx->B;
-    ma.delta = delta; ma.aprime = aprime; ma.y = y; ma.bold = bold; ma.w = w; ma.res = res;
-    ma.dw = dw; ma.rhs = rhs;
-    ma.sc = ctx->sc; ma.bar = ctx->bar + 2;
-    ma.phase_begin = 0; ma.phase_end = ggt ? 3 : kMxmPhases;
-    void* args[] = {&ma};
-    EFCP_CUDA(cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(k_mxm),
-                                          dim3(ctx->mxm_grid), dim3(kMxmThreads), args,
-                                          mxm_smem_bytes(m), st));
-    EFCP_LAUNCHED();
-  }
-  if (ggt) {
-    // m x m: eigendecomposition of S and the weights of u over the window rows
-    if (ggt_slots(m) <= 2)
-      k_ggt_weights<2><<<1, kGgtThreads, ggt_smem_bytes(m), st>>>(
-          ctx->S, m, slot, double(ctx->lambda), w, ctx->wf, ctx->sc, ctx->ggt_rot);
-    else
-      k_ggt_weights<4><<<1, kGgtThreads, ggt_smem_bytes(m), st>>>(
-          ctx->S, m, slot, double(ctx->lambda), w, ctx->wf, ctx->sc, ctx->ggt_rot);
-    EFCP_LAUNCHED();
-  }
-  // linear combination of the window rows
-  prof_mark(ctx, 3, st);
+  const size_t smem = slab_smem_bytes(ctx->W, m);
   const bool uvec = (reinterpret_cast<uintptr_t>(update) & 15) == 0;
   const float inv_lambda = 1.0f / ctx->lambda;
+  const double* dw = ggt ? nullptr : v.dw;
 #define EFCP_LCG_LAUNCH(VEC, ACC, VT, VPTR)                                                    \
   k_lcg<VEC, ACC, VT><<<ctx->grid_slab, kSlabThreads, smem, st>>>(                             \
-      ctx->R, VPTR, ctx->offs, k, m, ctx->W, ctx->n_slabs, w, ggt ? nullptr : dw, wfin, update, \
-      d, ctx->slab_ctr + 1, ctx->order, ctx->e, inv_lambda, ap)
+      ctx->R, VPTR, ctx->offs, k, m, ctx->W, ctx->n_slabs, v.w, dw, v.wfin, update, d,         \
+      ctx->slab_ctr + 1, ctx->order, ctx->e, inv_lambda, ap)
 #define EFCP_LCG_FIXED_LAUNCH(VEC, VT, VPTR)                                                    \
   k_lcg<VEC, false, VT, true><<<ctx->grid_slab, kSlabThreads, smem, st>>>(                     \
-      ctx->R, VPTR, ctx->offs, k, m, ctx->W, ctx->n_slabs, w, ggt ? nullptr : dw, wfin, update, \
-      d, ctx->slab_ctr + 1, ctx->order, ctx->e, inv_lambda, ap, ctx->vmax, ctx->lcg_redo,      \
+      ctx->R, VPTR, ctx->offs, k, m, ctx->W, ctx->n_slabs, v.w, dw, v.wfin, update, d,         \
+      ctx->slab_ctr + 1, ctx->order, ctx->e, inv_lambda, ap, ctx->vmax, ctx->lcg_redo,         \
       ctx->lcg_tol2)
   if (ctx->vmax) {
     if (ctx->V16) {
@@ -681,23 +713,150 @@ static int step_impl(efcp_ctx* ctx, const float* grad, float* update, void* stre
 #undef EFCP_LCG_LAUNCH
 #undef EFCP_LCG_FIXED_LAUNCH
   EFCP_LAUNCHED();
+  return EFCP_OK;
+}
+
+// EFCP_DEBUG_CHECKS: the new row's offsets, slab membership and 16-bit stream, and the slab
+// weights; a violation becomes the sticky internal-error status.
+int launch_debug_checks(efcp_ctx* ctx, int slot, cudaStream_t st) {
+  k_validate_rows<<<dim3(ctx->n_slabs, 1), 128, 0, st>>>(
+      ctx->I, ctx->R, ctx->offs, ctx->k, ctx->d, ctx->m, ctx->W, ctx->n_slabs, slot, slot + 1,
+      ctx->shard_tot ? 0 : 1, ctx->dbg_bad);
+  EFCP_LAUNCHED();
+  k_validate_colsum<<<ctx->n_slabs + 1, 256, 0, st>>>(ctx->offs, ctx->colsum, ctx->m,
+                                                      ctx->n_slabs, ctx->dbg_bad);
+  EFCP_LAUNCHED();
+  k_fold_bad<<<1, 1, 0, st>>>(ctx->dbg_bad, ctx->sc);
+  EFCP_LAUNCHED();
+  return EFCP_OK;
+}
+
+#define EFCP_TRY(call)             \
+  do {                             \
+    const int rc__ = (call);       \
+    if (rc__ != EFCP_OK) return rc__; \
+  } while (0)
+
+// One step: five launches (six for Sparse GGT).  With ap.theta set the linear combination
+// updates the parameters in place of writing u (update may then be NULL).
+int step_impl(efcp_ctx* ctx, const float* grad, float* update, void* stream_, LcgApply ap) {
+  if (!ctx || !grad || (!update && !ap.theta) || grad == update) return EFCP_EINVAL;
+  if (ctx->shard_tot) return EFCP_EINVAL;  // a shard steps through efcp_shard_phase
+  cudaStream_t st = static_cast<cudaStream_t>(stream_);
+  EFCP_CUDA(cudaSetDevice(ctx->device));  // the launches below go to the handle's device
+  const int slot = int(ctx->t % ctx->m);
+  const bool ggt = (ctx->flags & EFCP_PRECOND_GGT) != 0;
+  ctx->launches = 0;
+  prof_mark(ctx, 0, st);
+  EFCP_TRY(launch_ef(ctx, grad, st));
+  // global Top-k: exact selection, residual and ring insert; block-wise Top-k has selected
+  // already, only the ring insert is left
+  EFCP_TRY(launch_select(ctx, slot, ctx->block ? 4 : 0, kSelPhases, st));
+  prof_mark(ctx, 1, st);
+  EFCP_TRY(launch_sp(ctx, slot, st));
+  prof_mark(ctx, 2, st);
+  // m x m: sums of the slab partials, S row/column, remove-and-border update of the inverse,
+  // weights, residual and the refinement's correction (Sparse GGT: the sums and S, then its
+  // eigendecomposition)
+  EFCP_TRY(launch_mxm(ctx, slot, 0, ggt ? 3 : kMxmPhases, st));
+  if (ggt) EFCP_TRY(launch_ggt(ctx, slot, st));
+  prof_mark(ctx, 3, st);
+  EFCP_TRY(launch_lcg(ctx, update, ap, st));
   prof_mark(ctx, 4, st);
-  if (ctx->flags & EFCP_DEBUG_CHECKS) {
-    // the new row's offsets, slab membership and 16-bit stream, and the slab weights; a
-    // violation becomes the sticky internal-error status
-    k_validate_rows<<<dim3(ctx->n_slabs, 1), 128, 0, st>>>(ctx->I, ctx->R, ctx->offs, k, d, m,
-                                                           ctx->W, ctx->n_slabs, slot, slot + 1,
-                                                           ctx->dbg_bad);
-    EFCP_LAUNCHED();
-    k_validate_colsum<<<ctx->n_slabs + 1, 256, 0, st>>>(ctx->offs, ctx->colsum, m, ctx->n_slabs,
-                                                        ctx->dbg_bad);
-    EFCP_LAUNCHED();
-    k_fold_bad<<<1, 1, 0, st>>>(ctx->dbg_bad, ctx->sc);
-    EFCP_LAUNCHED();
-  }
+  if (ctx->flags & EFCP_DEBUG_CHECKS) EFCP_TRY(launch_debug_checks(ctx, slot, st));
   if (ctx->prof_on && ctx->prof_n < ctx->prof_cap) ++ctx->prof_n;
   ctx->t += 1;
   return EFCP_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+/*
+ * Coordinate-sharded state.  Phase p of a step (0..5) runs on every shard, then buffer p is
+ * summed over the shards (an all-reduce), then phase p + 1 runs:
+ *   0  a = xi + g on the shard's coordinates, digit-1 histogram      -> buffer 0: histogram 1
+ *   1  threshold bin of digit 1 (from the summed histogram), digit 2 -> buffer 1: histogram 2
+ *   2  threshold bin of digit 2, digit 3                             -> buffer 2: histogram 3
+ *   3  exact threshold key, the shard's counts above and at the key  -> buffer 3: the counts
+ *   4  selection (equal keys go to the shards of lower coordinates first), ring insert,
+ *      the shard's part of the scalar products                       -> buffer 4: delta
+ *   5  S, the m x m stage (replicated), the shard's part of the update
+ */
+int efcp_shard_phase(efcp_ctx* ctx, int32_t phase, const float* grad, float* update,
+                     void* stream_) {
+  if (!ctx || !ctx->shard_tot || phase < 0 || phase > 5) return EFCP_EINVAL;
+  if ((phase == 0 && !grad) || (phase == 5 && !update) || phase != ctx->next_phase)
+    return EFCP_EINVAL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream_);
+  EFCP_CUDA(cudaSetDevice(ctx->device));
+  const int slot = int(ctx->t % ctx->m);
+  switch (phase) {
+    case 0:
+      ctx->launches = 0;
+      EFCP_CUDA(cudaMemsetAsync(ctx->shard_tot, 0, size_t(ctx->n_shards) * 8, st));
+      EFCP_TRY(launch_ef(ctx, grad, st));
+      break;
+    case 1: EFCP_TRY(launch_select(ctx, slot, 0, 1, st)); break;
+    case 2: EFCP_TRY(launch_select(ctx, slot, 1, 2, st)); break;
+    case 3: EFCP_TRY(launch_select(ctx, slot, 2, 3, st)); break;
+    case 4:
+      EFCP_TRY(launch_select(ctx, slot, 3, kSelPhases, st));
+      EFCP_TRY(launch_sp(ctx, slot, st));
+      EFCP_TRY(launch_mxm(ctx, slot, 0, 2, st));
+      break;
+    default:
+      EFCP_TRY(launch_mxm(ctx, slot, 2, kMxmPhases, st));
+      EFCP_TRY(launch_lcg(ctx, update, LcgApply{nullptr, 0.f, 0.f}, st));
+      if (ctx->flags & EFCP_DEBUG_CHECKS) EFCP_TRY(launch_debug_checks(ctx, slot, st));
+      ctx->t += 1;
+      break;
+  }
+  ctx->next_phase = (phase + 1) % 6;
+  return EFCP_OK;
+}
+
+int efcp_shard_buffer(efcp_ctx* ctx, int32_t phase, void** dev_ptr, int64_t* count,
+                      int32_t* is_f64) {
+  if (!ctx || !ctx->shard_tot || !dev_ptr || !count || !is_f64 || phase < 0 || phase > 4)
+    return EFCP_EINVAL;
+  *is_f64 = phase == 4 ? 1 : 0;
+  switch (phase) {
+    case 0: *dev_ptr = ctx->hist; *count = kBins1; break;
+    case 1: *dev_ptr = ctx->hist + kBins1; *count = kBins2; break;
+    case 2: *dev_ptr = ctx->hist + kBins1 + kBins2; *count = kBins3; break;
+    case 3: *dev_ptr = ctx->shard_tot; *count = 2 * int64_t(ctx->n_shards); break;
+    default: *dev_ptr = ctx->vecs; *count = ctx->m; break;
+  }
+  return EFCP_OK;
+}
+
+int efcp_create_shard(efcp_ctx** out, int64_t d_global, int64_t d_lo, int64_t d_hi, int32_t m,
+                      int64_t k_global, int64_t row_cap, float lambda, uint32_t flags,
+                      int32_t shard, int32_t n_shards) {
+  if (!out) return EFCP_EINVAL;
+  *out = nullptr;
+  if (n_shards < 1 || n_shards > 1024 || shard < 0 || shard >= n_shards || d_lo < 0 ||
+      d_hi <= d_lo || d_hi > d_global || !valid_args(d_global, m, k_global))
+    return EFCP_EINVAL;
+  if (flags & (EFCP_RHS_ACCUMULATOR | EFCP_PRECOND_GGT)) return EFCP_EINVAL;
+  const int64_t d_loc = d_hi - d_lo;
+  if (row_cap <= 0) row_cap = std::min(k_global, d_loc);  // whatever the shard could be given
+  if (row_cap > d_loc) return EFCP_EINVAL;
+  ShardSpec sp{d_global, k_global, shard, n_shards};
+  return create_impl(out, d_loc, m, row_cap, lambda, flags, 0, nullptr, 0, true, &sp);
+}
+
+int64_t efcp_row_count(efcp_ctx* ctx, int32_t slot) {
+  if (!ctx || slot < 0 || slot >= ctx->m) return -1;
+  if (!ctx->shard_tot) return ctx->k;
+  int32_t n = 0;
+  if (cudaSetDevice(ctx->device) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess ||
+      cudaMemcpy(&n, ctx->offs + int64_t(ctx->n_slabs) * ctx->m + slot, 4,
+                 cudaMemcpyDeviceToHost) != cudaSuccess)
+    return -1;
+  return n;
 }
 
 int efcp_step(efcp_ctx* ctx, const float* grad, float* update, void* stream) {
@@ -803,16 +962,27 @@ int efcp_get_row(efcp_ctx* ctx, int32_t slot, int32_t* host_idx, float* host_val
   const size_t bytes = size_t(ctx->k) * 4;
   EFCP_CUDA(cudaMemcpy(host_idx, ctx->I + int64_t(slot) * ctx->k, bytes, cudaMemcpyDeviceToHost));
   EFCP_CUDA(cudaMemcpy(host_val, ctx->V + int64_t(slot) * ctx->k, bytes, cudaMemcpyDeviceToHost));
+  int64_t n = ctx->k;  // a shard's row holds what the step gave it; the rest reads as (0, 0)
+  if (ctx->shard_tot) {
+    int32_t cnt = 0;
+    EFCP_CUDA(cudaMemcpy(&cnt, ctx->offs + int64_t(ctx->n_slabs) * ctx->m + slot, 4,
+                         cudaMemcpyDeviceToHost));
+    n = std::max<int64_t>(0, std::min<int64_t>(cnt, ctx->k));
+    for (int64_t j = n; j < ctx->k; ++j) {
+      host_idx[j] = 0;
+      host_val[j] = 0.f;
+    }
+  }
   // the device keeps every slab segment of a row in a bank-interleaved order; callers get
   // the row in ascending index order (indices within a row are distinct)
   try {
-    std::vector<std::pair<int32_t, float>> tmp(static_cast<size_t>(ctx->k));
-    for (int64_t j = 0; j < ctx->k; ++j) tmp[size_t(j)] = {host_idx[j], host_val[j]};
+    std::vector<std::pair<int32_t, float>> tmp(static_cast<size_t>(n));
+    for (int64_t j = 0; j < n; ++j) tmp[size_t(j)] = {host_idx[j], host_val[j]};
     std::sort(tmp.begin(), tmp.end(),
               [](const std::pair<int32_t, float>& a, const std::pair<int32_t, float>& b) {
                 return a.first < b.first;
               });
-    for (int64_t j = 0; j < ctx->k; ++j) {
+    for (int64_t j = 0; j < n; ++j) {
       host_idx[j] = tmp[size_t(j)].first;
       host_val[j] = tmp[size_t(j)].second;
     }
@@ -908,7 +1078,8 @@ int efcp_validate(efcp_ctx* ctx, int64_t* bad_out) {
   const int rows = int(ctx->t < ctx->m ? ctx->t : ctx->m);
   if (rows > 0) {
     k_validate_rows<<<dim3(ctx->n_slabs, rows), 128>>>(ctx->I, ctx->R, ctx->offs, ctx->k, ctx->d,
-                                                       ctx->m, ctx->W, ctx->n_slabs, 0, rows, bad);
+                                                       ctx->m, ctx->W, ctx->n_slabs, 0, rows,
+                                                       ctx->shard_tot ? 0 : 1, bad);
   }
   k_validate_colsum<<<ctx->n_slabs + 1, 256>>>(ctx->offs, ctx->colsum, ctx->m, ctx->n_slabs, bad);
   unsigned long long h = 0;

@@ -380,7 +380,8 @@ __global__ void __launch_bounds__(kSelThreads) k_select_insert(const SelectArgs 
       }
     } else if (phase == 4) {
       // ---- the new row's offset in every slab; slab weights
-      const int64_t n_sel = A.sc->n_sel;
+      // an unsharded row always holds row_cap entries; a shard keeps what phase 3 counted
+      const int64_t n_sel = A.shard_tot ? int64_t(A.sc->n_sel) : A.row_cap;
       row_offsets(A.sel_idx, n_sel, A.W, A.n_slabs, A.m, A.slot, A.offs, A.colsum,
                   int64_t(blockIdx.x) * kSelThreads + tid, int64_t(gridDim.x) * kSelThreads);
     } else {

@@ -51,6 +51,21 @@ def test_two_gloo_ranks_barrier_and_max_over_ranks():
     assert rows[0]["g0"] != rows[1]["g0"]           # replicas draw different streams
 
 
+def test_sharded_step_orchestration_over_two_gloo_ranks():
+    """The coordinate-sharded step's host logic (phase order, which buffers are summed, who
+    gets the gradient and the update) with all-reduces over gloo: two ranks, each holding a
+    numpy stand-in of one shard that follows the library's phase protocol, must together
+    reproduce the unsharded oracle - state bit for bit, ties at the threshold split across
+    the boundary included."""
+    r = torchrun([os.path.join("tests", "shard_worker.py")])
+    assert r.returncode == 0, r.stderr[-2000:]
+    rows = sorted(json_lines(r.stdout), key=lambda x: x["rank"])
+    assert [x["rank"] for x in rows] == [0, 1]
+    assert all(x["order_ok"] for x in rows)
+    assert rows[0]["state_ok"]
+    assert rows[0]["worst_u"] <= 1e-6
+
+
 def test_reference_arm_prints_once_under_two_ranks():
     r = torchrun(["bench.py", "--impl", "reference", "--gpus", "2", "--steps", "2",
                   "--warmup", "1", "--workload", "c1_d65536_m32"])
