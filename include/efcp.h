@@ -47,6 +47,9 @@ typedef struct efcp_ctx efcp_ctx;
  *   EFCP_LCG_FIXED_TOL=x  0 <= x <= 1e-4: relative error a slab of the fixed-point accumulator
  *                         may have before it is accumulated again in fp32 (default 1e-5; 0
  *                         sends every slab through the fp32 route).
+ *   EFCP_SPLIT_PHASES=1   the two cooperative kernels of a step are launched once per phase
+ *                         instead of once per step, so that a profiler's launch list shows
+ *                         what each phase costs.  Same results, more launches.
  *   EFCP_SLAB_W=n         slab width in coordinates (multiple of 32, 256..49152) instead of the
  *                         width chosen from d, m and the SM count.  The width is part of a
  *                         checkpoint's header: a state imports only into a handle created with

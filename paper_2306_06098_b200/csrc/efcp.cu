@@ -81,6 +81,7 @@ struct efcp_ctx {
   uint32_t* shard_tot = nullptr;  // per shard: entries above / at the threshold key
   int next_phase = 0;             // of efcp_shard_phase
   bool is_shard = false;
+  bool split_phases = false;      // EFCP_SPLIT_PHASES=1: one launch per phase (profiling)
   float* wf = nullptr;
   int* slab_ctr = nullptr;   // work counters of the slab kernels (SP, LCG)
   int64_t* colsum = nullptr; // n_slabs + 1 column sums of offs
@@ -303,6 +304,7 @@ int configure(efcp_ctx* ctx, int64_t d, int32_t m, int64_t k, float lambda, uint
   ctx->W = z.W; ctx->n_slabs = z.n_slabs; ctx->n_chunks = z.n_chunks;
   ctx->grid_slab = z.grid_slab;
   if (const char* env = getenv("EFCP_NO_SPEC")) ctx->spec = atoi(env) == 0;
+  if (const char* env = getenv("EFCP_SPLIT_PHASES")) ctx->split_phases = atoi(env) != 0;
   // EFCP_LCG_FIXED_TOL: relative error a slab of the fixed-point LCG may have before it is redone
   // in fp32 (default 1e-5; 0 sends every slab through the fallback, which a parity test does)
   if (const char* env = getenv("EFCP_LCG_FIXED_TOL")) {
@@ -418,8 +420,9 @@ bool init_state(efcp_ctx* ctx) {
     });
   }
   {
-    // the cooperative kernels: as many blocks as are resident together, at most 2 per SM
-    // (a grid-wide barrier costs in proportion to the number of blocks)
+    // the cooperative kernels: as many blocks as are resident together, at most 2 (m x m)
+    // or 4 (selection: its passes are latency bound) per SM; a grid-wide barrier costs in
+    // proportion to the number of blocks
     int occ = 0;
     ok &= cudaFuncSetAttribute(k_mxm, attr, int(mxm_smem_bytes(m))) == cudaSuccess;
     ok &= cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_mxm, kMxmThreads,
@@ -430,7 +433,7 @@ bool init_state(efcp_ctx* ctx) {
     ok &= cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_select_insert, kSelThreads,
                                                         kSelSmemBytes) == cudaSuccess;
     ok &= occ >= 1;
-    ctx->sel_grid = std::min(kMaxCoopBlocks, ctx->num_sms * std::min(occ, 2));
+    ctx->sel_grid = std::min(kMaxCoopBlocks, ctx->num_sms * std::min(occ, 4));
   }
   if (ctx->flags & EFCP_PRECOND_GGT)
     ok &= cudaFuncSetAttribute(ggt_slots(m) <= 2 ? k_ggt_weights<2> : k_ggt_weights<4>, attr,
@@ -751,14 +754,24 @@ int step_impl(efcp_ctx* ctx, const float* grad, float* update, void* stream_, Lc
   EFCP_TRY(launch_ef(ctx, grad, st));
   // global Top-k: exact selection, residual and ring insert; block-wise Top-k has selected
   // already, only the ring insert is left
-  EFCP_TRY(launch_select(ctx, slot, ctx->block ? 4 : 0, kSelPhases, st));
+  if (ctx->split_phases) {
+    for (int ph = ctx->block ? 4 : 0; ph < kSelPhases; ++ph)
+      EFCP_TRY(launch_select(ctx, slot, ph, ph + 1, st));
+  } else {
+    EFCP_TRY(launch_select(ctx, slot, ctx->block ? 4 : 0, kSelPhases, st));
+  }
   prof_mark(ctx, 1, st);
   EFCP_TRY(launch_sp(ctx, slot, st));
   prof_mark(ctx, 2, st);
   // m x m: sums of the slab partials, S row/column, remove-and-border update of the inverse,
   // weights, residual and the refinement's correction (Sparse GGT: the sums and S, then its
   // eigendecomposition)
-  EFCP_TRY(launch_mxm(ctx, slot, 0, ggt ? 3 : kMxmPhases, st));
+  if (ctx->split_phases) {
+    for (int ph = 0; ph < (ggt ? 3 : kMxmPhases); ++ph)
+      EFCP_TRY(launch_mxm(ctx, slot, ph, ph + 1, st));
+  } else {
+    EFCP_TRY(launch_mxm(ctx, slot, 0, ggt ? 3 : kMxmPhases, st));
+  }
   if (ggt) EFCP_TRY(launch_ggt(ctx, slot, st));
   prof_mark(ctx, 3, st);
   EFCP_TRY(launch_lcg(ctx, update, ap, st));

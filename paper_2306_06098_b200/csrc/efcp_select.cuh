@@ -19,8 +19,11 @@
 //   5  slabs ordered heavy first; the row goes into the ring slot, every slab segment in the
 //      bank-interleaved order the slab kernels want
 //
-// Chunks are owned by blocks in contiguous runs, so that a block can rank its own chunks
-// from the totals of the blocks before it.  A launch runs the phases [phase_begin,
+// A warp works on a group of kSelGroup consecutive chunks at a time: their buckets, each a
+// few dozen entries at the benchmark's densities, are walked as one list in index order, so
+// that a warp has many independent loads in flight instead of a short dependent chain per
+// chunk.  Groups are owned by blocks in contiguous runs, so that a block can rank its own
+// groups from the totals of the blocks before it.  A launch runs the phases [phase_begin,
 // phase_end); a caller that has to exchange something between two phases (histograms summed
 // over the shards of a coordinate-sharded state) launches the ranges one after the other.
 // The buckets are the candidate list: nothing is compacted in between.
@@ -35,6 +38,7 @@ namespace efcp {
 constexpr int kSelThreads = 256;
 constexpr int kSelWarps = kSelThreads / 32;
 constexpr int kSelPhases = 6;
+constexpr int kSelGroup = 8;  // chunks whose buckets a warp walks as one list
 
 // dynamic shared memory: the larger of one histogram of digit 1 and the staging of phase 5
 constexpr size_t kSelLayoutBytes =
@@ -57,7 +61,7 @@ struct SelectArgs {
   uint32_t k_total;   // entries to keep (over all shards)
   uint32_t spec_limit;
   // ranking
-  int32_t* cnt_gt;    // per chunk: entries above T, then their exclusive prefix
+  int32_t* cnt_gt;    // per group of chunks: entries above T, then their exclusive prefix
   int32_t* cnt_eq;    // same for the entries equal to T
   int32_t* blk_tot;   // per block: totals of its chunks (gt, then eq at + gridDim.x)
   // a coordinate-sharded state: totals of every shard (gt, eq pairs, shard order = coordinate
@@ -121,6 +125,33 @@ __device__ __forceinline__ void flush_hist(const uint32_t* h, uint32_t* __restri
   }
 }
 
+// The buckets of the chunks [ch0, ch0 + kSelGroup) as one list in index order: calls
+// f(on, value, chunk, position in the chunk's bucket) for every entry, 32 entries per
+// call round (`on` is false for the lanes past the end of the last round, so f may vote).
+template <typename F>
+__device__ __forceinline__ void walk_group(const SelectArgs& A, int ch0, int lane, F&& f) {
+  const int nch = min(kSelGroup, A.n_chunks - ch0);
+  const int mine = lane < nch ? A.cnt[ch0 + lane] : 0;
+  int pre[kSelGroup + 1];  // exclusive prefix of the bucket fills, the same in every lane
+  pre[0] = 0;
+#pragma unroll
+  for (int q = 0; q < kSelGroup; ++q) pre[q + 1] = pre[q] + __shfl_sync(0xFFFFFFFFu, mine, q);
+  const int total = pre[kSelGroup];
+  for (int f0 = 0; f0 < total; f0 += 32) {
+    const int fl = f0 + lane;
+    const bool on = fl < total;
+    int t = 0;
+#pragma unroll
+    for (int q = 1; q < kSelGroup; ++q) t += fl >= pre[q] ? 1 : 0;
+    int base = 0;
+#pragma unroll
+    for (int q = 1; q < kSelGroup; ++q) base = t == q ? pre[q] : base;
+    const int ch = ch0 + (on ? t : 0), i = on ? fl - base : 0;
+    const float v = on ? A.bk_val[int64_t(ch) * kChunk + i] : 0.f;
+    f(on, v, ch, i);
+  }
+}
+
 __global__ void __launch_bounds__(kSelThreads) k_select_insert(const SelectArgs A) {
   extern __shared__ __align__(16) unsigned char sel_smraw[];
   uint32_t* hs = reinterpret_cast<uint32_t*>(sel_smraw);
@@ -129,10 +160,12 @@ __global__ void __launch_bounds__(kSelThreads) k_select_insert(const SelectArgs 
   __shared__ int s_tot[2];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const unsigned lt = (1u << lane) - 1u;
-  // the chunks this block owns
-  const int per_block = (A.n_chunks + int(gridDim.x) - 1) / int(gridDim.x);
-  const int ch_lo = min(A.n_chunks, int(blockIdx.x) * per_block);
-  const int ch_hi = min(A.n_chunks, ch_lo + per_block);
+  // the groups of chunks this block owns
+  const int n_groups = (A.n_chunks + kSelGroup - 1) / kSelGroup;
+  const int per_block = (n_groups + int(gridDim.x) - 1) / int(gridDim.x);
+  const int gr_lo = min(n_groups, int(blockIdx.x) * per_block);
+  const int gr_hi = min(n_groups, gr_lo + per_block);
+  const int ch_lo = gr_lo * kSelGroup, ch_hi = min(A.n_chunks, gr_hi * kSelGroup);
   unsigned int barriers = 0;
   for (int phase = A.phase_begin; phase < A.phase_end; ++phase) {
     if (phase > A.phase_begin) {
@@ -193,14 +226,11 @@ __global__ void __launch_bounds__(kSelThreads) k_select_insert(const SelectArgs 
       }
       for (int i = tid; i < kBins2; i += kSelThreads) hs[i] = 0u;
       __syncthreads();
-      for (int ch = ch_lo + warp; ch < ch_hi; ch += kSelWarps) {
-        const int n = A.cnt[ch];
-        const float* bv = A.bk_val + int64_t(ch) * kChunk;
-        for (int i = lane; i < n; i += 32) {
-          const uint32_t key = mag_key(bv[i]);
-          if ((key >> kShift1) == b1) atomicAdd(&hs[(key >> kShift2) & (kBins2 - 1)], 1u);
-        }
-      }
+      for (int gr = gr_lo + warp; gr < gr_hi; gr += kSelWarps)
+        walk_group(A, gr * kSelGroup, lane, [&](bool on, float v, int, int) {
+          const uint32_t key = mag_key(v);
+          if (on && (key >> kShift1) == b1) atomicAdd(&hs[(key >> kShift2) & (kBins2 - 1)], 1u);
+        });
       flush_hist(hs, A.hist2, kBins2);
     } else if (phase == 1) {
       // ---- digit 2: threshold bin, digit-3 histogram
@@ -221,14 +251,11 @@ __global__ void __launch_bounds__(kSelThreads) k_select_insert(const SelectArgs 
       for (int i = tid; i < kBins3; i += kSelThreads) hs[i] = 0u;
       __syncthreads();
       const uint32_t prefix = (b1 << kBits2) | b2;
-      for (int ch = ch_lo + warp; ch < ch_hi; ch += kSelWarps) {
-        const int n = A.cnt[ch];
-        const float* bv = A.bk_val + int64_t(ch) * kChunk;
-        for (int i = lane; i < n; i += 32) {
-          const uint32_t key = mag_key(bv[i]);
-          if ((key >> kShift2) == prefix) atomicAdd(&hs[key & (kBins3 - 1)], 1u);
-        }
-      }
+      for (int gr = gr_lo + warp; gr < gr_hi; gr += kSelWarps)
+        walk_group(A, gr * kSelGroup, lane, [&](bool on, float v, int, int) {
+          const uint32_t key = mag_key(v);
+          if (on && (key >> kShift2) == prefix) atomicAdd(&hs[key & (kBins3 - 1)], 1u);
+        });
       flush_hist(hs, A.hist3, kBins3);
     } else if (phase == 2) {
       // ---- digit 3: the exact threshold key; per chunk, entries above it and equal to it
@@ -247,19 +274,16 @@ __global__ void __launch_bounds__(kSelThreads) k_select_insert(const SelectArgs 
         for (int i = tid; i < kBins2; i += kSelThreads) A.hist2[i] = 0u;
       }
       int w_gt = 0, w_eq = 0;
-      for (int ch = ch_lo + warp; ch < ch_hi; ch += kSelWarps) {
-        const int n = A.cnt[ch];
-        const float* bv = A.bk_val + int64_t(ch) * kChunk;
+      for (int gr = gr_lo + warp; gr < gr_hi; gr += kSelWarps) {
         int gt = 0, eq = 0;
-        for (int i0 = 0; i0 < n; i0 += 32) {
-          const int i = i0 + lane;
-          const uint32_t key = i < n ? mag_key(bv[i]) : 0u;
-          gt += __popc(__ballot_sync(0xFFFFFFFFu, i < n && key > T));
-          eq += __popc(__ballot_sync(0xFFFFFFFFu, i < n && key == T));
-        }
+        walk_group(A, gr * kSelGroup, lane, [&](bool on, float v, int, int) {
+          const uint32_t key = mag_key(v);
+          gt += __popc(__ballot_sync(0xFFFFFFFFu, on && key > T));
+          eq += __popc(__ballot_sync(0xFFFFFFFFu, on && key == T));
+        });
         if (lane == 0) {
-          A.cnt_gt[ch] = gt;
-          A.cnt_eq[ch] = eq;
+          A.cnt_gt[gr] = gt;
+          A.cnt_eq[gr] = eq;
         }
         w_gt += gt;
         w_eq += eq;
@@ -327,43 +351,37 @@ __global__ void __launch_bounds__(kSelThreads) k_select_insert(const SelectArgs 
         }
         for (int i = tid; i < kBins3; i += kSelThreads) A.hist3[i] = 0u;
       }
-      // exclusive prefix of this block's chunk counts, in place
+      // exclusive prefix of this block's group counts, in place
       int run_gt = base_gt;
       int64_t run_eq = base_eq;
-      for (int c0 = ch_lo; c0 < ch_hi; c0 += kSelThreads) {
-        const int ch = c0 + tid;
-        const int g = ch < ch_hi ? A.cnt_gt[ch] : 0;
-        const int q = ch < ch_hi ? A.cnt_eq[ch] : 0;
+      for (int c0 = gr_lo; c0 < gr_hi; c0 += kSelThreads) {
+        const int gr = c0 + tid;
+        const int g = gr < gr_hi ? A.cnt_gt[gr] : 0;
+        const int q = gr < gr_hi ? A.cnt_eq[gr] : 0;
         int tg, tq;
         const int eg = block_excl_scan<int>(g, &tg, smi);
         const int eq = block_excl_scan<int>(q, &tq, smi);
-        if (ch < ch_hi) {
-          A.cnt_gt[ch] = run_gt + eg;
-          A.cnt_eq[ch] = int32_t(min(run_eq + eq, int64_t(0x7FFFFFFF)));
+        if (gr < gr_hi) {
+          A.cnt_gt[gr] = run_gt + eg;
+          A.cnt_eq[gr] = int32_t(min(run_eq + eq, int64_t(0x7FFFFFFF)));
         }
         run_gt += tg;
         run_eq += tq;
       }
       __syncthreads();
-      for (int ch = ch_lo + warp; ch < ch_hi; ch += kSelWarps) {
-        const int n = A.cnt[ch];
-        if (n == 0) continue;
-        const uint16_t* bo = A.bk_off + int64_t(ch) * kChunk;
-        const float* bv = A.bk_val + int64_t(ch) * kChunk;
-        const int64_t eq_before_chunk = A.cnt_eq[ch];
-        int64_t pos0 = out_base + A.cnt_gt[ch] + min(eq_before_chunk, n_eq);
-        int64_t eq_run = eq_before_chunk;
-        for (int i0 = 0; i0 < n; i0 += 32) {
-          const int i = i0 + lane;
-          const float v = i < n ? bv[i] : 0.f;
+      for (int gr = gr_lo + warp; gr < gr_hi; gr += kSelWarps) {
+        const int64_t eq_before_group = A.cnt_eq[gr];
+        int64_t pos0 = out_base + A.cnt_gt[gr] + min(eq_before_group, n_eq);
+        int64_t eq_run = eq_before_group;
+        walk_group(A, gr * kSelGroup, lane, [&](bool on, float v, int ch, int i) {
           const uint32_t key = mag_key(v);
-          const bool is_gt = i < n && key > T, is_eq = i < n && key == T;
+          const bool is_gt = on && key > T, is_eq = on && key == T;
           const unsigned eqb = __ballot_sync(0xFFFFFFFFu, is_eq);
           const bool keep = is_gt || (is_eq && eq_run + __popc(eqb & lt) < n_eq);
           const unsigned kb = __ballot_sync(0xFFFFFFFFu, keep);
           const int64_t pos = pos0 + __popc(kb & lt);
           if (keep && pos < A.row_cap) {
-            const int64_t j = int64_t(ch) * kChunk + bo[i];
+            const int64_t j = int64_t(ch) * kChunk + A.bk_off[int64_t(ch) * kChunk + i];
             A.sel_idx[pos] = int32_t(j);
             if (A.values_bf16) {  // c holds the rounded value, the residue stays in xi (exact)
               const float r = bf16_to_float(bf16_bits_rn(v));
@@ -376,7 +394,7 @@ __global__ void __launch_bounds__(kSelThreads) k_select_insert(const SelectArgs 
           }
           pos0 += __popc(kb);
           eq_run += __popc(eqb);
-        }
+        });
       }
     } else if (phase == 4) {
       // ---- the new row's offset in every slab; slab weights
@@ -384,6 +402,10 @@ __global__ void __launch_bounds__(kSelThreads) k_select_insert(const SelectArgs 
       const int64_t n_sel = A.shard_tot ? int64_t(A.sc->n_sel) : A.row_cap;
       row_offsets(A.sel_idx, n_sel, A.W, A.n_slabs, A.m, A.slot, A.offs, A.colsum,
                   int64_t(blockIdx.x) * kSelThreads + tid, int64_t(gridDim.x) * kSelThreads);
+      if (A.vmax)  // the insert below takes maxima into these
+        for (int64_t s2 = int64_t(blockIdx.x) * kSelThreads + tid; s2 < A.n_slabs;
+             s2 += int64_t(gridDim.x) * kSelThreads)
+          A.vmax[s2 * A.m + A.slot] = 0.f;
     } else {
       // ---- slabs heavy first (one block), and the row into its ring slot
       if (blockIdx.x == gridDim.x - 1) {
@@ -392,9 +414,10 @@ __global__ void __launch_bounds__(kSelThreads) k_select_insert(const SelectArgs 
         if (tid < 2) A.slab_ctr[tid] = 0;  // work counters of the two slab kernels
         __syncthreads();
       }
-      layout_row_slabs<kSelWarps>(A.sel_idx, A.sel_val, A.W, A.n_slabs, A.m, A.slot, A.offs,
-                                  A.row_idx, A.row_rel, A.row_val, A.row_v16, A.vmax, sel_smraw,
-                                  reinterpret_cast<float*>(sm), int(blockIdx.x), int(gridDim.x));
+      layout_row_slabs(A.sel_idx, A.sel_val, A.W, A.n_slabs, A.m, A.slot, A.offs, A.row_idx,
+                       A.row_rel, A.row_val, A.row_v16, A.vmax,
+                       sel_smraw + size_t(warp) * (kLayoutChunk * 10 + 128),
+                       int(blockIdx.x) * kSelWarps + warp, int(gridDim.x) * kSelWarps);
     }
   }
   grid_exit(A.bar);

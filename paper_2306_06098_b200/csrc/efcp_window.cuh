@@ -100,26 +100,29 @@ __device__ __forceinline__ void slab_order_block(const int64_t* __restrict__ col
 
 // Insert of the new row: from the ascending (index, value) list of the selection,
 //   ring slot <- the row, every segment [offs[s][slot], offs[s+1][slot]) in the
-//   bank-interleaved order described above.  The calling block (NW warps) takes the slabs
-//   block_id, block_id + n_blocks, ...; its warps share the chunks of a segment.  smraw: NW *
-//   (kLayoutChunk * 10 + 128) bytes of shared memory, s_max: NW floats.
-template <int NW>
+//   bank-interleaved order described above.  One warp handles one chunk at a time; a slab's
+//   chunks are shared by `wps` warps (1, 2, 4 or 8: as many as there are warps to go round),
+//   warp `gwarp` of `nwarps` taking the (slab, part) pairs gwarp, gwarp + nwarps, ...
+//   smraw: this warp's kLayoutChunk * 10 + 128 bytes of shared memory.  vmax[s][slot] must be
+//   zero on entry; it receives the largest magnitude of the segment.
 __device__ __forceinline__ void layout_row_slabs(
     const int32_t* __restrict__ src_idx, const float* __restrict__ src_val, int W, int n_slabs,
     int m, int slot, const int32_t* __restrict__ offs, int32_t* __restrict__ dst_idx,
     uint16_t* __restrict__ dst_rel, float* __restrict__ dst_val, bf16raw* __restrict__ dst_v16,
-    float* __restrict__ vmax, unsigned char* smraw, float* s_max, int block_id, int n_blocks) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  int32_t* ci = reinterpret_cast<int32_t*>(smraw) + warp * kLayoutChunk;
-  float* cv = reinterpret_cast<float*>(smraw + size_t(NW) * kLayoutChunk * 4) + warp * kLayoutChunk;
-  uint16_t* cq =
-      reinterpret_cast<uint16_t*>(smraw + size_t(NW) * kLayoutChunk * 8) + warp * kLayoutChunk;
-  int* cnt = reinterpret_cast<int*>(smraw + size_t(NW) * kLayoutChunk * 10) + warp * 32;
-  for (int s = block_id; s < n_slabs; s += n_blocks) {
+    float* __restrict__ vmax, unsigned char* smraw, int gwarp, int nwarps) {
+  const int lane = threadIdx.x & 31;
+  int32_t* ci = reinterpret_cast<int32_t*>(smraw);
+  float* cv = reinterpret_cast<float*>(smraw + kLayoutChunk * 4);
+  uint16_t* cq = reinterpret_cast<uint16_t*>(smraw + kLayoutChunk * 8);
+  int* cnt = reinterpret_cast<int*>(smraw + kLayoutChunk * 10);
+  int wps = 1;
+  while (wps < 8 && int64_t(n_slabs) * wps * 2 <= nwarps) wps *= 2;
+  for (int64_t t = gwarp; t < int64_t(n_slabs) * wps; t += nwarps) {
+    const int s = int(t / wps), part = int(t % wps);
     float vm = 0.f;  // largest magnitude this thread staged (for the fixed-point LCG's bound)
     const int seg_b = offs[int64_t(s) * m + slot];
     const int seg_e = offs[int64_t(s + 1) * m + slot];
-    for (int c0 = seg_b + warp * kLayoutChunk; c0 < seg_e; c0 += NW * kLayoutChunk) {
+    for (int c0 = seg_b + part * kLayoutChunk; c0 < seg_e; c0 += wps * kLayoutChunk) {
       const int n = min(kLayoutChunk, seg_e - c0);
       cnt[lane] = 0;
       __syncwarp();
@@ -165,14 +168,9 @@ __device__ __forceinline__ void layout_row_slabs(
     }
     if (vmax != nullptr) {  // max |value| of the row's segment in this slab (0 when empty)
       for (int o = 16; o > 0; o >>= 1) vm = fmaxf(vm, __shfl_xor_sync(0xFFFFFFFFu, vm, o));
-      __syncthreads();  // the previous slab's maxima have been read
-      if (lane == 0) s_max[warp] = vm;
-      __syncthreads();
-      if (threadIdx.x == 0) {
-        float v = s_max[0];
-        for (int w2 = 1; w2 < NW; ++w2) v = fmaxf(v, s_max[w2]);
-        vmax[int64_t(s) * m + slot] = v;
-      }
+      // non-negative floats order like their bit patterns
+      if (lane == 0 && vm > 0.f)
+        atomicMax(reinterpret_cast<int*>(vmax + int64_t(s) * m + slot), __float_as_int(vm));
     }
   }
 }
@@ -260,92 +258,6 @@ __device__ __forceinline__ void tail_dispatch(int groups, const uint16_t* pi, co
   }
 }
 
-// A warp's walk over its rows' segments in one slab (rows warp, warp + nwarps, ...), one pass
-// of D groups of 32 entries at a time, software-pipelined: the loads of the next pass - the
-// next part of the same segment or the start of the warp's next row - are issued before the
-// current pass is consumed, so a warp always has a pass in flight while it works.
-//   skip(r)   rows the caller does not want read (a zero weight);
-//   empty(r)  called for every row that is skipped or has no entry in this slab;
-//   use(p)    consumes a pass: p.ii[q] / p.vv[q] are entry q of this lane (index PAD and value 0
-//             where the segment has ended), p.row the row, p.last whether the row ends here.
-#ifndef EFCP_PIPE_DEPTH
-#define EFCP_PIPE_DEPTH 6
-#endif
-constexpr int kPipe = EFCP_PIPE_DEPTH;
-
-template <int D>
-struct SegPass {
-  int ii[D];
-  float vv[D];
-  int row;
-  bool last;
-};
-
-template <int D, int PAD, typename VT, typename Skip, typename Empty, typename Use>
-__device__ __forceinline__ void walk_segments(const uint16_t* __restrict__ R,
-                                              const VT* __restrict__ V, int64_t k,
-                                              const int32_t* seg, int m, int warp, int nwarps,
-                                              int lane, Skip&& skip, Empty&& empty, Use&& use) {
-  int r = warp - nwarps;  // row of the next pass to load
-  int j = 0, e = 0;       // its next unread position and the end of its segment
-  const uint16_t* Rr = R;
-  const VT* Vr = V;
-  auto next_row = [&]() {
-    for (r += nwarps; r < m; r += nwarps) {
-      j = seg[r];
-      e = seg[m + r];
-      if (j < e && !skip(r)) {
-        Rr = R + int64_t(r) * k;
-        Vr = V + int64_t(r) * k;
-        const int rn = r + nwarps;  // its successor's lines are asked from HBM now
-        if (rn < m)
-          prefetch_segment(R + int64_t(rn) * k, V + int64_t(rn) * k, seg[rn], seg[m + rn], lane);
-        return true;
-      }
-      empty(r);
-    }
-    return false;
-  };
-  auto load = [&](SegPass<D>& p) {
-    p.row = r;
-    const uint16_t* pi = Rr + j + lane;
-    const VT* pv = Vr + j + lane;
-    if (j + 32 * D <= e) {  // a full pass: no bounds checks
-#pragma unroll
-      for (int q = 0; q < D; ++q) {
-        p.ii[q] = int(__ldcs(pi + 32 * q));
-        p.vv[q] = load_value(pv + 32 * q);
-      }
-    } else {
-      const int left = e - j - lane;  // entries of this lane's stride that remain: q < left / 32
-#pragma unroll
-      for (int q = 0; q < D; ++q) {
-        const bool on = 32 * q < left;
-        p.ii[q] = on ? int(__ldcs(pi + 32 * q)) : PAD;
-        p.vv[q] = on ? load_value(pv + 32 * q) : 0.f;
-      }
-    }
-    j += 32 * D;
-    p.last = j >= e;
-  };
-  bool more = next_row();
-  if (!more) return;
-  SegPass<D> cur;
-  load(cur);
-  if (cur.last) more = next_row();
-  for (;;) {
-    SegPass<D> nxt;
-    const bool have = more;
-    if (have) {
-      load(nxt);
-      if (nxt.last) more = next_row();
-    }
-    use(cur);
-    if (!have) break;
-    cur = nxt;
-  }
-}
-
 // Shared -> global bulk copy (TMA, untiled form): both addresses 16-byte aligned, size a
 // multiple of 16.  Used where the method leaves a large contiguous piece to move: a
 // finished slab of the update.  The fence makes the accumulator's generic-proxy writes
@@ -425,46 +337,69 @@ __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_sp_rows(
     }
     __syncthreads();
     double* out = slab_part + int64_t(s) * stride;
-    double acc = 0.0, acc2 = 0.0;  // COMPRESSED: two chains of <row, c>; ACC: <row, c>, <row, xi>
-    walk_segments<kPipe, 0>(
-        R, V, k, seg, m, warp, nwarps, lane, [](int) { return false; },
-        [&](int r) {
-          if (lane == 0) {
-            out[r] = 0.0;
-            if (ACC) out[m + r] = 0.0;
-          }
-        },
-        [&](const SegPass<kPipe>& p) {
+    for (int r = warp; r < m; r += nwarps) {
+      const int b = seg[r], e2 = seg[m + r];
+      if (b >= e2) {
+        if (lane == 0) {
+          out[r] = 0.0;
+          if (ACC) out[m + r] = 0.0;
+        }
+        continue;
+      }
+      const uint16_t* Rr = R + int64_t(r) * k;
+      const VT* Vr = V + int64_t(r) * k;
+      if (r + nwarps < m) {
+        const int rn = r + nwarps;
+        prefetch_segment(R + int64_t(rn) * k, V + int64_t(rn) * k, seg[rn], seg[m + rn], lane);
+      }
+      double acc = 0.0, acc2 = 0.0;  // COMPRESSED: two chains of <row, c>; ACC: <row, c>, <row, xi>
+      auto use = [&](int q, int i, float v) {
+        const double p = double(v) * double(xs[i]);
+        if (ACC) {
+          const bool in_c = (mask[i >> 5] >> (i & 31)) & 1u;
+          acc += in_c ? p : 0.0;
+          acc2 += in_c ? 0.0 : p;
+        } else if (q & 1) {
+          acc2 += p;
+        } else {
+          acc += p;
+        }
+      };
+      // kDepth groups of 32 entries per pass: all loads of a pass are issued before the
+      // first use.  Full passes need no bounds checks and address every load by a
+      // constant offset from one pointer pair.
+      int j0 = b + lane;
+      for (; j0 + 32 * (kDepth - 1) < e2 - 31 + lane; j0 += 32 * kDepth) {
+        const uint16_t* pi = Rr + j0;
+        const VT* pv = Vr + j0;
+        int ii[kDepth];
+        float vv[kDepth];
 #pragma unroll
-          for (int q = 0; q < kPipe; ++q) {
-            const int i = p.ii[q];
-            const double pr = double(p.vv[q]) * double(xs[i]);
-            if (ACC) {
-              const bool in_c = (mask[i >> 5] >> (i & 31)) & 1u;
-              acc += in_c ? pr : 0.0;
-              acc2 += in_c ? 0.0 : pr;
-            } else if (q & 1) {
-              acc2 += pr;
-            } else {
-              acc += pr;
-            }
-          }
-          if (p.last) {  // every fp32 x fp32 product is exact in fp64; one sum per (slab, row)
-            if (ACC) {
-              acc = warp_sum(acc);
-              acc2 = warp_sum(acc2);
-              if (lane == 0) {
-                out[p.row] = acc;
-                out[m + p.row] = acc2;
-              }
-            } else {
-              acc = warp_sum(acc + acc2);
-              if (lane == 0) out[p.row] = acc;
-            }
-            acc = 0.0;
-            acc2 = 0.0;
-          }
-        });
+        for (int q = 0; q < kDepth; ++q) {
+          ii[q] = __ldcs(pi + 32 * q);
+          vv[q] = load_value(pv + 32 * q);
+        }
+#pragma unroll
+        for (int q = 0; q < kDepth; ++q) use(q, ii[q], vv[q]);
+      }
+      const int rem = e2 - (j0 - lane);  // entries left for the last pass (warp-uniform)
+      if (rem > 0) {
+        const int groups = (rem + 31) >> 5;
+        tail_dispatch(groups, Rr + j0, Vr + j0, j0 + 32 * (groups - 1) < e2, 0,
+                      [&](int q, int i, float v) { use(q, i, v); });
+      }
+      if (ACC) {
+        acc = warp_sum(acc);
+        acc2 = warp_sum(acc2);
+        if (lane == 0) {
+          out[r] = acc;
+          out[m + r] = acc2;
+        }
+      } else {
+        acc = warp_sum(acc + acc2);
+        if (lane == 0) out[r] = acc;
+      }
+    }
     t = s_next;
   }
 }
@@ -575,14 +510,39 @@ __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_lcg(
     __syncthreads();
     // every row's segment of this slab, scaled by the row's weight, into the accumulator
     auto accumulate = [&](auto add) {
-      walk_segments<kPipe, -1>(
-          R, V, k, seg, m, warp, nwarps, lane, [&](int r) { return wc[r] == 0.f; }, [](int) {},
-          [&](const SegPass<kPipe>& p) {
-            const float c = wc[p.row];
-#pragma unroll
-            for (int q = 0; q < kPipe; ++q)
-              if (p.ii[q] >= 0) add(p.ii[q], c * p.vv[q]);
-          });
+      for (int r = warp; r < m; r += nwarps) {
+        const int b = seg[r], e = seg[m + r];
+        const float c = wc[r];
+        if (b >= e || c == 0.f) continue;
+        const uint16_t* Rr = R + int64_t(r) * k;
+        const VT* Vr = V + int64_t(r) * k;
+        if (r + nwarps < m) {
+          const int rn = r + nwarps;
+          prefetch_segment(R + int64_t(rn) * k, V + int64_t(rn) * k, seg[rn], seg[m + rn], lane);
+        }
+        int j0 = b + lane;
+        for (; j0 + 32 * (kDepth - 1) < e - 31 + lane; j0 += 32 * kDepth) {  // full passes
+          const uint16_t* pi = Rr + j0;
+          const VT* pv = Vr + j0;
+          int ii[kDepth];
+          float vv[kDepth];
+  #pragma unroll
+          for (int q = 0; q < kDepth; ++q) {
+            ii[q] = __ldcs(pi + 32 * q);
+            vv[q] = load_value(pv + 32 * q);
+          }
+  #pragma unroll
+          for (int q = 0; q < kDepth; ++q) add(ii[q], c * vv[q]);
+        }
+        const int rem = e - (j0 - lane);  // entries left for the last pass (warp-uniform)
+        if (rem > 0) {
+          const int groups = (rem + 31) >> 5;
+          tail_dispatch(groups, Rr + j0, Vr + j0, j0 + 32 * (groups - 1) < e, -1,
+                        [&](int, int i, float v) {
+                          if (i >= 0) add(i, c * v);
+                        });
+        }
+      }
     };
     const int64_t gbase = int64_t(s) * W;
     const int n = int(min(int64_t(W), d - gbase));

@@ -1,5 +1,7 @@
 """GPU tests of the boundary itself: caller-supplied memory, the debug-checks flag, the
 bounded device-side wait (failure detection without a GPU fault), device selection."""
+import gc
+
 import numpy as np
 import pytest
 import torch
@@ -60,6 +62,7 @@ def test_handle_in_caller_memory_allocates_nothing(flags, block):
     warm.step(g_dev.zero_(), u_dev)
     assert warm.validate() == 0 and warm.status() == 0
     warm.close()
+    gc.collect()  # handles earlier tests left to the collector free their memory now, not later
     torch.cuda.synchronize()
     free0, _ = torch.cuda.mem_get_info()
     gpu = B.Efcp(d, m, k, lam, flags, block, workspace=ws)
@@ -69,14 +72,14 @@ def test_handle_in_caller_memory_allocates_nothing(flags, block):
         gpu.step(g_dev, u_dev)
         u_ref = cpu.step(g)
         free_t, _ = torch.cuda.mem_get_info()
-        assert free_t == free0, f"free device memory moved at step {t}"
+        assert free_t >= free0, f"device memory was allocated at step {t}"
         assert np.array_equal(bits(gpu.error()), bits(cpu.error()))
         assert rel_l2(u_dev.cpu().numpy(), u_ref) <= 1e-4
     assert gpu.validate() == 0 and gpu.status() == 0
     gpu.close()
     torch.cuda.synchronize()
     free1, _ = torch.cuda.mem_get_info()
-    assert free1 == free0
+    assert free1 >= free0
     # one byte short: refused, nothing leaks
     with pytest.raises(B.EfcpError) as ei:
         B.Efcp(d, m, k, lam, flags, block, workspace=ws[:need - 256])
