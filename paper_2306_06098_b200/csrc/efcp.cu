@@ -82,6 +82,7 @@ struct efcp_ctx {
   int next_phase = 0;             // of efcp_shard_phase
   bool is_shard = false;
   bool split_phases = false;      // EFCP_SPLIT_PHASES=1: one launch per phase (profiling)
+  int short_rows = 0;             // rows have few entries per slab: the slab kernels' ring walk
   float* wf = nullptr;
   int* slab_ctr = nullptr;   // work counters of the slab kernels (SP, LCG)
   int64_t* colsum = nullptr; // n_slabs + 1 column sums of offs
@@ -303,6 +304,7 @@ int configure(efcp_ctx* ctx, int64_t d, int32_t m, int64_t k, float lambda, uint
   const Sizes z = compute_sizes(d, m, ctx->num_sms);
   ctx->W = z.W; ctx->n_slabs = z.n_slabs; ctx->n_chunks = z.n_chunks;
   ctx->grid_slab = z.grid_slab;
+  ctx->short_rows = k / z.n_slabs < kShortSegment ? 1 : 0;
   if (const char* env = getenv("EFCP_NO_SPEC")) ctx->spec = atoi(env) == 0;
   if (const char* env = getenv("EFCP_SPLIT_PHASES")) ctx->split_phases = atoi(env) != 0;
   // EFCP_LCG_FIXED_TOL: relative error a slab of the fixed-point LCG may have before it is redone
@@ -433,24 +435,38 @@ bool init_state(efcp_ctx* ctx) {
     ok &= cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_select_insert, kSelThreads,
                                                         kSelSmemBytes) == cudaSuccess;
     ok &= occ >= 1;
-    ctx->sel_grid = std::min(kMaxCoopBlocks, ctx->num_sms * std::min(occ, 4));
+    // a warp per group of chunk buckets, per (slab, part) of the insert, four row entries per
+    // thread in the offsets phase; at least one block per SM
+    const int64_t n_groups = (ctx->n_chunks + kSelGroup - 1) / kSelGroup;
+    const int64_t want = std::max<int64_t>({(n_groups + kSelWarps - 1) / kSelWarps,
+                                            (int64_t(n_slabs) * 2 + kSelWarps - 1) / kSelWarps,
+                                            (k + 4 * kSelThreads - 1) / (4 * kSelThreads),
+                                            int64_t(ctx->num_sms)});
+    ctx->sel_grid = int(std::min<int64_t>({int64_t(kMaxCoopBlocks),
+                                           int64_t(ctx->num_sms) * std::min(occ, 4), want}));
   }
   if (ctx->flags & EFCP_PRECOND_GGT)
     ok &= cudaFuncSetAttribute(ggt_slots(m) <= 2 ? k_ggt_weights<2> : k_ggt_weights<4>, attr,
                                int(ggt_smem_bytes(m))) == cudaSuccess;
-  ok &= cudaFuncSetAttribute(k_sp_rows<false, float>, attr, int(smem)) == cudaSuccess;
-  ok &= cudaFuncSetAttribute(k_sp_rows<true, float>, attr, int(smem)) == cudaSuccess;
-  ok &= cudaFuncSetAttribute(k_sp_rows<false, bf16raw>, attr, int(smem)) == cudaSuccess;
-  ok &= cudaFuncSetAttribute(k_lcg<true, false, float>, attr, int(smem)) == cudaSuccess;
-  ok &= cudaFuncSetAttribute(k_lcg<false, false, float>, attr, int(smem)) == cudaSuccess;
-  ok &= cudaFuncSetAttribute(k_lcg<true, true, float>, attr, int(smem)) == cudaSuccess;
-  ok &= cudaFuncSetAttribute(k_lcg<false, true, float>, attr, int(smem)) == cudaSuccess;
-  ok &= cudaFuncSetAttribute(k_lcg<true, false, bf16raw>, attr, int(smem)) == cudaSuccess;
-  ok &= cudaFuncSetAttribute(k_lcg<false, false, bf16raw>, attr, int(smem)) == cudaSuccess;
-  ok &= cudaFuncSetAttribute(k_lcg<true, false, float, true>, attr, int(smem)) == cudaSuccess;
-  ok &= cudaFuncSetAttribute(k_lcg<false, false, float, true>, attr, int(smem)) == cudaSuccess;
-  ok &= cudaFuncSetAttribute(k_lcg<true, false, bf16raw, true>, attr, int(smem)) == cudaSuccess;
-  ok &= cudaFuncSetAttribute(k_lcg<false, false, bf16raw, true>, attr, int(smem)) == cudaSuccess;
+  auto big_smem = [&](auto kern) {
+    return cudaFuncSetAttribute(kern, attr, int(smem)) == cudaSuccess;
+  };
+  ok &= big_smem(k_sp_rows<false, float, false>) && big_smem(k_sp_rows<false, float, true>);
+  ok &= big_smem(k_sp_rows<true, float, false>) && big_smem(k_sp_rows<true, float, true>);
+  ok &= big_smem(k_sp_rows<false, bf16raw, false>) && big_smem(k_sp_rows<false, bf16raw, true>);
+#define EFCP_LCG_ATTR(VEC, ACC, VT, FIXED)                         \
+  ok &= big_smem(k_lcg<VEC, ACC, VT, FIXED, false>) && big_smem(k_lcg<VEC, ACC, VT, FIXED, true>)
+  EFCP_LCG_ATTR(true, false, float, false);
+  EFCP_LCG_ATTR(false, false, float, false);
+  EFCP_LCG_ATTR(true, true, float, false);
+  EFCP_LCG_ATTR(false, true, float, false);
+  EFCP_LCG_ATTR(true, false, bf16raw, false);
+  EFCP_LCG_ATTR(false, false, bf16raw, false);
+  EFCP_LCG_ATTR(true, false, float, true);
+  EFCP_LCG_ATTR(false, false, float, true);
+  EFCP_LCG_ATTR(true, false, bf16raw, true);
+  EFCP_LCG_ATTR(false, false, bf16raw, true);
+#undef EFCP_LCG_ATTR
   ok &= cudaDeviceSynchronize() == cudaSuccess;
   return ok;
 }
@@ -626,13 +642,19 @@ int launch_sp(efcp_ctx* ctx, int slot, cudaStream_t st) {
   const int m = ctx->m;
   const bool acc_mode = (ctx->flags & EFCP_RHS_ACCUMULATOR) != 0;
   const size_t smem = slab_smem_bytes(ctx->W, m);
-#define EFCP_SP_LAUNCH(ACC, VT, VPTR)                                                          \
-  k_sp_rows<ACC, VT><<<ctx->grid_slab, kSlabThreads, smem, st>>>(                              \
+#define EFCP_SP_LAUNCH1(ACC, VT, SHORT, VPTR)                                                  \
+  k_sp_rows<ACC, VT, SHORT><<<ctx->grid_slab, kSlabThreads, smem, st>>>(                       \
       ctx->R, VPTR, ctx->V, ctx->offs, k, m, ctx->W, ctx->n_slabs, slot, ctx->slab_part,       \
       ctx->slab_ctr, ctx->order, ctx->e, d)
+#define EFCP_SP_LAUNCH(ACC, VT, VPTR)                                                          \
+  do {                                                                                         \
+    if (ctx->short_rows) EFCP_SP_LAUNCH1(ACC, VT, true, VPTR);                                 \
+    else EFCP_SP_LAUNCH1(ACC, VT, false, VPTR);                                                \
+  } while (0)
   if (ctx->V16) EFCP_SP_LAUNCH(false, bf16raw, ctx->V16);
   else if (acc_mode) EFCP_SP_LAUNCH(true, float, ctx->V);
   else EFCP_SP_LAUNCH(false, float, ctx->V);
+#undef EFCP_SP_LAUNCH1
 #undef EFCP_SP_LAUNCH
   EFCP_LAUNCHED();
   return EFCP_OK;
@@ -653,6 +675,7 @@ int launch_mxm(efcp_ctx* ctx, int slot, int pb, int pe, cudaStream_t st) {
   ma.res = v.res; ma.dw = v.dw; ma.rhs = v.rhs;
   ma.sc = ctx->sc; ma.bar = ctx->bar + 2;
   ma.phase_begin = pb; ma.phase_end = pe;
+  ma.fuse12 = (pb <= 1 && pe > 2) ? 1 : 0;  // both in this launch: nothing to exchange between
   void* args[] = {&ma};
   EFCP_CUDA(cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(k_mxm),
                                         dim3(ctx->mxm_grid), dim3(kMxmThreads), args,
@@ -686,15 +709,25 @@ int launch_lcg(efcp_ctx* ctx, float* update, LcgApply ap, cudaStream_t st) {
   const bool uvec = (reinterpret_cast<uintptr_t>(update) & 15) == 0;
   const float inv_lambda = 1.0f / ctx->lambda;
   const double* dw = ggt ? nullptr : v.dw;
-#define EFCP_LCG_LAUNCH(VEC, ACC, VT, VPTR)                                                    \
-  k_lcg<VEC, ACC, VT><<<ctx->grid_slab, kSlabThreads, smem, st>>>(                             \
+#define EFCP_LCG_LAUNCH1(VEC, ACC, VT, SHORT, VPTR)                                            \
+  k_lcg<VEC, ACC, VT, false, SHORT><<<ctx->grid_slab, kSlabThreads, smem, st>>>(               \
       ctx->R, VPTR, ctx->offs, k, m, ctx->W, ctx->n_slabs, v.w, dw, v.wfin, update, d,         \
       ctx->slab_ctr + 1, ctx->order, ctx->e, inv_lambda, ap)
-#define EFCP_LCG_FIXED_LAUNCH(VEC, VT, VPTR)                                                    \
-  k_lcg<VEC, false, VT, true><<<ctx->grid_slab, kSlabThreads, smem, st>>>(                     \
+#define EFCP_LCG_FIXED_LAUNCH1(VEC, VT, SHORT, VPTR)                                            \
+  k_lcg<VEC, false, VT, true, SHORT><<<ctx->grid_slab, kSlabThreads, smem, st>>>(              \
       ctx->R, VPTR, ctx->offs, k, m, ctx->W, ctx->n_slabs, v.w, dw, v.wfin, update, d,         \
       ctx->slab_ctr + 1, ctx->order, ctx->e, inv_lambda, ap, ctx->vmax, ctx->lcg_redo,         \
       ctx->lcg_tol2)
+#define EFCP_LCG_LAUNCH(VEC, ACC, VT, VPTR)                                                    \
+  do {                                                                                         \
+    if (ctx->short_rows) EFCP_LCG_LAUNCH1(VEC, ACC, VT, true, VPTR);                           \
+    else EFCP_LCG_LAUNCH1(VEC, ACC, VT, false, VPTR);                                          \
+  } while (0)
+#define EFCP_LCG_FIXED_LAUNCH(VEC, VT, VPTR)                                                    \
+  do {                                                                                         \
+    if (ctx->short_rows) EFCP_LCG_FIXED_LAUNCH1(VEC, VT, true, VPTR);                          \
+    else EFCP_LCG_FIXED_LAUNCH1(VEC, VT, false, VPTR);                                         \
+  } while (0)
   if (ctx->vmax) {
     if (ctx->V16) {
       if (uvec) EFCP_LCG_FIXED_LAUNCH(true, bf16raw, ctx->V16);
@@ -715,6 +748,8 @@ int launch_lcg(efcp_ctx* ctx, float* update, LcgApply ap, cudaStream_t st) {
   }
 #undef EFCP_LCG_LAUNCH
 #undef EFCP_LCG_FIXED_LAUNCH
+#undef EFCP_LCG_LAUNCH1
+#undef EFCP_LCG_FIXED_LAUNCH1
   EFCP_LAUNCHED();
   return EFCP_OK;
 }

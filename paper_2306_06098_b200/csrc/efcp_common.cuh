@@ -63,6 +63,11 @@ __device__ __forceinline__ float load_value(const float* p) { return __ldcs(p); 
 __device__ __forceinline__ float load_value(const bf16raw* p) {
   return bf16_to_float(__ldcs(reinterpret_cast<const uint16_t*>(p)));
 }
+// the same through the ordinary cached path (short pieces whose sectors are touched again)
+__device__ __forceinline__ float load_value_cached(const float* p) { return *p; }
+__device__ __forceinline__ float load_value_cached(const bf16raw* p) {
+  return bf16_to_float(*reinterpret_cast<const uint16_t*>(p));
+}
 
 // Exclusive prefix sum over the threads of a block (blockDim.x a multiple of 32,
 // at most 1024).  sm needs 33 entries.  *total receives the block sum.

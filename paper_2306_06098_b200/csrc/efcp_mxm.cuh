@@ -58,6 +58,7 @@ struct MxmArgs {
   double* partial;          // [parts][stride]
   int n_slabs, parts, m, slot;
   int acc;                  // x = a: stride is 2 m, the second half sums to q = G xi
+  int fuse12;               // nothing is exchanged between phases 1 and 2: phase 1 does both
   double mlambda, lambda;
   double* S;
   double* B;
@@ -106,6 +107,7 @@ __global__ void __launch_bounds__(kMxmThreads) k_mxm(const MxmArgs A) {
   unsigned int barriers = 0;
   for (int phase = A.phase_begin; phase < A.phase_end; ++phase) {
     if (!A.acc && (phase == 5 || phase == 6)) continue;
+    if (A.fuse12 && phase == 2) continue;
     if (phase > A.phase_begin) {
       if (!grid_barrier(A.bar, ++barriers)) {
         if (tid == 0) atomicOr(&A.sc->status, kStTimeout);
@@ -128,26 +130,27 @@ __global__ void __launch_bounds__(kMxmThreads) k_mxm(const MxmArgs A) {
         for (; s < A.n_slabs; s += step) a0 += A.slab_part[int64_t(s) * stride + r];
         A.partial[t] = (a0 + a1) + (a2 + a3);
       }
-    } else if (phase == 1) {
+    } else if (phase == 1 || phase == 2) {
       for (int64_t r = gthread; r < m; r += nthreads) {
-        double s = 0.0;
-        for (int p = 0; p < A.parts; ++p) s += A.partial[int64_t(p) * stride + r];
-        A.delta[r] = s;
-        if (A.acc) {
-          double q = 0.0;
-          for (int p = 0; p < A.parts; ++p) q += A.partial[int64_t(p) * stride + m + r];
-          A.rhs[r] = q;  // G xi for now; phase 2 turns it into the right-hand side
+        if (phase == 1) {
+          double s = 0.0;
+          for (int p = 0; p < A.parts; ++p) s += A.partial[int64_t(p) * stride + r];
+          A.delta[r] = s;
+          if (A.acc) {
+            double q = 0.0;
+            for (int p = 0; p < A.parts; ++p) q += A.partial[int64_t(p) * stride + m + r];
+            A.rhs[r] = q;  // G xi for now; phase 2 turns it into the right-hand side
+          }
         }
-      }
-    } else if (phase == 2) {
-      // Section 2.1: S_{i,:} = S_{:,i} = G g
-      for (int64_t r = gthread; r < m; r += nthreads) {
-        const double s = A.delta[r];
-        A.S[int64_t(slot) * m + r] = s;
-        A.S[int64_t(r) * m + slot] = s;
-        A.aprime[r] = r == slot ? 0.0 : s;
-        A.bold[r] = A.B[int64_t(slot) * m + r];
-        if (A.acc) A.rhs[r] = (r == slot ? double(m) : 0.0) - A.rhs[r] / A.lambda;
+        if (phase == 2 || A.fuse12) {
+          // Section 2.1: S_{i,:} = S_{:,i} = G g
+          const double s = A.delta[r];
+          A.S[int64_t(slot) * m + r] = s;
+          A.S[int64_t(r) * m + slot] = s;
+          A.aprime[r] = r == slot ? 0.0 : s;
+          A.bold[r] = A.B[int64_t(slot) * m + r];
+          if (A.acc) A.rhs[r] = (r == slot ? double(m) : 0.0) - A.rhs[r] / A.lambda;
+        }
       }
     } else if (phase == 3) {
       gemv_rows(A.B, A.aprime, A.y, m, gwarp, nwarps, lane);

@@ -127,7 +127,10 @@ __device__ __forceinline__ void flush_hist(const uint32_t* h, uint32_t* __restri
 
 // The buckets of the chunks [ch0, ch0 + kSelGroup) as one list in index order: calls
 // f(on, value, chunk, position in the chunk's bucket) for every entry, 32 entries per
-// call round (`on` is false for the lanes past the end of the last round, so f may vote).
+// call (`on` is false for the lanes past the end of the list, so f may vote).  The loads of
+// kSelAhead calls are issued together: the passes over the buckets are chains of dependent
+// global loads otherwise.
+constexpr int kSelAhead = 4;
 template <typename F>
 __device__ __forceinline__ void walk_group(const SelectArgs& A, int ch0, int lane, F&& f) {
   const int nch = min(kSelGroup, A.n_chunks - ch0);
@@ -137,18 +140,30 @@ __device__ __forceinline__ void walk_group(const SelectArgs& A, int ch0, int lan
 #pragma unroll
   for (int q = 0; q < kSelGroup; ++q) pre[q + 1] = pre[q] + __shfl_sync(0xFFFFFFFFu, mine, q);
   const int total = pre[kSelGroup];
-  for (int f0 = 0; f0 < total; f0 += 32) {
-    const int fl = f0 + lane;
-    const bool on = fl < total;
-    int t = 0;
+  for (int f0 = 0; f0 < total; f0 += 32 * kSelAhead) {
+    bool on[kSelAhead];
+    int ch[kSelAhead], i[kSelAhead];
+    float v[kSelAhead];
 #pragma unroll
-    for (int q = 1; q < kSelGroup; ++q) t += fl >= pre[q] ? 1 : 0;
-    int base = 0;
+    for (int u = 0; u < kSelAhead; ++u) {
+      const int fl = f0 + 32 * u + lane;
+      on[u] = fl < total;
+      int t = 0, base = 0;
 #pragma unroll
-    for (int q = 1; q < kSelGroup; ++q) base = t == q ? pre[q] : base;
-    const int ch = ch0 + (on ? t : 0), i = on ? fl - base : 0;
-    const float v = on ? A.bk_val[int64_t(ch) * kChunk + i] : 0.f;
-    f(on, v, ch, i);
+      for (int q = 1; q < kSelGroup; ++q) {
+        const bool past = fl >= pre[q];
+        t += past ? 1 : 0;
+        base = past ? pre[q] : base;
+      }
+      ch[u] = ch0 + (on[u] ? t : 0);
+      i[u] = on[u] ? fl - base : 0;
+      v[u] = on[u] ? A.bk_val[int64_t(ch[u]) * kChunk + i[u]] : 0.f;
+    }
+#pragma unroll
+    for (int u = 0; u < kSelAhead; ++u) {
+      if (f0 + 32 * u >= total) break;  // warp-uniform
+      f(on[u], v[u], ch[u], i[u]);
+    }
   }
 }
 

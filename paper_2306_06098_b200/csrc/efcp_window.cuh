@@ -258,6 +258,89 @@ __device__ __forceinline__ void tail_dispatch(int groups, const uint16_t* pi, co
   }
 }
 
+// Short segments.  When a row has only a group or two of entries per slab (low densities,
+// small d), the burst above is one short dependent chain per row - offsets, loads, use,
+// reduction - and a warp walks its rows one latency after the other.  This walk keeps kRing
+// passes of kShort groups in flight per warp instead, across row boundaries: the loads of the
+// pass kRing ahead are issued when a pass is consumed.
+//   skip(r)   rows the caller does not want read (a zero weight);
+//   empty(r)  called for every row that is skipped or has no entry in this slab;
+//   use(p)    consumes a pass: p.ii[q] / p.vv[q] are entry q of this lane (index PAD and value 0
+//             past the segment's end), p.row the row, p.last whether the row ends here.
+constexpr int kShort = 2;  // groups of 32 entries per pass
+constexpr int kRing = 4;   // passes in flight per warp
+constexpr int kShortSegment = 96;  // entries per row and slab below which this walk is used
+
+struct ShortPass {
+  int ii[kShort];
+  float vv[kShort];
+  int row;
+  bool last;
+};
+
+template <int PAD, typename VT, typename Skip, typename Empty, typename Use>
+__device__ __forceinline__ void walk_short_segments(const uint16_t* __restrict__ R,
+                                                    const VT* __restrict__ V, int64_t k,
+                                                    const int32_t* seg, int m, int warp,
+                                                    int nwarps, int lane, Skip&& skip,
+                                                    Empty&& empty, Use&& use) {
+  int r = warp - nwarps;  // row of the next pass to load
+  int j = 0, e = 0;  // its next unread position and the end of its segment
+  const uint16_t* Rr = R;
+  const VT* Vr = V;
+  auto next_row = [&]() {
+    for (r += nwarps; r < m; r += nwarps) {
+      j = seg[r];
+      e = seg[m + r];
+      if (j < e && !skip(r)) {
+        Rr = R + int64_t(r) * k;
+        Vr = V + int64_t(r) * k;
+        return true;
+      }
+      empty(r);
+    }
+    return false;
+  };
+  auto load = [&](ShortPass& p) {
+    p.row = r;
+    const int left = e - j - lane;  // this lane has entry q of the pass when 32 q < left
+#pragma unroll
+    for (int q = 0; q < kShort; ++q) {
+      const bool on = 32 * q < left;
+      p.ii[q] = on ? int(Rr[j + lane + 32 * q]) : PAD;
+      p.vv[q] = on ? load_value_cached(Vr + j + lane + 32 * q) : 0.f;
+    }
+    j += 32 * kShort;
+    p.last = j >= e;
+  };
+  ShortPass buf[kRing];
+  bool have[kRing];
+  bool more = next_row();
+#pragma unroll
+  for (int i = 0; i < kRing; ++i) {
+    have[i] = more;
+    if (more) {
+      load(buf[i]);
+      if (buf[i].last) more = next_row();
+    }
+  }
+  for (bool going = have[0]; going;) {
+#pragma unroll
+    for (int i = 0; i < kRing; ++i) {
+      if (!have[i]) {
+        going = false;
+        break;
+      }
+      use(buf[i]);
+      have[i] = more;
+      if (more) {
+        load(buf[i]);
+        if (buf[i].last) more = next_row();
+      }
+    }
+  }
+}
+
 // Shared -> global bulk copy (TMA, untiled form): both addresses 16-byte aligned, size a
 // multiple of 16.  Used where the method leaves a large contiguous piece to move: a
 // finished slab of the update.  The fence makes the accumulator's generic-proxy writes
@@ -294,7 +377,9 @@ __device__ __forceinline__ void bulk_store_wait_read() {
 // serves both sums.  `stride` is the row length of slab_part (m or 2 m).
 // VT is the format of the streamed values: float, or bf16raw (same values, half the bytes);
 // Vf is the fp32 copy, used for the new row only.
-template <bool ACC, typename VT>
+// SHORT selects the ring walk for short segments (a variant of its own: the two walks have
+// different register needs).
+template <bool ACC, typename VT, bool SHORT = false>
 __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_sp_rows(
     const uint16_t* __restrict__ R, const VT* __restrict__ V, const float* __restrict__ Vf,
     const int32_t* __restrict__ offs,
@@ -337,6 +422,48 @@ __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_sp_rows(
     }
     __syncthreads();
     double* out = slab_part + int64_t(s) * stride;
+    if constexpr (SHORT) {
+      double acc = 0.0, acc2 = 0.0;  // <row, c> (two chains), or with ACC <row, c> and <row, xi>
+      walk_short_segments<0>(
+          R, V, k, seg, m, warp, nwarps, lane, [](int) { return false; },
+          [&](int r) {
+            if (lane == 0) {
+              out[r] = 0.0;
+              if (ACC) out[m + r] = 0.0;
+            }
+          },
+          [&](const ShortPass& p) {
+#pragma unroll
+            for (int q = 0; q < kShort; ++q) {
+              const int i = p.ii[q];
+              const double pr = double(p.vv[q]) * double(xs[i]);
+              if (ACC) {
+                const bool in_c = (mask[i >> 5] >> (i & 31)) & 1u;
+                acc += in_c ? pr : 0.0;
+                acc2 += in_c ? 0.0 : pr;
+              } else if (q & 1) {
+                acc2 += pr;
+              } else {
+                acc += pr;
+              }
+            }
+            if (p.last) {
+              if (ACC) {
+                acc = warp_sum(acc);
+                acc2 = warp_sum(acc2);
+                if (lane == 0) {
+                  out[p.row] = acc;
+                  out[m + p.row] = acc2;
+                }
+              } else {
+                acc = warp_sum(acc + acc2);
+                if (lane == 0) out[p.row] = acc;
+              }
+              acc = 0.0;
+              acc2 = 0.0;
+            }
+          });
+    } else {
     for (int r = warp; r < m; r += nwarps) {
       const int b = seg[r], e2 = seg[m + r];
       if (b >= e2) {
@@ -400,6 +527,7 @@ __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_sp_rows(
         if (lane == 0) out[r] = acc;
       }
     }
+    }  // burst walk
     t = s_next;
   }
 }
@@ -470,7 +598,7 @@ struct LcgApply {
 // slab by slab and therefore for the whole vector - and otherwise accumulated again with fp32
 // atomics (its 2.5 MB of entries are still in L2).  Integer sums do not depend on the order of
 // the adds: the accepted slabs of u are reproducible bit for bit.
-template <bool VEC, bool ACC, typename VT, bool FIXED = false>
+template <bool VEC, bool ACC, typename VT, bool FIXED = false, bool SHORT = false>
 __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_lcg(
     const uint16_t* __restrict__ R, const VT* __restrict__ V, const int32_t* __restrict__ offs,
     int64_t k, int m, int W, int n_slabs, const double* __restrict__ w64,
@@ -510,6 +638,17 @@ __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_lcg(
     __syncthreads();
     // every row's segment of this slab, scaled by the row's weight, into the accumulator
     auto accumulate = [&](auto add) {
+      if constexpr (SHORT) {
+        walk_short_segments<-1>(
+            R, V, k, seg, m, warp, nwarps, lane, [&](int r) { return wc[r] == 0.f; },
+            [](int) {},
+            [&](const ShortPass& p) {
+              const float c = wc[p.row];
+#pragma unroll
+              for (int q = 0; q < kShort; ++q)
+                if (p.ii[q] >= 0) add(p.ii[q], c * p.vv[q]);
+            });
+      } else {
       for (int r = warp; r < m; r += nwarps) {
         const int b = seg[r], e = seg[m + r];
         const float c = wc[r];
@@ -543,6 +682,7 @@ __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_lcg(
                         });
         }
       }
+      }  // burst walk
     };
     const int64_t gbase = int64_t(s) * W;
     const int n = int(min(int64_t(W), d - gbase));
