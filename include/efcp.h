@@ -171,7 +171,10 @@ int efcp_step(efcp_ctx* ctx, const float* grad, float* update, void* stream);
 /*
  * efcp_step_host - the same step for callers whose gradient and update live in host
  * memory (pinned memory gives the best copy rate): copies grad to the device, runs
- * the step, copies the update back, all on `stream`, and waits for the stream.
+ * the step, copies the update back and waits.  For large d the linear combination runs
+ * over four consecutive ranges of coordinates, and every finished range of the update
+ * starts its way to the host (on a stream of the handle's own) while the next range is
+ * still being accumulated.
  *   grad, update: host, d floats each.
  */
 int efcp_step_host(efcp_ctx* ctx, const float* grad, float* update, void* stream);

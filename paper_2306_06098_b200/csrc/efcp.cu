@@ -89,6 +89,8 @@ struct efcp_ctx {
   int32_t* order = nullptr;  // n_slabs slabs, heavy first
   float* stage_g = nullptr;  // efcp_step_host staging
   float* stage_u = nullptr;
+  cudaStream_t copy_stream = nullptr;    // efcp_step_host: device-to-host copies of finished ranges
+  cudaEvent_t host_ev[4] = {nullptr, nullptr, nullptr, nullptr};
   int last_cuda = 0;
   int launches = 0;
   unsigned long long* dbg_bad = nullptr;  // EFCP_DEBUG_CHECKS: violations found after a step
@@ -109,6 +111,8 @@ namespace {
 
 constexpr int kSpParts = 32;  // second-level partial sums of the scalar products
 constexpr int kMaxCoopBlocks = 1024;  // largest grid of the cooperative kernels
+constexpr int kHostRanges = 4;  // efcp_step_host: ranges of slabs that leave for the host one by one
+static_assert(kHostRanges == sizeof(efcp_ctx::host_ev) / sizeof(cudaEvent_t), "one event per range");
 
 struct Sizes {
   int W, n_slabs, n_chunks, grid_slab;
@@ -216,6 +220,12 @@ void free_all(efcp_ctx* ctx) {
   ctx->allocs.clear();
   for (cudaEvent_t ev : ctx->prof_ev) cudaEventDestroy(ev);
   ctx->prof_ev.clear();
+  for (cudaEvent_t& ev : ctx->host_ev) {
+    if (ev) cudaEventDestroy(ev);
+    ev = nullptr;
+  }
+  if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
+  ctx->copy_stream = nullptr;
 }
 
 inline void prof_mark(efcp_ctx* ctx, int which, cudaStream_t st) {
@@ -699,7 +709,10 @@ int launch_ggt(efcp_ctx* ctx, int slot, cudaStream_t st) {
 }
 
 // Linear combination of the window rows into `update` (or straight into the parameters).
-int launch_lcg(efcp_ctx* ctx, float* update, LcgApply ap, cudaStream_t st) {
+// count < 0: all slabs, heavy first.  Otherwise the slabs slab0 .. slab0 + count - 1 in
+// their natural order, with work counter number `ctr` (1..15).
+int launch_lcg(efcp_ctx* ctx, float* update, LcgApply ap, cudaStream_t st, int slab0 = 0,
+               int count = -1, int ctr = 1) {
   const int64_t k = ctx->k, d = ctx->d;
   const int m = ctx->m;
   const Vecs v = vecs_of(ctx);
@@ -709,14 +722,17 @@ int launch_lcg(efcp_ctx* ctx, float* update, LcgApply ap, cudaStream_t st) {
   const bool uvec = (reinterpret_cast<uintptr_t>(update) & 15) == 0;
   const float inv_lambda = 1.0f / ctx->lambda;
   const double* dw = ggt ? nullptr : v.dw;
+  const int n_launch = count < 0 ? ctx->n_slabs : count;
+  const int grid = std::min(ctx->grid_slab, n_launch);
+  const int32_t* order = count < 0 ? ctx->order : nullptr;
 #define EFCP_LCG_LAUNCH1(VEC, ACC, VT, SHORT, VPTR)                                            \
-  k_lcg<VEC, ACC, VT, false, SHORT><<<ctx->grid_slab, kSlabThreads, smem, st>>>(               \
-      ctx->R, VPTR, ctx->offs, k, m, ctx->W, ctx->n_slabs, v.w, dw, v.wfin, update, d,         \
-      ctx->slab_ctr + 1, ctx->order, ctx->e, inv_lambda, ap)
+  k_lcg<VEC, ACC, VT, false, SHORT><<<grid, kSlabThreads, smem, st>>>(                         \
+      ctx->R, VPTR, ctx->offs, k, m, ctx->W, n_launch, v.w, dw, v.wfin, update, d,             \
+      ctx->slab_ctr + ctr, order, slab0, ctx->e, inv_lambda, ap)
 #define EFCP_LCG_FIXED_LAUNCH1(VEC, VT, SHORT, VPTR)                                            \
-  k_lcg<VEC, false, VT, true, SHORT><<<ctx->grid_slab, kSlabThreads, smem, st>>>(              \
-      ctx->R, VPTR, ctx->offs, k, m, ctx->W, ctx->n_slabs, v.w, dw, v.wfin, update, d,         \
-      ctx->slab_ctr + 1, ctx->order, ctx->e, inv_lambda, ap, ctx->vmax, ctx->lcg_redo,         \
+  k_lcg<VEC, false, VT, true, SHORT><<<grid, kSlabThreads, smem, st>>>(                        \
+      ctx->R, VPTR, ctx->offs, k, m, ctx->W, n_launch, v.w, dw, v.wfin, update, d,             \
+      ctx->slab_ctr + ctr, order, slab0, ctx->e, inv_lambda, ap, ctx->vmax, ctx->lcg_redo,     \
       ctx->lcg_tol2)
 #define EFCP_LCG_LAUNCH(VEC, ACC, VT, VPTR)                                                    \
   do {                                                                                         \
@@ -777,7 +793,11 @@ int launch_debug_checks(efcp_ctx* ctx, int slot, cudaStream_t st) {
 
 // One step: five launches (six for Sparse GGT).  With ap.theta set the linear combination
 // updates the parameters in place of writing u (update may then be NULL).
-int step_impl(efcp_ctx* ctx, const float* grad, float* update, void* stream_, LcgApply ap) {
+// host_update != nullptr (efcp_step_host): the linear combination runs in kHostRanges launches
+// over consecutive ranges of slabs, and every finished range of `update` starts its copy to
+// host_update on the handle's copy stream while the next range is being accumulated.
+int step_impl(efcp_ctx* ctx, const float* grad, float* update, void* stream_, LcgApply ap,
+              float* host_update = nullptr) {
   if (!ctx || !grad || (!update && !ap.theta) || grad == update) return EFCP_EINVAL;
   if (ctx->shard_tot) return EFCP_EINVAL;  // a shard steps through efcp_shard_phase
   cudaStream_t st = static_cast<cudaStream_t>(stream_);
@@ -809,7 +829,23 @@ int step_impl(efcp_ctx* ctx, const float* grad, float* update, void* stream_, Lc
   }
   if (ggt) EFCP_TRY(launch_ggt(ctx, slot, st));
   prof_mark(ctx, 3, st);
-  EFCP_TRY(launch_lcg(ctx, update, ap, st));
+  if (host_update && ctx->n_slabs >= kHostRanges * ctx->num_sms) {
+    for (int q = 0; q < kHostRanges; ++q) {
+      const int s0 = int(int64_t(ctx->n_slabs) * q / kHostRanges);
+      const int s1 = int(int64_t(ctx->n_slabs) * (q + 1) / kHostRanges);
+      EFCP_TRY(launch_lcg(ctx, update, ap, st, s0, s1 - s0, 1 + q));
+      EFCP_CUDA(cudaEventRecord(ctx->host_ev[q], st));
+      EFCP_CUDA(cudaStreamWaitEvent(ctx->copy_stream, ctx->host_ev[q], 0));
+      const int64_t lo = int64_t(s0) * ctx->W, hi = std::min<int64_t>(ctx->d, int64_t(s1) * ctx->W);
+      EFCP_CUDA(cudaMemcpyAsync(host_update + lo, update + lo, size_t(hi - lo) * 4,
+                                cudaMemcpyDeviceToHost, ctx->copy_stream));
+    }
+  } else {
+    EFCP_TRY(launch_lcg(ctx, update, ap, st));
+    if (host_update)
+      EFCP_CUDA(cudaMemcpyAsync(host_update, update, size_t(ctx->d) * 4, cudaMemcpyDeviceToHost,
+                                st));
+  }
   prof_mark(ctx, 4, st);
   if (ctx->flags & EFCP_DEBUG_CHECKS) EFCP_TRY(launch_debug_checks(ctx, slot, st));
   if (ctx->prof_on && ctx->prof_n < ctx->prof_cap) ++ctx->prof_n;
@@ -987,11 +1023,16 @@ int efcp_step_host(efcp_ctx* ctx, const float* grad, float* update, void* stream
     if ((rc = dev_alloc(ctx, &ctx->stage_g, ctx->d * 4))) return rc;
     if ((rc = dev_alloc(ctx, &ctx->stage_u, ctx->d * 4))) return rc;
   }
+  if (!ctx->copy_stream) {
+    EFCP_CUDA(cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking));
+    for (cudaEvent_t& ev : ctx->host_ev) EFCP_CUDA(cudaEventCreateWithFlags(&ev, cudaEventDisableTiming));
+  }
   EFCP_CUDA(cudaMemcpyAsync(ctx->stage_g, grad, size_t(ctx->d) * 4, cudaMemcpyHostToDevice, st));
-  const int rc = efcp_step(ctx, ctx->stage_g, ctx->stage_u, stream_);
+  const int rc = step_impl(ctx, ctx->stage_g, ctx->stage_u, stream_, LcgApply{nullptr, 0.f, 0.f},
+                           update);
   if (rc != EFCP_OK) return rc;
-  EFCP_CUDA(cudaMemcpyAsync(update, ctx->stage_u, size_t(ctx->d) * 4, cudaMemcpyDeviceToHost, st));
   EFCP_CUDA(cudaStreamSynchronize(st));
+  EFCP_CUDA(cudaStreamSynchronize(ctx->copy_stream));
   return EFCP_OK;
 }
 

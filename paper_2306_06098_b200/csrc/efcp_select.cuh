@@ -426,7 +426,7 @@ __global__ void __launch_bounds__(kSelThreads) k_select_insert(const SelectArgs 
       if (blockIdx.x == gridDim.x - 1) {
         slab_order_block(A.colsum, A.n_slabs, A.order, reinterpret_cast<int*>(sel_smraw),
                          reinterpret_cast<int*>(sm));
-        if (tid < 2) A.slab_ctr[tid] = 0;  // work counters of the two slab kernels
+        if (tid < 16) A.slab_ctr[tid] = 0;  // work counters of the slab kernels' launches
         __syncthreads();
       }
       layout_row_slabs(A.sel_idx, A.sel_val, A.W, A.n_slabs, A.m, A.slot, A.offs, A.row_idx,

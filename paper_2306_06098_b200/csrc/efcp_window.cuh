@@ -603,7 +603,8 @@ __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_lcg(
     const uint16_t* __restrict__ R, const VT* __restrict__ V, const int32_t* __restrict__ offs,
     int64_t k, int m, int W, int n_slabs, const double* __restrict__ w64,
     const double* __restrict__ dw64, double* __restrict__ w_out, float* __restrict__ u,
-    int64_t d, int* ctr, const int32_t* __restrict__ order, const float* __restrict__ xi,
+    int64_t d, int* ctr, const int32_t* __restrict__ order, int slab0,
+    const float* __restrict__ xi,
     float inv_lambda, LcgApply ap, const float* __restrict__ vmax = nullptr,
     unsigned long long* __restrict__ redo_count = nullptr, double fixed_tol2 = 1e-10) {
   static_assert(!(FIXED && ACC), "the fixed-point accumulator starts from zero");
@@ -623,7 +624,9 @@ __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_lcg(
   for (int i = tid; i < (W >> 2); i += blockDim.x) acc4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
   __shared__ int s_next;
   for (int t = blockIdx.x; t < n_slabs;) {  // t: position in the hand-out order
-    const int s = order[t];
+    // order == nullptr: this launch covers the slabs slab0 .. slab0 + n_slabs - 1 in their
+    // natural order (the host entry point launches ranges so that finished ranges can leave)
+    const int s = order ? order[t] : slab0 + t;
     __syncthreads();
     if (tid == 0) s_next = int(gridDim.x) + atomicAdd(ctr, 1);
     for (int r = tid; r < m; r += blockDim.x) {

@@ -475,6 +475,32 @@ def test_host_entry_point_matches_device_entry_point():
         assert rel_l2(uh.numpy(), ud.cpu().numpy()) <= 1e-5
 
 
+def test_host_entry_point_sends_finished_ranges_early_at_large_d():
+    """Above about 600 slabs efcp_step_host runs the linear combination over four ranges of
+    slabs and copies every finished range to the host while the next is accumulated: the
+    result must be that of the device entry point."""
+    B = _binding()
+    d, m, k = 26_000_003, 2, 26_000
+    rng = np.random.default_rng(16)
+    a, b = B.Efcp(d, m, k, 1e-3), B.Efcp(d, m, k, 1e-3)
+    gh = torch.empty(d, dtype=torch.float32).pin_memory()
+    uh = torch.empty(d, dtype=torch.float32).pin_memory()
+    gd = torch.empty(d, dtype=torch.float32, device="cuda")
+    ud = torch.empty(d, dtype=torch.float32, device="cuda")
+    for t in range(4):
+        gh.copy_(torch.from_numpy(rng.standard_normal(d).astype(np.float32)))
+        gd.copy_(gh)
+        uh.fill_(float("nan"))
+        a.step(gd, ud)
+        b.step_host(gh, uh)
+        assert np.array_equal(bits(a.error()), bits(b.error()))
+        assert torch.isfinite(uh).all()
+        assert torch.equal(uh, ud.cpu())  # integer accumulation: no dependence on the slab order
+    assert a.fixed_point_fallbacks() == 0 and b.fixed_point_fallbacks() == 0
+    a.close()
+    b.close()
+
+
 # ---- full size, in the launch configuration the benchmark times
 def _device_stream(w, device="cuda"):
     return gradgen.GradStream.for_workload(w, device)
