@@ -35,12 +35,12 @@ UNIT = "steps/s"
 # profiles/ (dram__bytes_read.sum + dram__bytes_write.sum), keyed by workload; None until
 # a capture of that workload exists.  Scaled from a smaller capture where noted there.
 # Captured on a quarter-size copy of c4_bert_base (same slab width and segment lengths, see
-# profiles/): DRAM traffic / bytes to move was 1.104 for k_sp_rows and 1.078 for k_lcg, and it
+# profiles/): DRAM traffic / bytes to move was 1.103 for k_sp_rows and 1.079 for k_lcg, and it
 # is proportional to the bytes streamed, so the C4 figures are those ratios times the C4 bytes
 # per launch.
 NCU_TRAFFIC_BYTES = {
-    "c4_bert_base": {"sp": int(1.104 * 6 * 1024 * 1_094_822),
-                     "lcg": int(1.078 * (6 * 1024 * 1_094_822 + 4 * 109_482_240))},
+    "c4_bert_base": {"sp": int(1.103 * 6 * 1024 * 1_094_822),
+                     "lcg": int(1.079 * (6 * 1024 * 1_094_822 + 4 * 109_482_240))},
 }
 
 
