@@ -59,8 +59,6 @@ struct efcp_ctx {
   // scratch
   uint32_t* hist = nullptr;  // kBins1 + kBins2 + kBins3
   int32_t* chunk_off = nullptr;
-  int32_t* cand_idx = nullptr;
-  float* cand_val = nullptr;
   uint16_t* bk_off = nullptr;  // speculative candidate buckets, one of kChunk entries per chunk
   float* bk_val = nullptr;
   bool spec = true;            // EFCP_NO_SPEC=1 forces the two-pass candidate path
@@ -350,8 +348,6 @@ int alloc_all(efcp_ctx* ctx) {
   EFCP_ALLOC(chunk_off, int64_t(n_chunks + 1) * 4);
   EFCP_ALLOC(sel_gt, int64_t(n_chunks + 1) * 4);
   EFCP_ALLOC(sel_eq, int64_t(n_chunks + 1) * 4);
-  EFCP_ALLOC(cand_idx, d * 4);
-  EFCP_ALLOC(cand_val, d * 4);
   EFCP_ALLOC(bk_off, int64_t(n_chunks) * kChunk * 2);
   EFCP_ALLOC(bk_val, int64_t(n_chunks) * kChunk * 4);
   EFCP_ALLOC(sel_idx, k * 4);
