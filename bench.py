@@ -242,6 +242,44 @@ def run_reference(args, world, rank):
     print(json.dumps(line), flush=True)
 
 
+def run_local_shards(args):
+    """The coordinate-sharded step with all shards on one GPU of this process (exchange buffers
+    summed on the device): what splitting the step at its exchange points costs, without any
+    interconnect.  Not the benchmark's metric: a diagnostic line."""
+    from paper_2306_06098_b200 import binding, sharded
+    torch.cuda.set_device(0)
+    w = get_workload(args.workload)
+    n = args.local_shards
+    shards, ranges = sharded.create_local_shards(binding, w.d, w.m, w.k, w.lam, n)
+    stepper = sharded.ShardedStep(shards, sharded.sum_in_process)
+    gs = gradgen.GradStream.for_workload(w, "cuda")
+    ubuf = torch.empty(w.d, dtype=torch.float32, device="cuda")
+    split = lambda t: [t[lo:hi] for lo, hi in ranges]
+    prefill = w.m if args.prefill < 0 else args.prefill
+    for _ in range(prefill):
+        stepper.step(split(gs.next()), split(ubuf))
+    pool = [gs.next().clone() for _ in range(min(args.steps + args.warmup, 64))]
+    del gs
+    for i in range(args.warmup):
+        stepper.step(split(pool[i % len(pool)]), split(ubuf))
+    torch.cuda.synchronize()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for i in range(args.steps):
+        stepper.step(split(pool[(args.warmup + i) % len(pool)]), split(ubuf))
+    ev1.record()
+    torch.cuda.synchronize()
+    ms = ev0.elapsed_time(ev1) / args.steps
+    assert all(s.status() == 0 for s in shards)
+    print(json.dumps({"metric": METRIC, "value": 1e3 / ms, "unit": UNIT, "n_gpus": 1,
+                      "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
+                      "higher_is_better": True, "data": "synthetic", "dtype": "f32",
+                      "config": {"workload": w.name, "d": w.d, "m": w.m, "k": w.k,
+                                 "parallelism": f"{n} coordinate shards on one GPU, buffers "
+                                                f"summed on the device (no interconnect)",
+                                 "ranges": ranges, "prefill_steps": prefill}}), flush=True)
+
+
 def get_workload(name):
     if name.startswith("custom:"):
         f = name.split(":", 1)[1].split(",")
@@ -281,6 +319,9 @@ def main():
                     help="with --apply-update: clip |u| to this norm (adds the norm kernels)")
     ap.add_argument("--prefill", type=int, default=-1,
                     help="untimed steps before warm-up; -1 = m (fill the whole window)")
+    ap.add_argument("--local-shards", type=int, default=0,
+                    help="diagnostic: run the coordinate-sharded step with this many shards, all "
+                         "on GPU 0 of this process")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--cpu-steps", type=int, default=5)
     ap.add_argument("--cpu-single-steps", type=int, default=2,
@@ -292,6 +333,9 @@ def main():
     if args.impl == "reference":
         # rank 0 alone runs the oracle; no process group is needed for that
         run_reference(args, int(os.environ.get("WORLD_SIZE", "1")), int(os.environ.get("RANK", "0")))
+        return
+    if args.local_shards > 1:
+        run_local_shards(args)
         return
     world, rank, local = dist_setup(args.gpus)
 

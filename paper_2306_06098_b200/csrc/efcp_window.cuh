@@ -220,11 +220,7 @@ __device__ __forceinline__ void prefetch_segment(const uint16_t* Rr, const VT* V
   const char* p = (lane < 16) ? reinterpret_cast<const char*>(Rr + b)
                               : reinterpret_cast<const char*>(Vr + b);
   const int bytes = (e - b) * (lane < 16 ? 2 : int(sizeof(VT)));
-#ifdef EFCP_PREFETCH_L1
-  if (half * 128 < bytes) asm volatile("prefetch.global.L1 [%0];" ::"l"(p + half * 128));
-#else
   if (half * 128 < bytes) asm volatile("prefetch.global.L2 [%0];" ::"l"(p + half * 128));
-#endif
 }
 
 // The last pass over a segment: N groups of 32 entries (1 <= N <= kDepth), only the last of
