@@ -1,13 +1,16 @@
-// Error feedback + exact global Top-k (Algorithm 1: the error-feedback, compression and error-update statements; Section 3.1).
+// Error feedback and the building blocks of the exact global Top-k (Algorithm 1: the
+// error-feedback, compression and error-update statements; Section 3.1).
 //
 // Selection is a most-significant-digit radix select on the 31-bit magnitude key
-// (12 + 10 + 9 bits).  Digit 1 is histogrammed while a = xi + g is formed; every
-// entry at or above the threshold bin of digit 1 is then compacted, in index order,
-// into a candidate list, and digits 2 and 3 are resolved on that list only.  The
-// final ordered compaction writes the row (ascending indices) straight into the
-// ring slot and zeroes the kept coordinates of xi.  Ties at the threshold key are
-// taken in index order, so the result is the unique "first k of a sort by
-// (|a| descending, index ascending)".
+// (12 + 10 + 9 bits).  Ties at the threshold key are taken in index order, so the result is
+// the unique "first k of a sort by (|a| descending, index ascending)".
+//
+// Two users:
+//   * a step: k_ef_spec (below) forms a = xi + g, histograms digit 1 and leaves the
+//     speculative buckets; everything after it is the cooperative kernel of efcp_select.cuh;
+//   * efcp_topk_static, the stand-alone selection on a caller's vector: the chain of small
+//     kernels in this file (k_pick, k_count_chunks, k_scan_counts, k_compact_cand, k_hist3,
+//     k_count_sel, k_scan_sel), which compacts the candidates into a dense list first.
 #pragma once
 
 #include "efcp_common.cuh"
@@ -17,11 +20,10 @@ namespace efcp {
 // Speculation.  The threshold of the selection moves little from one step to the next, so
 // the kernel that forms a = xi + g already sets aside, chunk by chunk, every entry at or
 // above a guessed bin of digit 1 (the previous step's threshold bin minus kSpecMargin).
-// k_pick<.., 1> then knows the true threshold bin: if the guess was not above it and did
-// not let in too many entries, the candidate list is compacted from these buckets and the
-// accumulator is not read again; otherwise (first step, threshold fell by more than the
-// margin) the two-pass path below, k_count_chunks + k_compact_cand, runs as before.  Both
-// routes give the same exact selection.
+// Once the true threshold bin is known the guess is judged: if it was not above the bin
+// and did not let in too many entries, the buckets are the candidates and the accumulator is
+// not read again; otherwise (first step, threshold fell by more than the margin) they are
+// rebuilt with the exact bin.  Both routes give the same exact selection.
 constexpr int kSpecMargin = 1;
 
 __device__ __forceinline__ uint32_t spec_guess(const Scalars* sc, int enable) {
@@ -107,38 +109,6 @@ __global__ void __launch_bounds__(kChunkThreads, 8) k_ef_spec(
     if (c) atomicAdd(&hist1[i], c);
   }
   if (bad) atomicOr(&sc->status, kStNonFinite);
-}
-
-// The candidate list from the speculative buckets (runs only when sc->spec_ok): chunk ch's
-// entries go to cand[off[ch] ...), digit 2 of the entries inside the true threshold bin is
-// histogrammed.  One warp per chunk.
-__global__ void __launch_bounds__(256) k_compact_buckets(
-    const uint16_t* __restrict__ bk_off, const float* __restrict__ bk_val, const Scalars* sc,
-    const int32_t* __restrict__ off, int32_t* __restrict__ cand_idx, float* __restrict__ cand_val,
-    uint32_t* __restrict__ hist2, int n_chunks) {
-  if (!sc->spec_ok) return;
-  __shared__ uint32_t h[kBins2];
-  for (int i = threadIdx.x; i < kBins2; i += blockDim.x) h[i] = 0u;
-  __syncthreads();
-  const uint32_t b1 = sc->b1;
-  const int lane = threadIdx.x & 31, wpb = blockDim.x >> 5;
-  for (int ch = blockIdx.x * wpb + (threadIdx.x >> 5); ch < n_chunks; ch += gridDim.x * wpb) {
-    const int o0 = off[ch], n = off[ch + 1] - o0;
-    const uint16_t* bo = bk_off + int64_t(ch) * kChunk;
-    const float* bv = bk_val + int64_t(ch) * kChunk;
-    for (int i = lane; i < n; i += 32) {
-      const float v = bv[i];
-      cand_idx[o0 + i] = int32_t(int64_t(ch) * kChunk + bo[i]);
-      cand_val[o0 + i] = v;
-      const uint32_t key = mag_key(v);
-      if ((key >> kShift1) == b1) atomicAdd(&h[(key >> kShift2) & (kBins2 - 1)], 1u);
-    }
-  }
-  __syncthreads();
-  for (int i = threadIdx.x; i < kBins2; i += blockDim.x) {
-    const uint32_t cc = h[i];
-    if (cc) atomicAdd(&hist2[i], cc);
-  }
 }
 
 // Finds the threshold bin of one digit: the bin b with count(bins > b) < k_rem <=
@@ -228,7 +198,7 @@ __global__ void __launch_bounds__(kChunkThreads) k_count_chunks(const float* __r
                                                                  int32_t* __restrict__ cnt,
                                                                  int n_chunks) {
   __shared__ int sm[33];
-  if (sc->spec_ok) return;  // the speculative buckets already hold the counts
+  if (sc->spec_ok) return;  // (never set for the stand-alone selection)
   const uint32_t b1 = sc->b1;
   for (int ch = blockIdx.x; ch < n_chunks; ch += gridDim.x) {
     const int64_t base = int64_t(ch) * kChunk + threadIdx.x * kPerThread;
@@ -302,7 +272,7 @@ __global__ void __launch_bounds__(kChunkThreads, 8) k_compact_cand(
     int n_chunks) {
   __shared__ uint32_t h[kBins2];
   __shared__ int sm[33];
-  if (sc->spec_ok) return;  // k_compact_buckets builds the list instead
+  if (sc->spec_ok) return;  // (never set for the stand-alone selection)
   for (int i = threadIdx.x; i < kBins2; i += blockDim.x) h[i] = 0u;
   __syncthreads();
   const uint32_t b1 = sc->b1;
