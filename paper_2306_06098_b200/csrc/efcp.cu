@@ -1363,7 +1363,7 @@ __global__ void __launch_bounds__(512) k_hist1_only(const float* __restrict__ a,
   }
 }
 
-// Final ordered compaction of k_write_sel without the error-buffer update: the kept
+// Final ordered compaction of the stand-alone selection: the kept
 // (index, value) pairs in ascending index order.
 __global__ void __launch_bounds__(kChunkThreads) k_write_sel_only(
     const int32_t* __restrict__ cand_idx, const float* __restrict__ cand_val, const Scalars* sc,

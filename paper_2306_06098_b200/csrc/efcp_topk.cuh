@@ -387,68 +387,4 @@ __global__ void __launch_bounds__(1024) k_scan_sel(int32_t* __restrict__ cnt_gt,
   }
 }
 
-// Final ordered compaction: writes the kept (index, value) pairs in ascending index order
-// and sets the kept coordinates of xi to a - c: +0, or with bfloat16 window values
-// (values_bf16) the rounding residue a - bf16(a).
-__global__ void __launch_bounds__(kChunkThreads) k_write_sel(
-    const int32_t* __restrict__ cand_idx, const float* __restrict__ cand_val, const Scalars* sc,
-    const int32_t* __restrict__ off_gt, const int32_t* __restrict__ pre_eq,
-    int32_t* __restrict__ row_idx, float* __restrict__ row_val, float* __restrict__ e,
-    int64_t k_total, int values_bf16) {
-  __shared__ int sm[33];
-  const int n = sc->n_cand;
-  const uint32_t T = sc->T;
-  const int n_eq = int(sc->n_eq);
-  const int n_cc = (n + kChunk - 1) / kChunk;
-  for (int c = blockIdx.x; c < n_cc; c += gridDim.x) {
-    const int64_t base = int64_t(c) * kChunk + threadIdx.x * kPerThread;
-    float v[kPerThread];
-    bool ok[kPerThread];
-    load_chunk8(cand_val, base, n, v, ok);
-    int32_t ci[kPerThread];  // fetched now, with the values, not after the scans
-#pragma unroll
-    for (int q = 0; q < kPerThread; ++q) ci[q] = ok[q] ? cand_idx[base + q] : 0;
-    const int eq_before_chunk = pre_eq[c];
-    const int gt_before_chunk = off_gt[c];
-    bool is_eq[kPerThread];
-    int my_eq = 0;
-#pragma unroll
-    for (int q = 0; q < kPerThread; ++q) {
-      const uint32_t key = mag_key(v[q]);
-      is_eq[q] = ok[q] && key == T;
-      ok[q] = ok[q] && key > T;
-      my_eq += is_eq[q] ? 1 : 0;
-    }
-    int tot;
-    int eq_rank = eq_before_chunk + block_excl_scan<int>(my_eq, &tot, sm);
-    int my_sel = 0;
-#pragma unroll
-    for (int q = 0; q < kPerThread; ++q) {
-      if (is_eq[q]) {
-        ok[q] = eq_rank < n_eq;
-        ++eq_rank;
-      }
-      my_sel += ok[q] ? 1 : 0;
-    }
-    int64_t pos = int64_t(gt_before_chunk) + min(eq_before_chunk, n_eq) +
-                  block_excl_scan<int>(my_sel, &tot, sm);
-#pragma unroll
-    for (int q = 0; q < kPerThread; ++q) {
-      if (ok[q] && pos < k_total) {
-        const int32_t j = ci[q];
-        row_idx[pos] = j;
-        if (values_bf16) {  // c holds the rounded value, the residue stays in xi (exact)
-          const float r = bf16_to_float(bf16_bits_rn(v[q]));
-          row_val[pos] = r;
-          e[j] = __fsub_rn(v[q], r);
-        } else {
-          row_val[pos] = v[q];
-          e[j] = 0.0f;
-        }
-        ++pos;
-      }
-    }
-  }
-}
-
 }  // namespace efcp

@@ -532,51 +532,6 @@ __global__ void __launch_bounds__(kSlabThreads, kSlabBlocksPerSM) k_sp_rows(
   }
 }
 
-// part2[y][r] = sum of slab_part[s][r] over s = y, y + gridDim.y, ... in increasing s.
-__global__ void __launch_bounds__(128) k_sp_reduce(const double* __restrict__ slab_part,
-                                                    int n_slabs, int m,
-                                                    double* __restrict__ part2) {
-  const int r = blockIdx.x * blockDim.x + threadIdx.x;
-  if (r >= m) return;
-  const int step = gridDim.y;
-  double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
-  int s = blockIdx.y;
-  for (; s + 3 * step < n_slabs; s += 4 * step) {
-    a0 += slab_part[int64_t(s) * m + r];
-    a1 += slab_part[int64_t(s + step) * m + r];
-    a2 += slab_part[int64_t(s + 2 * step) * m + r];
-    a3 += slab_part[int64_t(s + 3 * step) * m + r];
-  }
-  for (; s < n_slabs; s += step) a0 += slab_part[int64_t(s) * m + r];
-  part2[int64_t(blockIdx.y) * m + r] = (a0 + a1) + (a2 + a3);
-}
-
-// delta[r] = sum of the per-block partials in block order; S row/column `slot` := delta
-// (Section 2.1: S_{i,:} = S_{:,i} = G g); aprime = delta with entry `slot` cleared.
-// With rhs != null (x = a_t): `partial` rows are 2 m long, the second half sums to
-// q = G xi_t, and rhs = m e_slot - q / lambda (the right-hand side of the weights, see
-// efcp_mxm.cuh).
-__global__ void __launch_bounds__(128) k_sp_finish(const double* __restrict__ partial, int nparts,
-                                                    int m, int slot, double* __restrict__ delta,
-                                                    double* __restrict__ S,
-                                                    double* __restrict__ aprime,
-                                                    double* __restrict__ rhs, double lambda) {
-  const int r = blockIdx.x * blockDim.x + threadIdx.x;
-  if (r >= m) return;
-  const int stride = rhs ? 2 * m : m;
-  double s = 0.0;
-  for (int p = 0; p < nparts; ++p) s += partial[int64_t(p) * stride + r];
-  delta[r] = s;
-  S[int64_t(slot) * m + r] = s;
-  S[int64_t(r) * m + slot] = s;
-  aprime[r] = r == slot ? 0.0 : s;
-  if (rhs) {
-    double q = 0.0;
-    for (int p = 0; p < nparts; ++p) q += partial[int64_t(p) * stride + m + r];
-    rhs[r] = (r == slot ? double(m) : 0.0) - q / lambda;
-  }
-}
-
 // Linear combination of the window rows, u = sum_r w_r row_r, one slab at a time in a
 // shared-memory accumulator (Eq. (2) in the form that has no x/lambda term, see
 // efcp_mxm.cuh).  Every element of u is written exactly once.
