@@ -98,3 +98,24 @@ def test_footprint_formula_reproduces_the_papers_memory_figures():
     assert abs(dense / (round(b16 / d, -1) * d) - gold["saving_bf16"]) < 0.05
     from paper_2306_06098_b200 import gradgen
     assert 4 * 1024 * gradgen.C4.d // 2 ** 30 == gold["bert_base_dense_window_gib"]  # 417.6
+
+
+def test_workspace_size_is_computed_without_a_device():
+    """efcp_workspace_bytes runs the handle's own allocation list with an arena that only adds
+    up sizes; it needs no GPU (it assumes a B200's SM count then) and tracks the options."""
+    from paper_2306_06098_b200 import binding as B
+    from paper_2306_06098_b200 import gradgen
+    w = gradgen.C4
+    base = B.workspace_bytes(w.d, w.m, w.k)
+    assert base == B.state_bytes(w.d, w.m, w.k) > 0
+    mk = w.m * w.k
+    # state the method defines: xi, (I, V); plus the 16-bit index stream the kernels read
+    assert base > 4 * w.d + 10 * mk
+    assert base < 4 * w.d + 10 * mk + 12 * w.d  # scratch: buckets, tables, m x m (a few GB at most)
+    assert B.workspace_bytes(w.d, w.m, w.k, B.VALUES_BF16) - base >= 2 * mk          # second value stream
+    assert B.workspace_bytes(w.d, w.m, w.k, B.LCG_FP32) < base                        # no bound table
+    assert B.workspace_bytes(w.d, w.m, w.k, 0, 8192) > base                           # rows a little longer
+    for bad in ((0, 1, 1), (10, 0, 1), (10, 1, 11), (2 ** 31, 1, 1)):
+        assert B.workspace_bytes(*bad) == -1
+    assert B.workspace_bytes(1000, 4, 10, 1 | 2) == -1  # flags that cannot be combined
+    assert B.workspace_bytes(1000, 4, 10, 0, 48) == -1   # block length must be a multiple of 32
