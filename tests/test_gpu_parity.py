@@ -475,6 +475,40 @@ def test_host_entry_point_matches_device_entry_point():
         assert rel_l2(uh.numpy(), ud.cpu().numpy()) <= 1e-5
 
 
+def test_inverse_does_not_drift_over_twenty_turns_of_the_ring():
+    """The explicitly kept inverse is only ever updated, never rebuilt.  20,000 steps of the
+    ResNet-20-shaped stream (about 19,000 row replacements in a full m = 1024 window, the order
+    of a whole training run) must leave the residual of the m x m solve where it started, and
+    the update must still solve the defining system at the end."""
+    B = _binding()
+    w = gradgen.C2
+    gs = _device_stream(w)
+    gpu = B.Efcp(w.d, w.m, w.k, w.lam)
+    u = torch.empty(w.d, dtype=torch.float32, device="cuda")
+    worst = 0.0
+    for t in range(20_000):
+        gpu.step(gs.next(), u)
+        if t % 500 == 499:
+            worst = max(worst, gpu.last_residual())
+    assert gpu.status() == 0
+    print(f"m x m residual over 20000 steps of {w.name}: worst {worst:.3e}")
+    assert worst < 1e-9
+    lam = float(np.float32(w.lam))
+    I, V = gpu.window()
+    slot = (gpu.step_count - 1) % w.m
+    ud = u.double()
+    x = torch.zeros(w.d, dtype=torch.float64, device="cuda")
+    x.index_add_(0, I[slot].long(), V[slot].double())
+    Fu = lam * ud
+    bound = lam * ud.abs()
+    for r in range(w.m):
+        idx, val = I[r].long(), V[r].double()
+        Fu.index_add_(0, idx, val * ((val * ud[idx]).sum() / w.m))
+        bound.index_add_(0, idx, val.abs() * ((val.abs() * ud[idx].abs()).sum() / w.m))
+    assert float((Fu - x).norm()) <= 4 * 2.0 ** -24 * float(bound.norm())
+    gpu.close()
+
+
 def test_host_entry_point_sends_finished_ranges_early_at_large_d():
     """Above about 600 slabs efcp_step_host runs the linear combination over four ranges of
     slabs and copies every finished range to the host while the next is accumulated: the
