@@ -42,7 +42,7 @@ constexpr int kSelGroup = 8;  // chunks whose buckets a warp walks as one list
 
 // dynamic shared memory: the larger of one histogram of digit 1 and the staging of phase 5
 constexpr size_t kSelLayoutBytes =
-    size_t(kSelWarps) * (kLayoutChunk * (4 + 4 + 2) + 32 * 4);
+    size_t(kSelWarps) * kLayoutWarpBytes;
 constexpr size_t kSelSmemBytes = kSelLayoutBytes > size_t(kBins1) * 4 ? kSelLayoutBytes
                                                                       : size_t(kBins1) * 4;
 
@@ -431,7 +431,7 @@ __global__ void __launch_bounds__(kSelThreads) k_select_insert(const SelectArgs 
       }
       layout_row_slabs(A.sel_idx, A.sel_val, A.W, A.n_slabs, A.m, A.slot, A.offs, A.row_idx,
                        A.row_rel, A.row_val, A.row_v16, A.vmax,
-                       sel_smraw + size_t(warp) * (kLayoutChunk * 10 + 128),
+                       sel_smraw + size_t(warp) * kLayoutWarpBytes,
                        int(blockIdx.x) * kSelWarps + warp, int(gridDim.x) * kSelWarps);
     }
   }

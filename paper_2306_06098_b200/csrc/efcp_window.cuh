@@ -36,6 +36,10 @@
 namespace efcp {
 
 constexpr int kLayoutChunk = 512;   // entries permuted together (a multiple of 32)
+constexpr int kLayoutLevels = 64;   // occurrence levels with precomputed ranks (more: slow path)
+// shared memory of one warp of the insert: indices, values, occurrence numbers of a chunk,
+// per-bank counts, per-level bank masks and level starts
+constexpr int kLayoutWarpBytes = kLayoutChunk * 10 + 32 * 4 + kLayoutLevels * 6;
 
 // offs[s][slot] for the new row from its ascending index list of n entries: entry `pos`
 // starts every slab between its predecessor's slab (exclusive) and its own (inclusive); the
@@ -103,7 +107,7 @@ __device__ __forceinline__ void slab_order_block(const int64_t* __restrict__ col
 //   bank-interleaved order described above.  One warp handles one chunk at a time; a slab's
 //   chunks are shared by `wps` warps (1, 2, 4 or 8: as many as there are warps to go round),
 //   warp `gwarp` of `nwarps` taking the (slab, part) pairs gwarp, gwarp + nwarps, ...
-//   smraw: this warp's kLayoutChunk * 10 + 128 bytes of shared memory.  vmax[s][slot] must be
+//   smraw: this warp's kLayoutWarpBytes of shared memory.  vmax[s][slot] must be
 //   zero on entry; it receives the largest magnitude of the segment.
 __device__ __forceinline__ void layout_row_slabs(
     const int32_t* __restrict__ src_idx, const float* __restrict__ src_val, int W, int n_slabs,
@@ -115,6 +119,9 @@ __device__ __forceinline__ void layout_row_slabs(
   float* cv = reinterpret_cast<float*>(smraw + kLayoutChunk * 4);
   uint16_t* cq = reinterpret_cast<uint16_t*>(smraw + kLayoutChunk * 8);
   int* cnt = reinterpret_cast<int*>(smraw + kLayoutChunk * 10);
+  uint32_t* lvl_mask = reinterpret_cast<uint32_t*>(smraw + kLayoutChunk * 10 + 128);
+  uint16_t* lvl_start = reinterpret_cast<uint16_t*>(smraw + kLayoutChunk * 10 + 128 +
+                                                    kLayoutLevels * 4);
   int wps = 1;
   while (wps < 8 && int64_t(n_slabs) * wps * 2 <= nwarps) wps *= 2;
   for (int64_t t = gwarp; t < int64_t(n_slabs) * wps; t += nwarps) {
@@ -147,16 +154,38 @@ __device__ __forceinline__ void layout_row_slabs(
         }
         __syncwarp();
       }
-      // position in the (occurrence, bank) order
+      // position in the (occurrence, bank) order: level q (the q-th entry of every bank that
+      // has one) starts where the levels below it end, and inside it the banks go in order.
+      // Levels and their bank masks are tabulated when there are at most kLayoutLevels.
+      const int my_cnt = cnt[lane];
+      int maxc = my_cnt;
+      for (int o = 16; o > 0; o >>= 1) maxc = max(maxc, __shfl_xor_sync(0xFFFFFFFFu, maxc, o));
+      const bool tabulated = maxc <= kLayoutLevels;
+      if (tabulated) {
+        int start = 0;
+        for (int q = 0; q < maxc; ++q) {
+          const unsigned mk = __ballot_sync(0xFFFFFFFFu, my_cnt > q);
+          if (lane == 0) {
+            lvl_mask[q] = mk;
+            lvl_start[q] = uint16_t(start);
+          }
+          start += __popc(mk);
+        }
+        __syncwarp();
+      }
       for (int a0 = 0; a0 < n; a0 += 32) {
         const int a = a0 + lane;
         if (a < n) {
           const int idx = ci[a], bank = idx & 31, q = cq[a];
           int pos = 0;
+          if (tabulated) {
+            pos = int(lvl_start[q]) + __popc(lvl_mask[q] & ((1u << bank) - 1u));
+          } else {
 #pragma unroll 8
-          for (int bb = 0; bb < 32; ++bb) {
-            const int c = cnt[bb];
-            pos += min(c, q) + ((bb < bank && c > q) ? 1 : 0);
+            for (int bb = 0; bb < 32; ++bb) {
+              const int c = cnt[bb];
+              pos += min(c, q) + ((bb < bank && c > q) ? 1 : 0);
+            }
           }
           dst_idx[c0 + pos] = idx;
           dst_rel[c0 + pos] = uint16_t(idx - s * W);
